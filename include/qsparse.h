@@ -1,0 +1,218 @@
+/*
+ * qsparse.h — C boundary of the Qsparse-local-SGD synchronisation round for one B200.
+ *
+ * The library holds R simulated workers as an R x d fp32 batch in the memory of ONE
+ * GPU and runs, with its own sm_100a kernels, one synchronisation step of
+ * Qsparse-local-SGD (Basu, Data, Karakus, Diggavi; Algorithm 1, and Algorithm 2 for
+ * the asynchronous variant):
+ *
+ *   worker r :  u_r = m_r + (x - xw_r)            argument of the compressor (Alg. 1, worker branch)
+ *               g_r = Q Comp_k(u_r)               composed operator (Section 2.3, Lemmas 1-3;
+ *                                                 per-segment by Corollary 1)
+ *               m_r <- u_r - g_r                  memory update (Alg. 1, worker branch)
+ *               g_r -> wire record                "send g to the master"
+ *   master   :  x <- x - (1/R) sum_r g_r          (Alg. 1, master branch; sum over the
+ *                                                 participating set S in Alg. 2, divisor still R)
+ *               xw_r <- x                         broadcast
+ *
+ * Conventions common to every call
+ *   - All array arguments named "device" are pointers into the memory of the GPU that
+ *     was current when qs_init ran; "host" arrays are ordinary host memory and are
+ *     read before the call returns.  The caller owns every buffer it passes; the
+ *     library owns only its scratch, freed by qs_destroy.
+ *   - x is d floats; xw, mem (and anchors) are R x d floats, row r = worker r,
+ *     rows contiguous (row stride d).  No alignment beyond 4 bytes is required, but
+ *     the 128-bit fast path is taken only when d is a multiple of 4 and the bases are
+ *     16-byte aligned.
+ *   - Calls enqueue work on the stream given to qs_init and return at once.  The
+ *     return value reports argument and launch errors; errors found on the device
+ *     (non-finite input, a bounded wait that ran out) are recorded in a device status
+ *     word that qs_sync_status reads after synchronising the stream.
+ *   - Status codes: QS_OK = 0, negative = error.  Nothing is printed, nothing aborts.
+ *   - worker_mask: host array of R bytes, non-zero = worker takes part; NULL = all.
+ *   - R <= 32, 1 <= k <= d < 2^32, 1 <= s <= 65535, round < 2^56.
+ *
+ * Arithmetic (identical, operation for operation, to the CPU checker under oracle/):
+ *   fp32 with no fused multiply-add; u = mem + (x - xw); Top_k orders by the bit
+ *   pattern of |u| (larger first), ties by lower index, and always keeps exactly k
+ *   coordinates; Rand_k keeps the k smallest (h_i, i) with h_i a Philox4x32-10 word;
+ *   norms are the exactly rounded sum of squares (magnitudes), see qs_compress_feedback.
+ */
+#ifndef QSPARSE_H
+#define QSPARSE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qs_ctx qs_ctx;
+
+enum {
+    QS_OK = 0,
+    QS_INVALID_ARG = -1, /* bad argument; nothing was enqueued                         */
+    QS_ALLOC = -2,       /* scratch allocation failed                                  */
+    QS_CUDA = -3,        /* a CUDA runtime call failed; see qs_last_error              */
+    QS_CAPACITY = -4,    /* caller's wire stride is smaller than qs_wire_words         */
+    QS_NONFINITE = -5,   /* an inf or NaN reached the compressor (device status)       */
+    QS_STATE = -6,       /* call out of order (no buffers bound, nothing compressed)   */
+    QS_TIMEOUT = -7      /* a bounded device-side wait ran out (device status)         */
+};
+
+/* Sparsifiers of Section 2.2. */
+#define QS_TOPK 0
+#define QS_RANDK 1
+/* Quantizers: QSGD s-level stochastic (Definition 1, example 1) composed without scaling
+ * (Lemma 1) or divided by 1 + beta_{k,s} (Lemma 2); Sign scaled by the l1 norm over k
+ * (Definition 2, Lemma 3 with m = 1). */
+#define QS_QSGD 0
+#define QS_QSGD_SCALED 1
+#define QS_SIGN_L1 2
+/* op argument of qs_init */
+#define QS_OP(sparsifier, quantizer) ((sparsifier) | ((quantizer) << 4))
+
+/* Round argument meaning "use the context's counter, then increment it". */
+#define QS_ROUND_AUTO UINT64_MAX
+
+/*
+ * qs_init — create a context for R workers of d coordinates, keeping k per worker with
+ * an s-level quantizer (Section 2; Algorithm 1 line 1 fixes the zero initial state, which
+ * is the caller's to provide in the buffers it binds).
+ *   out          receives the context (host pointer).
+ *   op           QS_OP(sparsifier, quantizer).
+ *   seed         key of the Philox4x32-10 generator; the word for (round, worker,
+ *                element, stream) uses counter (element >> 2, worker, round_lo,
+ *                (round_hi << 8) | stream) and output word element & 3; stream 0 feeds
+ *                the quantizer, stream 1 the Rand_k subset.
+ *   cuda_stream  a cudaStream_t (NULL = the legacy default stream).
+ * Allocates all scratch (about 8 R d bytes of candidate storage plus small tables); one
+ * segment [0, d) with k is installed.  Returns QS_INVALID_ARG, QS_ALLOC or QS_CUDA on
+ * failure, in which case *out is NULL.
+ */
+int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t seed,
+            void* cuda_stream);
+
+/*
+ * qs_set_segments — piecewise operator of Corollary 1: segment g covers coordinates
+ * [offsets[g], offsets[g+1]) and keeps k_seg[g] of them with its own norm and scaling.
+ *   offsets (host, nseg+1, offsets[0] = 0, increasing, offsets[nseg] = d), k_seg (host,
+ *   nseg, 1 <= k_seg[g] <= segment length).  Reallocates the tables; resets the
+ *   threshold predictions.  Synchronises the stream.
+ */
+int qs_set_segments(qs_ctx* ctx, int nseg, const int64_t* offsets, const int64_t* k_seg);
+
+/*
+ * qs_bind — give the context the state it works on (all device, caller-owned):
+ *   x global model (d), xw local models (R x d), mem memories (R x d),
+ *   anchors (R x d) or NULL.  anchors == NULL selects Algorithm 1 (every worker's
+ *   reference point is x); with anchors the rounds follow Algorithm 2: worker r forms
+ *   its update from anchors_r, and a broadcast also overwrites anchors_r.
+ */
+int qs_bind(qs_ctx* ctx, float* x, float* xw, float* mem, float* anchors);
+
+/*
+ * qs_local_step — the local SGD step of Algorithm 1 (line 5) for the masked workers:
+ *   xw_r <- xw_r - eta * grad_r, a multiply and a subtract, each rounded to fp32.
+ *   grad: device, R x d.
+ */
+int qs_local_step(qs_ctx* ctx, const float* grad, float eta, const uint8_t* worker_mask);
+
+/*
+ * qs_compress_feedback — worker half of a synchronisation (Alg. 1 lines 9-10; Alg. 2
+ * lines 9-10) for the masked workers: forms u, finds the kept set of each segment,
+ * computes the norm of the kept k-vector (the quantizer acts on it as a length-k
+ * vector, proof of Lemma 1), the levels and signs, and writes m <- u - g into mem.
+ * The result (indices, levels, signs, norms, counts) stays in scratch for qs_pack.
+ *   Norm: the exact sum of the squares (QSGD) or magnitudes (Sign) of the kept values,
+ *   rounded once to fp64; sqrt in fp64 for QSGD; rounded to fp32.
+ *   Level: a = |u| * s; p = a / N; l = floor(p); U = (w >> 8) * 2^-24;
+ *   level = min(l + (U < p - l), s); N == 0 gives level 0.
+ *   Value: QSGD g = (N * level) / s (times fl32(1 / (1 + beta_{k,s})) when scaled,
+ *   beta_{k,s} = min(k / s^2, sqrt(k) / s)); Sign g = N1 / k; negated when u < 0.
+ * Non-finite u sets QS_NONFINITE in the device status.
+ */
+int qs_compress_feedback(qs_ctx* ctx, uint64_t round, const uint8_t* worker_mask);
+
+/*
+ * qs_pack — "send g to the master" (Alg. 1 line 9): writes the records of the last
+ * qs_compress_feedback.  wire: device, R rows of stride_words 32-bit words; row r:
+ *   directory: nseg pairs (n, norm bits); then for each segment three streams, each
+ *   padded to a word, fields LSB first: n segment-local indices (ascending) of
+ *   max(1, ceil(log2 d_seg)) bits; n sign bits; for QSGD n fields (level - 1) of
+ *   max(1, ceil(log2 s)) bits.  QSGD drops level-0 entries, Sign sends all k.  Words
+ *   after the record, up to qs_wire_words, are zero.
+ * bits_out: device, R int64, or NULL: exact record size in bits,
+ *   sum over segments of 64 + n (b_idx + 1 + b_lvl).
+ * Rows of workers outside the last mask are not written.
+ * Returns QS_CAPACITY (nothing written) if stride_words < qs_wire_words(ctx).
+ */
+int qs_pack(qs_ctx* ctx, uint32_t* wire, int64_t stride_words, int64_t* bits_out);
+
+/*
+ * qs_unpack_accumulate — master (Alg. 1 line 17; Alg. 2 line 18): decodes the records
+ * of the masked workers from the wire words alone and updates x at every index some
+ * worker sent: acc = 0; acc += g_r in increasing r; x <- x - acc / R.
+ */
+int qs_unpack_accumulate(qs_ctx* ctx, const uint32_t* wire, int64_t stride_words,
+                         const uint8_t* worker_mask);
+
+/*
+ * qs_broadcast — Alg. 1 lines 11 and 18 (Alg. 2 lines 11 and 18): xw_r <- x, and
+ * anchors_r <- x when anchors are bound, for the masked workers.
+ */
+int qs_broadcast(qs_ctx* ctx, const uint8_t* worker_mask);
+
+/*
+ * qs_sync_round — the whole synchronisation for the masked workers, with the same
+ * final bytes in x, xw, mem, anchors, wire and bits_out as qs_compress_feedback,
+ * qs_pack, qs_unpack_accumulate, qs_broadcast in that order, but with the broadcast
+ * folded into the pass that forms u and the few changed coordinates patched after the
+ * decode.  wire / stride_words / bits_out as in qs_pack.
+ */
+int qs_sync_round(qs_ctx* ctx, uint64_t round, const uint8_t* worker_mask, uint32_t* wire,
+                  int64_t stride_words, int64_t* bits_out);
+
+/*
+ * qs_export_selection — copies the result of the last compression out of scratch, for
+ * checking against a reference (all device, any may be NULL):
+ *   sel_idx  R x K int64, global indices of the kept sets, ascending, segments in order
+ *            (K = sum of k_seg);  level R x K int32 (Sign: 1);  sign R x K bytes (1 = u < 0);
+ *   norm R x nseg floats;  n R x nseg int64 (entries sent).
+ */
+int qs_export_selection(qs_ctx* ctx, int64_t* sel_idx, int32_t* level, uint8_t* sign,
+                        float* norm, int64_t* n);
+
+/* Words one worker's record can need (n = k in every segment); < 0 on a bad context. */
+int64_t qs_wire_words(const qs_ctx* ctx);
+/* Bit count of a record whose segments send n[g] entries (host array, nseg). */
+int64_t qs_record_bits(const qs_ctx* ctx, const int64_t* n);
+/* Sum of k_seg. */
+int64_t qs_total_k(const qs_ctx* ctx);
+
+/* Synchronises the stream and returns the first error recorded on the device since the
+ * last call (QS_OK if none), clearing it. */
+int qs_sync_status(qs_ctx* ctx);
+/* Text of the last host-side error of this context (never NULL). */
+const char* qs_last_error(const qs_ctx* ctx);
+
+/* Round counter used by QS_ROUND_AUTO; with the seed and the bound buffers it is the
+ * whole state needed to resume a run. */
+uint64_t qs_get_round(const qs_ctx* ctx);
+int qs_set_round(qs_ctx* ctx, uint64_t round);
+
+/*
+ * qs_get_stats — host counters since qs_init (synchronises the stream): out[0] rounds
+ * compressed, out[1] worker-rounds whose predicted threshold missed and took the exact
+ * histogram pass, out[2] candidates examined in the last round, out[3] kernels launched
+ * since qs_init.  Writes min(n, 4) values.
+ */
+int qs_get_stats(qs_ctx* ctx, int64_t* out, int n);
+
+/* Frees the scratch and the context (NULL is allowed). */
+void qs_destroy(qs_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QSPARSE_H */

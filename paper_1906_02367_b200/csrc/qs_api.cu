@@ -1,0 +1,447 @@
+// C boundary of the sync-round library: context, tables, scratch and the order of launches.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "qs_kernels.h"
+
+using namespace qs;
+
+struct qs_ctx {
+    Plan P;
+    cudaStream_t st;
+    int sms;
+    bool bound, aligned, compressed;
+    Active last;                       // workers of the last compression
+    std::vector<int64_t> off, kseg;    // host copies of the segment table
+    int64_t wire_words;
+    uint64_t round;
+    int64_t launches, rounds;
+    std::string err;
+    std::vector<void*> owned;          // everything cudaMalloc'ed for the current tables
+};
+
+namespace {
+
+int fail(qs_ctx* c, int code, const char* what) {
+    if (c) c->err = what;
+    return code;
+}
+
+int cuda_fail(qs_ctx* c, cudaError_t e, const char* where) {
+    if (c) c->err = std::string(where) + ": " + cudaGetErrorString(e);
+    return QS_CUDA;
+}
+
+#define QS_CUDA_TRY(ctx, call)                                  \
+    do {                                                        \
+        cudaError_t e_ = (call);                                \
+        if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call); \
+    } while (0)
+
+int after_launch(qs_ctx* c, int kernels, const char* where) {
+    c->launches += kernels;
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) return cuda_fail(c, e, where);
+    return QS_OK;
+}
+
+void release(qs_ctx* c) {
+    for (void* p : c->owned) cudaFree(p);
+    c->owned.clear();
+}
+
+template <class T>
+int dev_alloc(qs_ctx* c, T** out, size_t count, bool zero) {
+    void* p = nullptr;
+    const size_t bytes = (count ? count : 1) * sizeof(T);
+    if (cudaMalloc(&p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, QS_ALLOC, "scratch allocation failed");
+    }
+    c->owned.push_back(p);
+    if (zero && cudaMemsetAsync(p, 0, bytes, c->st) != cudaSuccess) return fail(c, QS_CUDA, "memset failed");
+    *out = static_cast<T*>(p);
+    return QS_OK;
+}
+
+template <class T>
+int dev_upload(qs_ctx* c, const T** out, const std::vector<T>& host) {
+    T* p = nullptr;
+    int rc = dev_alloc(c, &p, host.size(), false);
+    if (rc != QS_OK) return rc;
+    if (!host.empty())
+        QS_CUDA_TRY(c, cudaMemcpyAsync(p, host.data(), host.size() * sizeof(T), cudaMemcpyHostToDevice, c->st));
+    *out = p;
+    return QS_OK;
+}
+
+int ceil_log2(uint64_t v) {
+    int b = 0;
+    while ((1ull << b) < v) ++b;
+    return b;
+}
+
+// candidates aimed for in a segment of n coordinates keeping k
+uint32_t candidate_target(int sp, uint64_t n, uint64_t k) {
+    double slack;
+    if (sp == QS_RANDK) {
+        slack = 6.0 * std::sqrt((double)k) + 32.0;           // the hash is uniform: binomial spread
+    } else {
+        const double ratio = (double)k / (double)n;
+        const double frac = ratio <= 0.002 ? 1.0 : ratio <= 0.02 ? 0.5 : 0.25;
+        slack = std::fmax(std::fmax(frac * (double)k, 16.0 * std::sqrt((double)k)), 32.0);
+    }
+    const double t = (double)k + slack;
+    return (uint32_t)(t >= (double)n ? n : (uint64_t)t);
+}
+
+int make_active(const qs_ctx* c, const uint8_t* mask, Active* a) {
+    a->n = 0;
+    a->bits = 0;
+    for (int r = 0; r < c->P.R; ++r)
+        if (!mask || mask[r]) {
+            a->r[a->n++] = r;
+            a->bits |= 1u << r;
+        }
+    return a->n;
+}
+
+int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t* kseg) {
+    Plan& P = c->P;
+    const int64_t d = (int64_t)P.d;
+    if (nseg < 1 || !offsets || !kseg || offsets[0] != 0 || offsets[nseg] != d)
+        return fail(c, QS_INVALID_ARG, "segments must start at 0 and end at d");
+    for (int g = 0; g < nseg; ++g) {
+        const int64_t n = offsets[g + 1] - offsets[g];
+        if (n < 1 || kseg[g] < 1 || kseg[g] > n) return fail(c, QS_INVALID_ARG, "need 1 <= k_seg <= segment length");
+    }
+    QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    release(c);
+    c->off.assign(offsets, offsets + nseg + 1);
+    c->kseg.assign(kseg, kseg + nseg);
+    c->compressed = false;
+
+    const int R = P.R;
+    P.nseg = nseg;
+    P.U = (uint32_t)R * nseg;
+    P.ngroups = (uint32_t)((d + GROUP - 1) / GROUP);
+    P.nblk = (P.ngroups + EMIT_GROUPS - 1) / EMIT_GROUPS;
+    P.cap = (uint64_t)d;
+    P.bl = std::max(1, ceil_log2((uint64_t)P.s));
+    P.maxchunks = (uint32_t)R * (uint32_t)((d + CHUNK - 1) / CHUNK + nseg);
+
+    std::vector<uint32_t> h_off(nseg + 1), h_k(nseg), h_kp(nseg + 1, 0), h_target(nseg), h_grp, h_guess;
+    std::vector<float> h_c(nseg);
+    std::vector<uint8_t> h_bi(nseg);
+    std::vector<FbBlock> h_fb;
+    const bool has_lvl = P.qz != QS_SIGN_L1;
+    int64_t words = 2 * (int64_t)nseg;
+    for (int g = 0; g < nseg; ++g) {
+        const uint64_t n = (uint64_t)(offsets[g + 1] - offsets[g]), k = (uint64_t)kseg[g];
+        h_off[g] = (uint32_t)offsets[g];
+        h_k[g] = (uint32_t)k;
+        h_kp[g + 1] = h_kp[g] + (uint32_t)k;
+        h_target[g] = candidate_target(P.sp, n, k);
+        const double a = (double)k / ((double)P.s * (double)P.s), b = std::sqrt((double)k) / (double)P.s;
+        h_c[g] = (float)(1.0 / (1.0 + (a < b ? a : b)));
+        h_bi[g] = (uint8_t)std::max(1, ceil_log2(n));
+        words += words_for((uint32_t)k, h_bi[g]) + words_for((uint32_t)k, 1) + (has_lvl ? words_for((uint32_t)k, P.bl) : 0);
+        for (uint64_t s0 = 0; s0 < n; s0 += FB_CHUNK)
+            h_fb.push_back(FbBlock{(uint32_t)g, (uint32_t)(offsets[g] + s0), (uint32_t)std::min<uint64_t>(FB_CHUNK, n - s0)});
+    }
+    h_off[nseg] = (uint32_t)d;
+    P.K = h_kp[nseg];
+    P.nfb = (uint32_t)h_fb.size();
+    c->wire_words = words;
+    if (nseg > 1) {
+        h_grp.resize(P.ngroups);
+        int sg = 0;
+        for (uint32_t g = 0; g < P.ngroups; ++g) {
+            const int64_t e = (int64_t)g * GROUP;
+            while (sg + 1 < nseg && e >= offsets[sg + 1]) ++sg;
+            h_grp[g] = (uint32_t)sg;
+        }
+    }
+    // first prediction: none for Top_k (the first round takes the exact pass); for Rand_k the
+    // hash is uniform, so the cut that lets `target` coordinates through is known in advance
+    h_guess.assign((size_t)R * nseg, NO_GUESS);
+    if (P.sp == QS_RANDK)
+        for (int r = 0; r < R; ++r)
+            for (int g = 0; g < nseg; ++g) {
+                const uint64_t n = (uint64_t)(offsets[g + 1] - offsets[g]);
+                const uint64_t cut = h_target[g] >= n ? 0xffffffffull
+                                                      : std::min<uint64_t>(0xffffffffull, ((uint64_t)h_target[g] << 32) / n);
+                h_guess[(size_t)r * nseg + g] = ~(uint32_t)cut;
+            }
+
+    int rc;
+#define UP(field, vec) if ((rc = dev_upload(c, &P.field, vec)) != QS_OK) return rc
+    UP(seg_off, h_off); UP(kseg, h_k); UP(kprefix, h_kp); UP(grp_seg, h_grp); UP(target, h_target);
+    UP(cscale, h_c); UP(bidx, h_bi); UP(fb_tab, h_fb);
+#undef UP
+    const uint32_t* g_up = nullptr;
+    if ((rc = dev_upload(c, &g_up, h_guess)) != QS_OK) return rc;
+    P.guess = const_cast<uint32_t*>(g_up);
+#define AL(field, count, zero) if ((rc = dev_alloc(c, &P.field, (size_t)(count), zero)) != QS_OK) return rc
+    AL(bitmap, (size_t)R * P.ngroups * 4, true);
+    AL(blk_count, (size_t)R * P.nblk, true);
+    AL(blk_base, (size_t)R * P.nblk, true);
+    AL(ncand, R, true);
+    AL(fail, R, true);
+    AL(units, P.U, true);
+    AL(total_chunks, 1, true);
+    AL(cand_idx, (size_t)R * P.cap, false);
+    AL(cand_val, (size_t)R * P.cap, false);
+    AL(cand_q, (size_t)R * P.cap, false);
+    if (P.sp == QS_RANDK) { AL(cand_key, (size_t)R * P.cap, false); } else P.cand_key = nullptr;
+    AL(hist, (size_t)4 * P.U * 256, true);
+    AL(eacc, (size_t)P.U * 256 * 2, true);
+    AL(chunk_cnt, (size_t)P.maxchunks + 1, true);
+    AL(chunk_sel, (size_t)P.maxchunks + 1, true);
+    AL(chunk_nz, (size_t)P.maxchunks + 1, true);
+    AL(fb_hist, (size_t)P.U * FB_BINS, true);
+    AL(sel_idx, (size_t)R * P.K, true);
+    AL(sel_q, (size_t)R * P.K, true);
+    AL(pay_off, P.U, true);
+    AL(bits, R, true);
+    AL(dec_ent, (size_t)R * (nseg + 1), true);
+    AL(dec_pay, P.U, true);
+    AL(touch, (size_t)d, true);
+    AL(status, 1, true);
+    AL(stats, 2, true);
+#undef AL
+    QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    return QS_OK;
+}
+
+// scratch that must be zero when a round starts; restored after a device-side error
+int rezero(qs_ctx* c) {
+    Plan& P = c->P;
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.hist, 0, sizeof(uint32_t) * 4 * P.U * 256, c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.eacc, 0, sizeof(unsigned long long) * P.U * 256 * 2, c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.fb_hist, 0, sizeof(uint32_t) * P.U * FB_BINS, c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.touch, 0, sizeof(uint32_t) * P.d, c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.fail, 0, sizeof(uint32_t) * P.R, c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.status, 0, sizeof(int), c->st));
+    return QS_OK;
+}
+
+uint64_t take_round(qs_ctx* c, uint64_t round) {
+    if (round == QS_ROUND_AUTO) return c->round++;
+    c->round = round + 1;
+    return round;
+}
+
+int compress(qs_ctx* c, uint64_t round, const Active& act, int mode) {
+    Plan& P = c->P;
+    P.round_lo = (uint32_t)round;
+    P.round_hi = (uint32_t)(round >> 32);
+    int rc;
+    launch_pass_a(P, act, mode, c->aligned, c->sms, c->st);
+    if ((rc = after_launch(c, N_PASS_A, "pass_a")) != QS_OK) return rc;
+    launch_candidates(P, act, 0, c->st);
+    if ((rc = after_launch(c, N_CANDIDATES, "candidates")) != QS_OK) return rc;
+    // exact pass for the workers whose prediction left a segment short; no-ops otherwise
+    launch_fallback(P, act, c->sms, c->st);
+    if ((rc = after_launch(c, N_FALLBACK, "fallback")) != QS_OK) return rc;
+    launch_candidates(P, act, 1, c->st);
+    if ((rc = after_launch(c, N_CANDIDATES, "candidates (exact)")) != QS_OK) return rc;
+    launch_select(P, act, c->sms, c->st);
+    if ((rc = after_launch(c, N_SELECT, "select")) != QS_OK) return rc;
+    launch_quantize(P, act, c->sms, c->st);
+    if ((rc = after_launch(c, N_QUANTIZE, "quantize")) != QS_OK) return rc;
+    c->last = act;
+    c->compressed = true;
+    c->rounds += 1;
+    return QS_OK;
+}
+
+int pack(qs_ctx* c, uint32_t* wire, int64_t stride, int64_t* bits_out) {
+    const Active& act = c->last;
+    if (act.n == c->P.R) {
+        QS_CUDA_TRY(c, cudaMemset2DAsync(wire, (size_t)stride * 4, 0, (size_t)c->wire_words * 4, (size_t)act.n, c->st));
+    } else {
+        for (int w = 0; w < act.n; ++w)
+            QS_CUDA_TRY(c, cudaMemsetAsync(wire + (size_t)act.r[w] * stride, 0, (size_t)c->wire_words * 4, c->st));
+    }
+    launch_pack(c->P, act, wire, stride, (long long*)bits_out, c->sms, c->st);
+    return after_launch(c, N_PACK, "pack");
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t seed, void* cuda_stream) {
+    if (!out) return QS_INVALID_ARG;
+    *out = nullptr;
+    const int sp = op & 15, qz = op >> 4;
+    if (R < 1 || R > MAX_R || d < 1 || d >= (1ll << 32) || k < 1 || k > d || s < 1 || s > 65535) return QS_INVALID_ARG;
+    if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1)) return QS_INVALID_ARG;
+    qs_ctx* c = new qs_ctx();
+    std::memset(&c->P, 0, sizeof(Plan));
+    c->st = static_cast<cudaStream_t>(cuda_stream);
+    c->bound = c->aligned = c->compressed = false;
+    c->round = 0;
+    c->launches = c->rounds = 0;
+    c->wire_words = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return QS_CUDA;
+    }
+    Plan& P = c->P;
+    P.R = R; P.d = (uint32_t)d; P.s = s; P.sp = sp; P.qz = qz;
+    P.seed_lo = (uint32_t)seed; P.seed_hi = (uint32_t)(seed >> 32);
+    const int64_t offsets[2] = {0, d};
+    const int rc = install_segments(c, 1, offsets, &k);
+    if (rc != QS_OK) { release(c); delete c; return rc; }
+    *out = c;
+    return QS_OK;
+}
+
+int qs_set_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t* k_seg) {
+    if (!c) return QS_INVALID_ARG;
+    return install_segments(c, nseg, offsets, k_seg);
+}
+
+int qs_bind(qs_ctx* c, float* x, float* xw, float* mem, float* anchors) {
+    if (!c || !x || !xw || !mem) return fail(c, QS_INVALID_ARG, "x, xw and mem are required");
+    c->P.x = x; c->P.xw = xw; c->P.mem = mem; c->P.anchors = anchors;
+    c->aligned = (c->P.d % 4 == 0) && aligned16(x) && aligned16(xw) && aligned16(mem) && aligned16(anchors);
+    c->bound = true;
+    c->compressed = false;
+    return QS_OK;
+}
+
+int qs_local_step(qs_ctx* c, const float* grad, float eta, const uint8_t* worker_mask) {
+    if (!c || !grad) return fail(c, QS_INVALID_ARG, "grad is required");
+    if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
+    Active act;
+    if (!make_active(c, worker_mask, &act)) return QS_OK;
+    launch_local_step(c->P, act, grad, eta, c->aligned && aligned16(grad), c->sms, c->st);
+    return after_launch(c, N_LOCAL_STEP, "local_step");
+}
+
+int qs_compress_feedback(qs_ctx* c, uint64_t round, const uint8_t* worker_mask) {
+    if (!c) return QS_INVALID_ARG;
+    if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
+    if (round != QS_ROUND_AUTO && round >= (1ull << 56)) return fail(c, QS_INVALID_ARG, "round must be below 2^56");
+    Active act;
+    if (!make_active(c, worker_mask, &act)) { c->last = act; c->compressed = true; return QS_OK; }
+    return compress(c, take_round(c, round), act, 0);
+}
+
+int qs_pack(qs_ctx* c, uint32_t* wire, int64_t stride_words, int64_t* bits_out) {
+    if (!c || !wire) return fail(c, QS_INVALID_ARG, "wire is required");
+    if (!c->compressed) return fail(c, QS_STATE, "nothing compressed yet");
+    if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
+    if (c->last.n == 0) return QS_OK;
+    return pack(c, wire, stride_words, bits_out);
+}
+
+int qs_unpack_accumulate(qs_ctx* c, const uint32_t* wire, int64_t stride_words, const uint8_t* worker_mask) {
+    if (!c || !wire) return fail(c, QS_INVALID_ARG, "wire is required");
+    if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
+    if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
+    Active act;
+    if (!make_active(c, worker_mask, &act)) return QS_OK;
+    launch_decode(c->P, act, wire, stride_words, 0, c->sms, c->st);
+    return after_launch(c, N_DECODE, "decode");
+}
+
+int qs_broadcast(qs_ctx* c, const uint8_t* worker_mask) {
+    if (!c) return QS_INVALID_ARG;
+    if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
+    Active act;
+    if (!make_active(c, worker_mask, &act)) return QS_OK;
+    launch_broadcast(c->P, act, c->aligned, c->sms, c->st);
+    return after_launch(c, N_BROADCAST, "broadcast");
+}
+
+int qs_sync_round(qs_ctx* c, uint64_t round, const uint8_t* worker_mask, uint32_t* wire, int64_t stride_words,
+                  int64_t* bits_out) {
+    if (!c || !wire) return fail(c, QS_INVALID_ARG, "wire is required");
+    if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
+    if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
+    if (round != QS_ROUND_AUTO && round >= (1ull << 56)) return fail(c, QS_INVALID_ARG, "round must be below 2^56");
+    Active act;
+    if (!make_active(c, worker_mask, &act)) return QS_OK;
+    int rc = compress(c, take_round(c, round), act, 1);
+    if (rc != QS_OK) return rc;
+    if ((rc = pack(c, wire, stride_words, bits_out)) != QS_OK) return rc;
+    launch_decode(c->P, act, wire, stride_words, 1, c->sms, c->st);
+    return after_launch(c, N_DECODE, "decode");
+}
+
+int qs_export_selection(qs_ctx* c, int64_t* sel_idx, int32_t* level, uint8_t* sign, float* norm, int64_t* n) {
+    if (!c) return QS_INVALID_ARG;
+    if (!c->compressed) return fail(c, QS_STATE, "nothing compressed yet");
+    launch_export(c->P, (long long*)sel_idx, level, sign, norm, (long long*)n, c->sms, c->st);
+    return after_launch(c, N_EXPORT, "export");
+}
+
+int64_t qs_wire_words(const qs_ctx* c) { return c ? c->wire_words : (int64_t)QS_INVALID_ARG; }
+
+int64_t qs_record_bits(const qs_ctx* c, const int64_t* n) {
+    if (!c || !n) return QS_INVALID_ARG;
+    const bool has_lvl = c->P.qz != QS_SIGN_L1;
+    int64_t bits = 0;
+    for (int g = 0; g < c->P.nseg; ++g) {
+        const int bi = std::max(1, ceil_log2((uint64_t)(c->off[g + 1] - c->off[g])));
+        bits += 64 + n[g] * (bi + 1 + (has_lvl ? c->P.bl : 0));
+    }
+    return bits;
+}
+
+int64_t qs_total_k(const qs_ctx* c) { return c ? (int64_t)c->P.K : (int64_t)QS_INVALID_ARG; }
+
+int qs_sync_status(qs_ctx* c) {
+    if (!c) return QS_INVALID_ARG;
+    QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    int code = 0;
+    QS_CUDA_TRY(c, cudaMemcpy(&code, c->P.status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (code != QS_OK) {
+        c->err = code == QS_NONFINITE ? "non-finite value reached the compressor" : "device-side check failed";
+        c->compressed = false;
+        const int rc = rezero(c);
+        if (rc != QS_OK) return rc;
+        QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    }
+    return code;
+}
+
+const char* qs_last_error(const qs_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+uint64_t qs_get_round(const qs_ctx* c) { return c ? c->round : 0; }
+
+int qs_set_round(qs_ctx* c, uint64_t round) {
+    if (!c || round >= (1ull << 56)) return QS_INVALID_ARG;
+    c->round = round;
+    return QS_OK;
+}
+
+int qs_get_stats(qs_ctx* c, int64_t* out, int n) {
+    if (!c || !out) return QS_INVALID_ARG;
+    QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    long long dev[2] = {0, 0};
+    QS_CUDA_TRY(c, cudaMemcpy(dev, c->P.stats, sizeof(dev), cudaMemcpyDeviceToHost));
+    const int64_t v[4] = {c->rounds, (int64_t)dev[0], (int64_t)dev[1], c->launches};
+    for (int i = 0; i < n && i < 4; ++i) out[i] = v[i];
+    return QS_OK;
+}
+
+void qs_destroy(qs_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->st);
+    release(c);
+    delete c;
+}
+
+}  // extern "C"

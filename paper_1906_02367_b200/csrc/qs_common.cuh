@@ -1,0 +1,186 @@
+// Shared declarations of the sync-round kernels (sm_100a).
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/qsparse.h"
+
+namespace qs {
+
+constexpr int MAX_R = 32;            // decode keeps one bit per worker in a 32-bit word
+constexpr int GROUP = 128;           // coordinates per candidate-bitmap group (one warp, 4 each)
+constexpr int EMIT_GROUPS = 256;     // groups per candidate-emission block (32768 coordinates)
+constexpr int CHUNK = 2048;          // candidates per selection chunk (256 threads x 8)
+constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (top 11 key bits)
+constexpr int FB_SHIFT = 21;
+constexpr int FB_CHUNK = 65536;      // coordinates per fallback-histogram block
+constexpr uint32_t NO_GUESS = 0xFFFFFFFFu;
+
+// cand_q fields
+constexpr uint32_t Q_NEG = 1u << 16;
+constexpr uint32_t Q_SEL = 1u << 17;
+
+struct Active {          // workers taking part in a call, ascending
+    int n;
+    uint32_t bits;
+    int r[MAX_R];
+};
+
+struct Unit {            // one (worker, segment) pair
+    uint32_t start;      // first candidate, position in the worker's list
+    uint32_t c;          // number of candidates
+    uint32_t chunk_base; // first chunk in the global chunk numbering
+    uint32_t nchunks;
+    uint32_t tau;        // sort key of the last kept coordinate
+    uint32_t tie_max;    // largest index kept among keys equal to tau
+    uint32_t n;          // entries sent (non-zero level)
+    float norm;
+    uint32_t emin, emax; // exponent range seen by the norm accumulation
+};
+
+struct FbBlock {         // fallback histogram work item: one stretch of one segment
+    uint32_t seg, start, len;
+};
+
+struct Plan {
+    int R, nseg, s, sp, qz, bl;
+    uint32_t d, ngroups, nblk, K, U, nfb, maxchunks;
+    uint32_t seed_lo, seed_hi, round_lo, round_hi;
+    uint64_t cap;
+    // tables (device)
+    const uint32_t* seg_off;   // nseg + 1
+    const uint32_t* kseg;      // nseg
+    const uint32_t* kprefix;   // nseg + 1
+    const uint32_t* grp_seg;   // ngroups: segment of the group's first coordinate
+    const uint32_t* target;    // nseg: candidates aimed for
+    const float* cscale;       // nseg: fl32(1 / (1 + beta_{k,s}))
+    const uint8_t* bidx;       // nseg: bits per index field
+    const FbBlock* fb_tab;     // nfb
+    // bound state
+    float* x; float* xw; float* mem; float* anchors;
+    // scratch
+    uint32_t* guess;           // R x nseg, sort-key space
+    uint32_t* bitmap;          // R x ngroups x 4
+    uint32_t* blk_count;       // R x nblk
+    uint32_t* blk_base;        // R x nblk
+    uint32_t* ncand;           // R
+    uint32_t* fail;            // R
+    Unit* units;               // U = R x nseg
+    uint32_t* total_chunks;    // 1
+    uint32_t* cand_idx;        // R x cap
+    float* cand_val;           // R x cap
+    uint32_t* cand_key;        // R x cap (Rand_k only)
+    uint32_t* cand_q;          // R x cap
+    uint32_t* hist;            // 4 x U x 256, zero between rounds
+    unsigned long long* eacc;  // U x 256 x 2, zero between rounds
+    uint32_t* chunk_cnt;       // maxchunks + 1 (kept | sent << 16 per chunk)
+    uint32_t* chunk_sel;       // maxchunks + 1 exclusive sums of kept
+    uint32_t* chunk_nz;        // maxchunks + 1 exclusive sums of sent
+    uint32_t* fb_hist;         // U x FB_BINS, zero between rounds
+    uint32_t* sel_idx;         // R x K
+    uint32_t* sel_q;           // R x K
+    uint32_t* pay_off;         // R x nseg: word offset of the segment's streams
+    long long* bits;           // R
+    uint32_t* dec_ent;         // R x (nseg + 1)
+    uint32_t* dec_pay;         // R x nseg
+    uint32_t* touch;           // d, zero between rounds
+    int* status;
+    long long* stats;          // device counters: [0] fallback worker-rounds, [1] candidates
+};
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+        k.x += 0x9E3779B9u;
+        k.y += 0xBB67AE85u;
+    }
+    return c;
+}
+
+// the four words for coordinates 4q .. 4q+3 of one worker
+__device__ __forceinline__ uint4 philox_quad(const Plan& P, uint32_t worker, uint32_t q,
+                                             uint32_t stream) {
+    return philox4x32_10(make_uint4(q, worker, P.round_lo, (P.round_hi << 8) | stream),
+                         make_uint2(P.seed_lo, P.seed_hi));
+}
+
+__device__ __forceinline__ uint32_t philox_word(const Plan& P, uint32_t worker, uint32_t e,
+                                                uint32_t stream) {
+    const uint4 o = philox_quad(P, worker, e >> 2, stream);
+    const uint32_t j = e & 3u;
+    return j == 0 ? o.x : j == 1 ? o.y : j == 2 ? o.z : o.w;
+}
+
+// Sort key: larger = kept first.  Top_k: |u| bit pattern (shifted up by the spare sign bit);
+// Rand_k: complement of the hash, so that the smallest hashes come first.
+__device__ __forceinline__ uint32_t topk_key(float u) { return __float_as_uint(u) << 1; }
+
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// Exclusive scan over the block (blockDim.x a multiple of 32, at most 1024); every thread
+// gets the block total too.  sh: 33 words.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* sh, uint32_t* total) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const uint32_t incl = warp_incl_scan(v, lane);
+    __syncthreads();                       // sh may still be read from a previous call
+    if (lane == 31) sh[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+        const uint32_t w = lane < nw ? sh[lane] : 0u;
+        const uint32_t wi = warp_incl_scan(w, lane);
+        sh[lane] = wi - w;
+        if (lane == 31) sh[32] = wi;
+    }
+    __syncthreads();
+    *total = sh[32];
+    return sh[wid] + incl - v;
+}
+
+__device__ __forceinline__ void set_status(const Plan& P, int code) { atomicCAS(P.status, 0, code); }
+
+__host__ __device__ __forceinline__ uint32_t words_for(uint32_t nfields, uint32_t width) {
+    return (uint32_t)(((uint64_t)nfields * width + 31u) >> 5);
+}
+
+// fp32 level of the QSGD quantizer and the value it stands for
+__device__ __forceinline__ int qsgd_level(float u, float N, int s, uint32_t w) {
+    if (N == 0.0f) return 0;
+    const float a = fabsf(u) * (float)s;
+    const float p = a / N;
+    const float l = floorf(p);
+    const float f = p - l;
+    const float U = (float)(w >> 8) * 5.9604644775390625e-08f;
+    const int level = (int)l + (U < f ? 1 : 0);
+    return level < s ? level : s;
+}
+
+__device__ __forceinline__ float coord_value(const Plan& P, float N, int level, bool neg, float c,
+                                             uint32_t k) {
+    float g;
+    if (P.qz == QS_SIGN_L1) {
+        g = N / (float)k;
+    } else {
+        g = (N * (float)level) / (float)P.s;
+        if (P.qz == QS_QSGD_SCALED) g = g * c;
+    }
+    return neg ? -g : g;
+}
+
+}  // namespace qs
