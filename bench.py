@@ -1,0 +1,308 @@
+#!/usr/bin/env python
+"""Benchmark of the fused synchronisation round on the ResNet-50-shaped workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one qs_sync_round (form u, select, quantize, memory update, pack, decode, update x,
+broadcast) over R = 8 workers of d = 25,557,032 coordinates laid out as ResNet-50's 161 tensors,
+Top_k with k = 0.1% d over the flat vector composed with the sign/l1 quantizer; a fresh Laplace
+drift is added to the workers' models before every step, outside the timed region.  The reported
+value is the minimum bytes a round has to move (16 R d + 8 d + record bytes written and read)
+divided by the round time.  Prints one JSON line.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1906_02367_b200 import inputs as I  # noqa: E402
+
+R = 8
+METRIC = "sync_round_effective_bandwidth"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def workload(variant, shrink=1):
+    sizes = I.scaled_sizes(I.resnet50_tensor_sizes(), shrink)
+    off = I.segments_from_sizes(sizes)
+    d = int(off[-1])
+    if variant == "per_tensor":
+        return sizes, off, d, off, I.k_per_tensor_ratio(sizes)
+    return sizes, off, d, np.array([0, d], np.int64), np.array([I.k_from_ratio(d, 1, 1000)], np.int64)
+
+
+def min_bytes(d, wire_bytes):
+    """Bytes one round cannot avoid: read xw, mem and write mem, xw (16 B per worker coordinate),
+    read and write x (8 B per coordinate), records written once and read once."""
+    return 16 * R * d + 8 * d + 2 * wire_bytes
+
+
+def peak_hbm():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 7] or [r for _, r in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[0]) for r in rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons,
+                "power_w_max": max(float(r[2]) for r in rows), "samples": len(rows)}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1906_02367_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    sizes, off, d, seg_off, kseg = workload(args.variant, args.shrink)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234 + rank)
+    scales = I.tensor_scales(len(sizes), seed=0)
+    per_elem = torch.from_numpy(np.repeat(scales, np.diff(off))).to(dev)
+    x = torch.from_numpy(I.model_init(d, seed=rank)).to(dev)
+    xw = x.expand(R, d).contiguous()
+    mem = torch.zeros((R, d), dtype=torch.float32, device=dev)
+    e1 = torch.empty((R, d), dtype=torch.float32, device=dev)
+    e2 = torch.empty_like(e1)
+
+    def drift():
+        # Laplace(0, b_t) per tensor as the difference of two exponentials
+        e1.exponential_(generator=gen)
+        e2.exponential_(generator=gen)
+        e1.sub_(e2).mul_(per_elem)
+        xw.add_(e1)
+
+    ctx = B.Context(R, d, int(kseg[0]), 1, B.QS_TOPK, B.QS_SIGN_L1, seed=rank)
+    if len(kseg) > 1:
+        ctx.set_segments(seg_off, kseg)
+    ctx.bind(x, xw, mem)
+    wire = ctx.new_wire()
+    bits = torch.zeros(R, dtype=torch.int64, device=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        drift()
+        ctx.sync_round(wire, bits_out=bits)
+    assert ctx.sync_status() == 0, ctx.last_error()
+    st0 = ctx.stats()
+    ctx.enable_phase_timing(True)
+    ctx.phase_timing()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid)) if rank == 0 else None
+    barrier()
+    t0 = time.time()
+    for i in range(args.steps):
+        drift()                       # untimed: the local steps that precede a synchronisation
+        starts[i].record()
+        ctx.sync_round(wire, bits_out=bits)
+        ends[i].record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    assert ctx.sync_status() == 0, ctx.last_error()
+    per_step = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    total_ms = float(sum(per_step))
+    phases = ctx.phase_timing()
+    ctx.enable_phase_timing(False)
+    st1 = ctx.stats()
+    wire_bytes = int(bits.sum().item() + 7) // 8
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    bmin = min_bytes(d, wire_bytes)
+    value = world * bmin * args.steps / (total_ms * 1e-3) / 1e9
+    peak, peak_src = peak_hbm()
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"ResNet-50-shaped round: R=8, d={d} (161 tensors), Top_k k=0.1% ({args.variant}), "
+                               "sign/l1 quantizer, Laplace drift per tensor, memory carried",
+                   "variant": args.variant, "R": R, "d": d, "k_total": int(kseg.sum()),
+                   "l2_policy": "inputs (3.4 GB per round) larger than L2", "multi_gpu": "independent replicas"},
+        "worker_elements_per_s": world * R * d * args.steps / (total_ms * 1e-3),
+        "pct_of_nominal_8TBps": 100.0 * value / world / NOMINAL_HBM_GBS,
+        "pct_of_measured_copy": 100.0 * value / world / peak,
+        "min_bytes_per_round": bmin, "wire_bytes_per_round": wire_bytes,
+        "ms_per_step_median": float(np.median(per_step)),
+        "gpu_launches": st1["launches"] - st0["launches"],
+        "fallback_worker_rounds": st1["fallback_worker_rounds"] - st0["fallback_worker_rounds"],
+        "phases_ms_per_round": {k: v / max(1, phases["rounds"]) for k, v in phases.items() if k != "rounds"},
+        "clocks": clocks,
+    }
+    # roofline of the dominant kernel (the dense pass): 16 B per worker coordinate + 4 B per coordinate
+    dense_ms = phases["dense_pass"] / max(1, phases["rounds"])
+    dense_bytes = 16 * R * d + 4 * d
+    achieved = dense_bytes / (dense_ms * 1e-3) / 1e9 if dense_ms > 0 else 0.0
+    result["roofline"] = {"kernel": "pass_a_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                          "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                          "algorithmic_bytes_per_launch": dense_bytes, "ms_per_launch": dense_ms}
+
+    if rank == 0 and world == 1 and not args.no_e2e:
+        result["e2e"] = run_e2e(torch, ctx, x, xw, mem, wire, bits, drift, d)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        drift()
+        torch.cuda.synchronize()
+        result["cpu_baseline"] = cpu_round(x.cpu().numpy(), xw.cpu().numpy(), mem.cpu().numpy(), seg_off, kseg, d)
+    ctx.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(result))
+
+
+def run_e2e(torch, ctx, x, xw, mem, wire, bits, drift, d, steps=3):
+    """Same round with the state living in pinned host memory: every step copies x, xw, mem to the
+    device, runs qs_sync_round and copies x, xw, mem and the records back."""
+    hx = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
+    hxw = torch.empty(xw.shape, dtype=xw.dtype, pin_memory=True)
+    hmem = torch.empty(mem.shape, dtype=mem.dtype, pin_memory=True)
+    hwire = torch.empty(wire.shape, dtype=wire.dtype, pin_memory=True)
+    times = []
+    for i in range(steps + 1):
+        drift()
+        hx.copy_(x); hxw.copy_(xw); hmem.copy_(mem)
+        torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        x.copy_(hx, non_blocking=True); xw.copy_(hxw, non_blocking=True); mem.copy_(hmem, non_blocking=True)
+        ctx.sync_round(wire, bits_out=bits)
+        hx.copy_(x, non_blocking=True); hxw.copy_(xw, non_blocking=True); hmem.copy_(mem, non_blocking=True)
+        hwire.copy_(wire, non_blocking=True)
+        e.record()
+        torch.cuda.synchronize()
+        if i:
+            times.append(s.elapsed_time(e))
+    wire_bytes = int(bits.sum().item() + 7) // 8
+    state = 4 * (d + 2 * R * d)
+    ms = float(np.mean(times))
+    return {"value": min_bytes(d, wire_bytes) / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+            "h2d_bytes_per_step": state, "d2h_bytes_per_step": state + wire.numel() * 4, "steps": steps}
+
+
+def cpu_round(x, xw, mem, seg_off, kseg, d):
+    """The oracle, as it stands, on the host cores: one round over the given state."""
+    from oracle import oracle as O
+    cores = os.cpu_count() or 1
+    plan = O.Plan(R, d, s=1, sparsifier=O.TOPK, quantizer=O.SIGN_L1, seed=0, offsets=seg_off, kseg=kseg)
+    threads = min(cores, R)
+    t0 = time.perf_counter()
+    out = O.sync_round(plan, 0, x, xw, mem, mode=O.NTH, nthreads=threads)
+    dt = time.perf_counter() - t0
+    assert out["rc"] == 0
+    wire_bytes = int(out["bits"].sum() + 7) // 8
+    return {"value": min_bytes(d, wire_bytes) / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "seconds": dt, "sample": f"one round, R={R}, d={d}, nth_element selection, workers spread over {threads} threads"}
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: each step is one round over a prefix of the workload
+    sized so that the whole run ends within a few minutes."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    sizes, off, d, seg_off, kseg = workload("flat")
+    steps = args.steps + args.warmup
+    budget_s = 150.0
+    sample_d = int(min(d, max(1 << 16, 2.0e6 * budget_s / steps)))       # ~2 M coordinates x 8 workers per second
+    rng = np.random.default_rng(0)
+    x = I.model_init(sample_d, seed=0)
+    xw = np.broadcast_to(x, (R, sample_d)).copy()
+    mem = np.zeros((R, sample_d), np.float32)
+    scales = np.repeat(I.tensor_scales(len(sizes), seed=0), np.diff(off))[:sample_d]
+    times, last = [], None
+    for i in range(steps):
+        xw += (rng.laplace(0.0, 1.0, (R, sample_d)).astype(np.float32) * scales[None, :])
+        last = cpu_round(x, xw, mem, np.array([0, sample_d], np.int64),
+                         np.array([I.k_from_ratio(sample_d, 1, 1000)], np.int64), sample_d)
+        if i >= args.warmup:
+            times.append(last["seconds"])
+    ms = 1e3 * float(np.mean(times))
+    value = min_bytes(sample_d, 0) / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"ResNet-50-shaped round, prefix of {sample_d} of {d} coordinates, R=8, Top_k 0.1% flat, sign/l1"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor"])
+    ap.add_argument("--shrink", type=int, default=1, help="divide every tensor size (profiling on a small case)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

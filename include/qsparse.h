@@ -204,10 +204,22 @@ int qs_set_round(qs_ctx* ctx, uint64_t round);
 /*
  * qs_get_stats — host counters since qs_init (synchronises the stream): out[0] rounds
  * compressed, out[1] worker-rounds whose predicted threshold missed and took the exact
- * histogram pass, out[2] candidates examined in the last round, out[3] kernels launched
- * since qs_init.  Writes min(n, 4) values.
+ * histogram pass, out[2] candidates examined, out[3] kernels launched.  Writes min(n, 4)
+ * values.
  */
 int qs_get_stats(qs_ctx* ctx, int64_t* out, int n);
+
+/*
+ * qs_enable_phase_timing / qs_get_phase_timing — measurement aid, not part of the method:
+ * when on, qs_sync_round records CUDA events on the context's stream between its phases.
+ * qs_get_phase_timing synchronises and returns, summed over the rounds since the last call
+ * and then cleared: ms[0] the dense pass (form u, candidate flags, old-model broadcast: one
+ * kernel launch per round), ms[1] candidate list and selection, ms[2] norm / quantizer /
+ * memory update, ms[3] pack, ms[4] decode and update; ms[5] the number of rounds.  Writes
+ * min(n, 6) values.
+ */
+int qs_enable_phase_timing(qs_ctx* ctx, int on);
+int qs_get_phase_timing(qs_ctx* ctx, double* ms, int n);
 
 /* Frees the scratch and the context (NULL is allowed). */
 void qs_destroy(qs_ctx* ctx);

@@ -22,7 +22,7 @@ EXPORTS = [
     "qs_init", "qs_set_segments", "qs_bind", "qs_local_step", "qs_compress_feedback", "qs_pack",
     "qs_unpack_accumulate", "qs_broadcast", "qs_sync_round", "qs_export_selection", "qs_wire_words",
     "qs_record_bits", "qs_total_k", "qs_sync_status", "qs_last_error", "qs_get_round", "qs_set_round",
-    "qs_get_stats", "qs_destroy",
+    "qs_get_stats", "qs_enable_phase_timing", "qs_get_phase_timing", "qs_destroy",
 ]
 
 _lib = None
@@ -64,6 +64,8 @@ def lib():
         L.qs_get_round.restype = u64
         L.qs_set_round.argtypes = [vp, u64]
         L.qs_get_stats.argtypes = [vp, vp, C.c_int]
+        L.qs_enable_phase_timing.argtypes = [vp, C.c_int]
+        L.qs_get_phase_timing.argtypes = [vp, vp, C.c_int]
         L.qs_destroy.argtypes = [vp]
         L.qs_destroy.restype = None
         _lib = L
@@ -185,6 +187,15 @@ class Context:
         self._check(lib().qs_get_stats(self._h, out.ctypes.data_as(C.c_void_p), 4))
         return {"rounds": int(out[0]), "fallback_worker_rounds": int(out[1]), "candidates": int(out[2]),
                 "launches": int(out[3])}
+
+    def enable_phase_timing(self, on=True):
+        self._check(lib().qs_enable_phase_timing(self._h, int(bool(on))))
+
+    def phase_timing(self):
+        out = np.zeros(6, dtype=np.float64)
+        self._check(lib().qs_get_phase_timing(self._h, out.ctypes.data_as(C.c_void_p), 6))
+        names = ("dense_pass", "select", "quantize", "pack", "decode")
+        return {"rounds": int(out[5]), **{n: float(out[i]) for i, n in enumerate(names)}}
 
     def new_wire(self):
         return torch.zeros((self.R, self.wire_words()), dtype=torch.int32, device=self._keep[0].device)

@@ -21,9 +21,35 @@ struct qs_ctx {
     int64_t launches, rounds;
     std::string err;
     std::vector<void*> owned;          // everything cudaMalloc'ed for the current tables
+    // optional per-phase timing of qs_sync_round (events on the context's stream)
+    bool timing;
+    std::vector<cudaEvent_t> ev;       // TIMING_ROUNDS x TIMING_MARKS
+    int ev_used;
+    double phase_ms[5];
+    int64_t timed_rounds;
 };
 
 namespace {
+
+constexpr int TIMING_MARKS = 6, TIMING_ROUNDS = 256;
+
+void mark(qs_ctx* c, int slot) {
+    if (c->timing) cudaEventRecord(c->ev[(size_t)c->ev_used * TIMING_MARKS + slot], c->st);
+}
+
+// adds the recorded rounds to the per-phase sums (synchronises the stream)
+void fold_timing(qs_ctx* c) {
+    if (!c->ev_used) return;
+    cudaStreamSynchronize(c->st);
+    for (int i = 0; i < c->ev_used; ++i)
+        for (int ph = 0; ph < TIMING_MARKS - 1; ++ph) {
+            float ms = 0.0f;
+            if (cudaEventElapsedTime(&ms, c->ev[(size_t)i * TIMING_MARKS + ph], c->ev[(size_t)i * TIMING_MARKS + ph + 1]) == cudaSuccess)
+                c->phase_ms[ph] += ms;
+        }
+    c->timed_rounds += c->ev_used;
+    c->ev_used = 0;
+}
 
 int fail(qs_ctx* c, int code, const char* what) {
     if (c) c->err = what;
@@ -240,8 +266,10 @@ int compress(qs_ctx* c, uint64_t round, const Active& act, int mode) {
     P.round_lo = (uint32_t)round;
     P.round_hi = (uint32_t)(round >> 32);
     int rc;
+    if (mode == 1) mark(c, 0);
     launch_pass_a(P, act, mode, c->aligned, c->sms, c->st);
     if ((rc = after_launch(c, N_PASS_A, "pass_a")) != QS_OK) return rc;
+    if (mode == 1) mark(c, 1);
     launch_candidates(P, act, 0, c->st);
     if ((rc = after_launch(c, N_CANDIDATES, "candidates")) != QS_OK) return rc;
     // exact pass for the workers whose prediction left a segment short; no-ops otherwise
@@ -251,8 +279,10 @@ int compress(qs_ctx* c, uint64_t round, const Active& act, int mode) {
     if ((rc = after_launch(c, N_CANDIDATES, "candidates (exact)")) != QS_OK) return rc;
     launch_select(P, act, c->sms, c->st);
     if ((rc = after_launch(c, N_SELECT, "select")) != QS_OK) return rc;
+    if (mode == 1) mark(c, 2);
     launch_quantize(P, act, c->sms, c->st);
     if ((rc = after_launch(c, N_QUANTIZE, "quantize")) != QS_OK) return rc;
+    if (mode == 1) mark(c, 3);
     c->last = act;
     c->compressed = true;
     c->rounds += 1;
@@ -290,6 +320,10 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     c->round = 0;
     c->launches = c->rounds = 0;
     c->wire_words = 0;
+    c->timing = false;
+    c->ev_used = 0;
+    c->timed_rounds = 0;
+    for (double& a : c->phase_ms) a = 0.0;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
         cudaGetLastError();
@@ -376,8 +410,34 @@ int qs_sync_round(qs_ctx* c, uint64_t round, const uint8_t* worker_mask, uint32_
     int rc = compress(c, take_round(c, round), act, 1);
     if (rc != QS_OK) return rc;
     if ((rc = pack(c, wire, stride_words, bits_out)) != QS_OK) return rc;
+    mark(c, 4);
     launch_decode(c->P, act, wire, stride_words, 1, c->sms, c->st);
-    return after_launch(c, N_DECODE, "decode");
+    rc = after_launch(c, N_DECODE, "decode");
+    mark(c, 5);
+    if (c->timing && ++c->ev_used == TIMING_ROUNDS) fold_timing(c);
+    return rc;
+}
+
+int qs_enable_phase_timing(qs_ctx* c, int on) {
+    if (!c) return QS_INVALID_ARG;
+    fold_timing(c);
+    if (on && c->ev.empty()) {
+        c->ev.resize((size_t)TIMING_ROUNDS * TIMING_MARKS);
+        for (auto& e : c->ev) QS_CUDA_TRY(c, cudaEventCreate(&e));
+    }
+    c->timing = on != 0;
+    return QS_OK;
+}
+
+int qs_get_phase_timing(qs_ctx* c, double* ms, int n) {
+    if (!c || !ms) return QS_INVALID_ARG;
+    fold_timing(c);
+    const double v[6] = {c->phase_ms[0], c->phase_ms[1], c->phase_ms[2], c->phase_ms[3], c->phase_ms[4],
+                         (double)c->timed_rounds};
+    for (int i = 0; i < n && i < 6; ++i) ms[i] = v[i];
+    for (double& a : c->phase_ms) a = 0.0;
+    c->timed_rounds = 0;
+    return QS_OK;
 }
 
 int qs_export_selection(qs_ctx* c, int64_t* sel_idx, int32_t* level, uint8_t* sign, float* norm, int64_t* n) {
@@ -440,6 +500,7 @@ int qs_get_stats(qs_ctx* c, int64_t* out, int n) {
 void qs_destroy(qs_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->st);
+    for (auto& e : c->ev) cudaEventDestroy(e);
     release(c);
     delete c;
 }
