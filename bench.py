@@ -185,6 +185,7 @@ def run_ours(args):
         "gpu_launches": st1["launches"] - st0["launches"],
         "fallback_worker_rounds": st1["fallback_worker_rounds"] - st0["fallback_worker_rounds"],
         "phases_ms_per_round": {k: v / max(1, phases["rounds"]) for k, v in phases.items() if k != "rounds"},
+        "kernels_per_round": (st1["launches"] - st0["launches"]) / max(1, args.steps),
         "clocks": clocks,
     }
     # roofline of the dominant kernel (the dense pass): 16 B per worker coordinate + 4 B per coordinate

@@ -211,12 +211,12 @@ int qs_get_stats(qs_ctx* ctx, int64_t* out, int n);
 
 /*
  * qs_enable_phase_timing / qs_get_phase_timing — measurement aid, not part of the method:
- * when on, qs_sync_round records CUDA events on the context's stream between its phases.
+ * when on, qs_sync_round records CUDA events on the context's stream around its dense pass.
  * qs_get_phase_timing synchronises and returns, summed over the rounds since the last call
  * and then cleared: ms[0] the dense pass (form u, candidate flags, old-model broadcast: one
- * kernel launch per round), ms[1] candidate list and selection, ms[2] norm / quantizer /
- * memory update, ms[3] pack, ms[4] decode and update; ms[5] the number of rounds.  Writes
- * min(n, 6) values.
+ * kernel launch per round), ms[1] the rest of the round (selection, quantizer, memory update,
+ * pack, decode, update: one persistent kernel), ms[2] the number of rounds.  Writes
+ * min(n, 3) values.
  */
 int qs_enable_phase_timing(qs_ctx* ctx, int on);
 int qs_get_phase_timing(qs_ctx* ctx, double* ms, int n);

@@ -192,10 +192,9 @@ class Context:
         self._check(lib().qs_enable_phase_timing(self._h, int(bool(on))))
 
     def phase_timing(self):
-        out = np.zeros(6, dtype=np.float64)
-        self._check(lib().qs_get_phase_timing(self._h, out.ctypes.data_as(C.c_void_p), 6))
-        names = ("dense_pass", "select", "quantize", "pack", "decode")
-        return {"rounds": int(out[5]), **{n: float(out[i]) for i, n in enumerate(names)}}
+        out = np.zeros(3, dtype=np.float64)
+        self._check(lib().qs_get_phase_timing(self._h, out.ctypes.data_as(C.c_void_p), 3))
+        return {"rounds": int(out[2]), "dense_pass": float(out[0]), "rest_of_round": float(out[1])}
 
     def new_wire(self):
         return torch.zeros((self.R, self.wire_words()), dtype=torch.int32, device=self._keep[0].device)

@@ -12,7 +12,7 @@ using namespace qs;
 struct qs_ctx {
     Plan P;
     cudaStream_t st;
-    int sms;
+    int sms, mid_grid;
     bool bound, aligned, compressed;
     Active last;                       // workers of the last compression
     std::vector<int64_t> off, kseg;    // host copies of the segment table
@@ -25,13 +25,13 @@ struct qs_ctx {
     bool timing;
     std::vector<cudaEvent_t> ev;       // TIMING_ROUNDS x TIMING_MARKS
     int ev_used;
-    double phase_ms[5];
+    double phase_ms[2];
     int64_t timed_rounds;
 };
 
 namespace {
 
-constexpr int TIMING_MARKS = 6, TIMING_ROUNDS = 256;
+constexpr int TIMING_MARKS = 3, TIMING_ROUNDS = 512;
 
 void mark(qs_ctx* c, int slot) {
     if (c->timing) cudaEventRecord(c->ev[(size_t)c->ev_used * TIMING_MARKS + slot], c->st);
@@ -237,6 +237,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(dec_pay, P.U, true);
     AL(touch, (size_t)d, true);
     AL(status, 1, true);
+    AL(bar, 2, true);
     AL(stats, 2, true);
 #undef AL
     QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
@@ -252,6 +253,8 @@ int rezero(qs_ctx* c) {
     QS_CUDA_TRY(c, cudaMemsetAsync(P.touch, 0, sizeof(uint32_t) * P.d, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.fail, 0, sizeof(uint32_t) * P.R, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.status, 0, sizeof(int), c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 2 * sizeof(uint32_t), c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.blk_count, 0, sizeof(uint32_t) * P.R * P.nblk, c->st));
     return QS_OK;
 }
 
@@ -261,44 +264,48 @@ uint64_t take_round(qs_ctx* c, uint64_t round) {
     return round;
 }
 
-int compress(qs_ctx* c, uint64_t round, const Active& act, int mode) {
-    Plan& P = c->P;
-    P.round_lo = (uint32_t)round;
-    P.round_hi = (uint32_t)(round >> 32);
-    int rc;
-    if (mode == 1) mark(c, 0);
-    launch_pass_a(P, act, mode, c->aligned, c->sms, c->st);
-    if ((rc = after_launch(c, N_PASS_A, "pass_a")) != QS_OK) return rc;
-    if (mode == 1) mark(c, 1);
-    launch_candidates(P, act, 0, c->st);
-    if ((rc = after_launch(c, N_CANDIDATES, "candidates")) != QS_OK) return rc;
-    // exact pass for the workers whose prediction left a segment short; no-ops otherwise
-    launch_fallback(P, act, c->sms, c->st);
-    if ((rc = after_launch(c, N_FALLBACK, "fallback")) != QS_OK) return rc;
-    launch_candidates(P, act, 1, c->st);
-    if ((rc = after_launch(c, N_CANDIDATES, "candidates (exact)")) != QS_OK) return rc;
-    launch_select(P, act, c->sms, c->st);
-    if ((rc = after_launch(c, N_SELECT, "select")) != QS_OK) return rc;
-    if (mode == 1) mark(c, 2);
-    launch_quantize(P, act, c->sms, c->st);
-    if ((rc = after_launch(c, N_QUANTIZE, "quantize")) != QS_OK) return rc;
-    if (mode == 1) mark(c, 3);
-    c->last = act;
-    c->compressed = true;
-    c->rounds += 1;
-    return QS_OK;
-}
-
-int pack(qs_ctx* c, uint32_t* wire, int64_t stride, int64_t* bits_out) {
-    const Active& act = c->last;
+int clear_wire(qs_ctx* c, const Active& act, uint32_t* wire, int64_t stride) {
     if (act.n == c->P.R) {
         QS_CUDA_TRY(c, cudaMemset2DAsync(wire, (size_t)stride * 4, 0, (size_t)c->wire_words * 4, (size_t)act.n, c->st));
     } else {
         for (int w = 0; w < act.n; ++w)
             QS_CUDA_TRY(c, cudaMemsetAsync(wire + (size_t)act.r[w] * stride, 0, (size_t)c->wire_words * 4, c->st));
     }
-    launch_pack(c->P, act, wire, stride, (long long*)bits_out, c->sms, c->st);
-    return after_launch(c, N_PACK, "pack");
+    return QS_OK;
+}
+
+int run_mid(qs_ctx* c, const Active& act, int do_compress, int do_pack, int do_decode, int patch, uint32_t* wire,
+            int64_t stride, int64_t* bits_out) {
+    const cudaError_t e = launch_mid(c->P, act, do_compress, do_pack, do_decode, patch, wire, stride,
+                                     (long long*)bits_out, c->mid_grid, c->st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "persistent kernel");
+    return after_launch(c, 1, "persistent kernel");
+}
+
+// dense pass, then the persistent kernel for the stages asked for
+int round_body(qs_ctx* c, uint64_t round, const Active& act, bool fused, uint32_t* wire, int64_t stride,
+               int64_t* bits_out) {
+    Plan& P = c->P;
+    P.round_lo = (uint32_t)round;
+    P.round_hi = (uint32_t)(round >> 32);
+    int rc;
+    if (fused) mark(c, 0);
+    launch_pass_a(P, act, fused ? 1 : 0, c->aligned, c->sms, c->st);
+    if ((rc = after_launch(c, 1, "pass_a")) != QS_OK) return rc;
+    if (fused) {
+        mark(c, 1);
+        if ((rc = clear_wire(c, act, wire, stride)) != QS_OK) return rc;
+    }
+    rc = run_mid(c, act, 1, fused, fused, fused, wire, stride, bits_out);
+    if (fused) {
+        mark(c, 2);
+        if (c->timing && ++c->ev_used == TIMING_ROUNDS) fold_timing(c);
+    }
+    if (rc != QS_OK) return rc;
+    c->last = act;
+    c->compressed = true;
+    c->rounds += 1;
+    return QS_OK;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -330,6 +337,9 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
         delete c;
         return QS_CUDA;
     }
+    const int per_sm = mid_blocks_per_sm(sp == QS_RANDK);
+    if (per_sm < 1) { delete c; return QS_CUDA; }
+    c->mid_grid = c->sms * (per_sm < 2 ? per_sm : 2);
     Plan& P = c->P;
     P.R = R; P.d = (uint32_t)d; P.s = s; P.sp = sp; P.qz = qz;
     P.seed_lo = (uint32_t)seed; P.seed_hi = (uint32_t)(seed >> 32);
@@ -360,7 +370,7 @@ int qs_local_step(qs_ctx* c, const float* grad, float eta, const uint8_t* worker
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
     launch_local_step(c->P, act, grad, eta, c->aligned && aligned16(grad), c->sms, c->st);
-    return after_launch(c, N_LOCAL_STEP, "local_step");
+    return after_launch(c, 1, "local_step");
 }
 
 int qs_compress_feedback(qs_ctx* c, uint64_t round, const uint8_t* worker_mask) {
@@ -369,7 +379,7 @@ int qs_compress_feedback(qs_ctx* c, uint64_t round, const uint8_t* worker_mask) 
     if (round != QS_ROUND_AUTO && round >= (1ull << 56)) return fail(c, QS_INVALID_ARG, "round must be below 2^56");
     Active act;
     if (!make_active(c, worker_mask, &act)) { c->last = act; c->compressed = true; return QS_OK; }
-    return compress(c, take_round(c, round), act, 0);
+    return round_body(c, take_round(c, round), act, false, nullptr, 0, nullptr);
 }
 
 int qs_pack(qs_ctx* c, uint32_t* wire, int64_t stride_words, int64_t* bits_out) {
@@ -377,7 +387,9 @@ int qs_pack(qs_ctx* c, uint32_t* wire, int64_t stride_words, int64_t* bits_out) 
     if (!c->compressed) return fail(c, QS_STATE, "nothing compressed yet");
     if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
     if (c->last.n == 0) return QS_OK;
-    return pack(c, wire, stride_words, bits_out);
+    const int rc = clear_wire(c, c->last, wire, stride_words);
+    if (rc != QS_OK) return rc;
+    return run_mid(c, c->last, 0, 1, 0, 0, wire, stride_words, bits_out);
 }
 
 int qs_unpack_accumulate(qs_ctx* c, const uint32_t* wire, int64_t stride_words, const uint8_t* worker_mask) {
@@ -386,8 +398,7 @@ int qs_unpack_accumulate(qs_ctx* c, const uint32_t* wire, int64_t stride_words, 
     if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
-    launch_decode(c->P, act, wire, stride_words, 0, c->sms, c->st);
-    return after_launch(c, N_DECODE, "decode");
+    return run_mid(c, act, 0, 0, 1, 0, const_cast<uint32_t*>(wire), stride_words, nullptr);
 }
 
 int qs_broadcast(qs_ctx* c, const uint8_t* worker_mask) {
@@ -396,7 +407,7 @@ int qs_broadcast(qs_ctx* c, const uint8_t* worker_mask) {
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
     launch_broadcast(c->P, act, c->aligned, c->sms, c->st);
-    return after_launch(c, N_BROADCAST, "broadcast");
+    return after_launch(c, 1, "broadcast");
 }
 
 int qs_sync_round(qs_ctx* c, uint64_t round, const uint8_t* worker_mask, uint32_t* wire, int64_t stride_words,
@@ -407,15 +418,7 @@ int qs_sync_round(qs_ctx* c, uint64_t round, const uint8_t* worker_mask, uint32_
     if (round != QS_ROUND_AUTO && round >= (1ull << 56)) return fail(c, QS_INVALID_ARG, "round must be below 2^56");
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
-    int rc = compress(c, take_round(c, round), act, 1);
-    if (rc != QS_OK) return rc;
-    if ((rc = pack(c, wire, stride_words, bits_out)) != QS_OK) return rc;
-    mark(c, 4);
-    launch_decode(c->P, act, wire, stride_words, 1, c->sms, c->st);
-    rc = after_launch(c, N_DECODE, "decode");
-    mark(c, 5);
-    if (c->timing && ++c->ev_used == TIMING_ROUNDS) fold_timing(c);
-    return rc;
+    return round_body(c, take_round(c, round), act, true, wire, stride_words, bits_out);
 }
 
 int qs_enable_phase_timing(qs_ctx* c, int on) {
@@ -432,9 +435,8 @@ int qs_enable_phase_timing(qs_ctx* c, int on) {
 int qs_get_phase_timing(qs_ctx* c, double* ms, int n) {
     if (!c || !ms) return QS_INVALID_ARG;
     fold_timing(c);
-    const double v[6] = {c->phase_ms[0], c->phase_ms[1], c->phase_ms[2], c->phase_ms[3], c->phase_ms[4],
-                         (double)c->timed_rounds};
-    for (int i = 0; i < n && i < 6; ++i) ms[i] = v[i];
+    const double v[3] = {c->phase_ms[0], c->phase_ms[1], (double)c->timed_rounds};
+    for (int i = 0; i < n && i < 3; ++i) ms[i] = v[i];
     for (double& a : c->phase_ms) a = 0.0;
     c->timed_rounds = 0;
     return QS_OK;
@@ -444,7 +446,7 @@ int qs_export_selection(qs_ctx* c, int64_t* sel_idx, int32_t* level, uint8_t* si
     if (!c) return QS_INVALID_ARG;
     if (!c->compressed) return fail(c, QS_STATE, "nothing compressed yet");
     launch_export(c->P, (long long*)sel_idx, level, sign, norm, (long long*)n, c->sms, c->st);
-    return after_launch(c, N_EXPORT, "export");
+    return after_launch(c, 1, "export");
 }
 
 int64_t qs_wire_words(const qs_ctx* c) { return c ? c->wire_words : (int64_t)QS_INVALID_ARG; }

@@ -85,6 +85,7 @@ struct Plan {
     uint32_t* dec_pay;         // R x nseg
     uint32_t* touch;           // d, zero between rounds
     int* status;
+    uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel
     long long* stats;          // device counters: [0] fallback worker-rounds, [1] candidates
 };
 
