@@ -221,6 +221,14 @@ int qs_get_stats(qs_ctx* ctx, int64_t* out, int n);
 int qs_enable_phase_timing(qs_ctx* ctx, int on);
 int qs_get_phase_timing(qs_ctx* ctx, double* ms, int n);
 
+/*
+ * qs_get_stage_trace — measurement aid: microseconds, from the start of the last persistent
+ * kernel of this context, at which its block 0 reached each grid barrier (us[1], us[2], ...,
+ * -1 = not reached) and left the kernel (us[31]); us[0] = 0.  Synchronises the stream.
+ * Writes min(n, 32) values.
+ */
+int qs_get_stage_trace(qs_ctx* ctx, double* us, int n);
+
 /* Frees the scratch and the context (NULL is allowed). */
 void qs_destroy(qs_ctx* ctx);
 

@@ -22,7 +22,7 @@ EXPORTS = [
     "qs_init", "qs_set_segments", "qs_bind", "qs_local_step", "qs_compress_feedback", "qs_pack",
     "qs_unpack_accumulate", "qs_broadcast", "qs_sync_round", "qs_export_selection", "qs_wire_words",
     "qs_record_bits", "qs_total_k", "qs_sync_status", "qs_last_error", "qs_get_round", "qs_set_round",
-    "qs_get_stats", "qs_enable_phase_timing", "qs_get_phase_timing", "qs_destroy",
+    "qs_get_stats", "qs_enable_phase_timing", "qs_get_phase_timing", "qs_get_stage_trace", "qs_destroy",
 ]
 
 _lib = None
@@ -66,6 +66,7 @@ def lib():
         L.qs_get_stats.argtypes = [vp, vp, C.c_int]
         L.qs_enable_phase_timing.argtypes = [vp, C.c_int]
         L.qs_get_phase_timing.argtypes = [vp, vp, C.c_int]
+        L.qs_get_stage_trace.argtypes = [vp, vp, C.c_int]
         L.qs_destroy.argtypes = [vp]
         L.qs_destroy.restype = None
         _lib = L
@@ -195,6 +196,12 @@ class Context:
         out = np.zeros(3, dtype=np.float64)
         self._check(lib().qs_get_phase_timing(self._h, out.ctypes.data_as(C.c_void_p), 3))
         return {"rounds": int(out[2]), "dense_pass": float(out[0]), "rest_of_round": float(out[1])}
+
+    def stage_trace(self):
+        """Microseconds at which block 0 of the last persistent kernel reached each barrier; last = end."""
+        out = np.zeros(32, dtype=np.float64)
+        self._check(lib().qs_get_stage_trace(self._h, out.ctypes.data_as(C.c_void_p), 32))
+        return [float(v) for v in out]
 
     def new_wire(self):
         return torch.zeros((self.R, self.wire_words()), dtype=torch.int32, device=self._keep[0].device)

@@ -1,6 +1,7 @@
 // C boundary of the sync-round library: context, tables, scratch and the order of launches.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <string>
 #include <vector>
@@ -13,7 +14,7 @@ struct qs_ctx {
     Plan P;
     cudaStream_t st;
     int sms, mid_grid;
-    bool bound, aligned, compressed;
+    bool bound, aligned, compressed, use_tma;
     Active last;                       // workers of the last compression
     std::vector<int64_t> off, kseg;    // host copies of the segment table
     int64_t wire_words;
@@ -238,6 +239,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(touch, (size_t)d, true);
     AL(status, 1, true);
     AL(bar, 2, true);
+    AL(trace, TRACE_SLOTS, true);
     AL(stats, 2, true);
 #undef AL
     QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
@@ -274,10 +276,10 @@ int clear_wire(qs_ctx* c, const Active& act, uint32_t* wire, int64_t stride) {
     return QS_OK;
 }
 
-int run_mid(qs_ctx* c, const Active& act, int do_compress, int do_pack, int do_decode, int patch, uint32_t* wire,
-            int64_t stride, int64_t* bits_out) {
-    const cudaError_t e = launch_mid(c->P, act, do_compress, do_pack, do_decode, patch, wire, stride,
-                                     (long long*)bits_out, c->mid_grid, c->st);
+int run_mid(qs_ctx* c, const Active& act, int do_compress, int do_pack, int do_decode, int do_broadcast,
+            uint32_t* wire, int64_t stride, int64_t* bits_out) {
+    const cudaError_t e = launch_mid(c->P, act, do_compress, do_pack, do_decode, 0, do_broadcast, c->aligned ? 1 : 0,
+                                     wire, stride, (long long*)bits_out, c->mid_grid, c->st);
     if (e != cudaSuccess) return cuda_fail(c, e, "persistent kernel");
     return after_launch(c, 1, "persistent kernel");
 }
@@ -290,7 +292,12 @@ int round_body(qs_ctx* c, uint64_t round, const Active& act, bool fused, uint32_
     P.round_hi = (uint32_t)(round >> 32);
     int rc;
     if (fused) mark(c, 0);
-    launch_pass_a(P, act, fused ? 1 : 0, c->aligned, c->sms, c->st);
+    if (c->use_tma && pass_a_tma_usable(P, c->aligned)) {
+        const cudaError_t e = launch_pass_a_tma(P, act, c->sms, c->st);
+        if (e != cudaSuccess) return cuda_fail(c, e, "pass_a (bulk copy)");
+    } else {
+        launch_pass_a(P, act, 0, c->aligned, c->sms, c->st);
+    }
     if ((rc = after_launch(c, 1, "pass_a")) != QS_OK) return rc;
     if (fused) {
         mark(c, 1);
@@ -324,6 +331,7 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     std::memset(&c->P, 0, sizeof(Plan));
     c->st = static_cast<cudaStream_t>(cuda_stream);
     c->bound = c->aligned = c->compressed = false;
+    c->use_tma = std::getenv("QSPARSE_NO_TMA") == nullptr;
     c->round = 0;
     c->launches = c->rounds = 0;
     c->wire_words = 0;
@@ -486,6 +494,16 @@ uint64_t qs_get_round(const qs_ctx* c) { return c ? c->round : 0; }
 int qs_set_round(qs_ctx* c, uint64_t round) {
     if (!c || round >= (1ull << 56)) return QS_INVALID_ARG;
     c->round = round;
+    return QS_OK;
+}
+
+int qs_get_stage_trace(qs_ctx* c, double* us, int n) {
+    if (!c || !us) return QS_INVALID_ARG;
+    QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    unsigned long long t[TRACE_SLOTS];
+    QS_CUDA_TRY(c, cudaMemcpy(t, c->P.trace, sizeof(t), cudaMemcpyDeviceToHost));
+    // slot 0 = kernel start, slots 1.. = barriers in order (0 = not reached), last slot = kernel end
+    for (int i = 0; i < n && i < TRACE_SLOTS; ++i) us[i] = t[i] ? (double)(t[i] - t[0]) * 1e-3 : -1.0;
     return QS_OK;
 }
 

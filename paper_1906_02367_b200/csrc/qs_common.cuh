@@ -15,6 +15,7 @@ constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (to
 constexpr int FB_SHIFT = 21;
 constexpr int FB_CHUNK = 65536;      // coordinates per fallback-histogram block
 constexpr uint32_t NO_GUESS = 0xFFFFFFFFu;
+constexpr int TRACE_SLOTS = 32;       // time stamps of the persistent kernel's barriers
 
 // cand_q fields
 constexpr uint32_t Q_NEG = 1u << 16;
@@ -86,6 +87,7 @@ struct Plan {
     uint32_t* touch;           // d, zero between rounds
     int* status;
     uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel
+    unsigned long long* trace; // TRACE_SLOTS global-timer stamps of the last persistent launch, or null
     long long* stats;          // device counters: [0] fallback worker-rounds, [1] candidates
 };
 

@@ -37,6 +37,25 @@ __device__ __forceinline__ void store_quad(float* __restrict__ row, uint32_t e0,
     }
 }
 
+// Store that asks the L2 to keep the line: used for the few quads that hold a candidate, which
+// the selection stages read back right after this pass.
+template <bool ALIGNED>
+__device__ __forceinline__ void store_quad_keep(float* __restrict__ row, uint32_t e0, uint32_t d, const float v[4],
+                                                uint64_t policy) {
+    if (ALIGNED) {
+        if (e0 < d)
+            asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(row + e0), "f"(v[0]),
+                         "f"(v[1]), "f"(v[2]), "f"(v[3]), "l"(policy)
+                         : "memory");
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (e0 + j < d)
+                asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(row + e0 + j), "f"(v[j]), "l"(policy)
+                             : "memory");
+    }
+}
+
 constexpr int WB = 4;            // workers whose loads are issued together
 constexpr int TAB_MAX = 11 * 1024;   // words of shared memory for the threshold and offset tables
 
@@ -59,6 +78,8 @@ __global__ void __launch_bounds__(256) pass_a_kernel(const Plan P, const Active 
         seg_off = sh_tab + ng;
     }
     bool bad = false;
+    uint64_t keep;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
     for (uint32_t g = blockIdx.x * 8u + (threadIdx.x >> 5); g < P.ngroups; g += nwarps) {
         const uint32_t e0 = g * (uint32_t)GROUP + (uint32_t)lane * 4u;
         int sg[4] = {0, 0, 0, 0};
@@ -106,7 +127,8 @@ __global__ void __launch_bounds__(256) pass_a_kernel(const Plan P, const Active 
                     const uint32_t sk = RANDK ? ~hh[j] : key;
                     fl[j] = (e0 + j < P.d) && (sk >= gj);
                 }
-                store_quad<ALIGNED>(P.mem + row, e0, P.d, u);
+                if (fl[0] | fl[1] | fl[2] | fl[3]) store_quad_keep<ALIGNED>(P.mem + row, e0, P.d, u, keep);
+                else store_quad<ALIGNED>(P.mem + row, e0, P.d, u);
                 if (mode == 1) {
                     store_quad<ALIGNED>(P.xw + row, e0, P.d, xq);
                     if (ANCH) store_quad<ALIGNED>(P.anchors + row, e0, P.d, xq);

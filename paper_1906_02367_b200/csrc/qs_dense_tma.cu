@@ -1,0 +1,245 @@
+// Dense pass with the bulk-copy engine (TMA) feeding shared memory: the 16-byte-aligned fast path.
+//
+// A block walks tiles of 2048 coordinates (two 128-coordinate groups per warp) and, for every
+// tile, the active workers in turn.  One thread keeps a ring of (xw, mem) tile pairs filling
+// with cp.async.bulk loads several items ahead; each arrival is announced on an mbarrier.  The
+// eight warps read their quads from shared memory, form u = mem + (x - xw), overwrite the mem
+// tile in place, vote the candidate flags into the bitmap, and the finished tile goes back to
+// global memory as one bulk store.  Loads and stores never pass through registers of the
+// computing warps, so the depth of the ring, not the occupancy, sets the bytes in flight.
+//
+// Every wait is bounded: a barrier that does not complete records QS_TIMEOUT, the block waits
+// for its own copies in flight and leaves.
+#include "qs_kernels.h"
+
+namespace qs {
+
+#ifndef QS_TMA_GP
+#define QS_TMA_GP 2
+#endif
+#ifndef QS_TMA_STAGES
+#define QS_TMA_STAGES 3
+#endif
+#ifndef QS_TMA_PER_SM
+#define QS_TMA_PER_SM 3
+#endif
+constexpr int GP = QS_TMA_GP;              // groups of 128 coordinates per warp and tile
+constexpr int TILE = 1024 * GP;            // coordinates per tile: 8 warps x GP groups
+constexpr int STAGES = QS_TMA_STAGES;      // (xw, mem) tile pairs in the ring
+#ifndef QS_TMA_XSLOTS
+#define QS_TMA_XSLOTS 2
+#endif
+constexpr int XSLOTS = QS_TMA_XSLOTS;      // x tiles in their ring
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // give up on an mbarrier after two seconds
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// bounded wait; false when the time limit ran out
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+    }
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_addr(src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+struct TmaSmem {
+    float stage[STAGES][2][TILE];          // [0] xw tile, [1] mem tile (overwritten with u)
+    float xs[XSLOTS][TILE];
+    uint64_t full[STAGES];
+    uint64_t xfull[XSLOTS];
+    int abort_flag;
+};
+
+// Synchronous algorithm only (every worker's reference point is x); rows 16-byte aligned.
+template <bool RANDK>
+__global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Active act, const int prefetch) {
+    extern __shared__ __align__(128) unsigned char sh_raw[];
+    TmaSmem& S = *reinterpret_cast<TmaSmem*>(sh_raw);
+    uint32_t* tab = reinterpret_cast<uint32_t*>(sh_raw + sizeof(TmaSmem));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ntiles = (P.d + TILE - 1) / TILE;
+    const int nact = act.n;
+    // thresholds of all workers, then segment offsets
+    const uint32_t ng = (uint32_t)P.R * P.nseg;
+    for (uint32_t i = threadIdx.x; i < ng; i += 256) tab[i] = P.guess[i];
+    for (uint32_t i = threadIdx.x; i <= (uint32_t)P.nseg; i += 256) tab[ng + i] = P.seg_off[i];
+    const uint32_t* seg_off = tab + ng;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) mbar_init(&S.full[s], 1);
+        for (int s = 0; s < XSLOTS; ++s) mbar_init(&S.xfull[s], 1);
+        S.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // items of this block: tile iteration `it` (tile = blockIdx.x + it * gridDim.x) x active worker
+    const uint32_t my_tiles = blockIdx.x < ntiles ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint64_t nitems = (uint64_t)my_tiles * nact;
+
+    auto issue = [&](uint64_t j) {           // thread 0: start the loads of item j
+        const uint32_t it = (uint32_t)(j / nact);
+        const int w = (int)(j % nact);
+        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        const uint32_t e0 = tile * TILE;
+        const uint32_t bytes = (P.d - e0 < TILE ? P.d - e0 : TILE) * 4u;
+        const int s = (int)(j % STAGES);
+        const size_t row = (size_t)act.r[w] * P.d + e0;
+        if (w == 0) {
+            const int xsl = (int)(it % XSLOTS);
+            mbar_expect(&S.xfull[xsl], bytes);
+            bulk_load(S.xs[xsl], P.x + e0, bytes, &S.xfull[xsl]);
+        }
+        mbar_expect(&S.full[s], 2u * bytes);
+        bulk_load(S.stage[s][0], P.xw + row, bytes, &S.full[s]);
+        bulk_load(S.stage[s][1], P.mem + row, bytes, &S.full[s]);
+    };
+
+    if (threadIdx.x == 0)
+        for (uint64_t j = 0; j < (uint64_t)prefetch && j < nitems; ++j) issue(j);
+
+    bool bad = false;
+    int sg[GP][4] = {};                      // segments of this lane's quads, refreshed once per tile
+    uint64_t j = 0;
+    for (; j < nitems; ++j) {
+        const uint32_t it = (uint32_t)(j / nact);
+        const int w = (int)(j % nact);
+        const int r = act.r[w];
+        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        const int s = (int)(j % STAGES), xsl = (int)(it % XSLOTS);
+        if (threadIdx.x == 0 && j + prefetch < nitems) {
+            bulk_wait_read<1>();             // the ring slot about to be refilled has been read by its store
+            issue(j + prefetch);
+        }
+        bool ok = mbar_wait(&S.full[s], (uint32_t)((j / STAGES) & 1));
+        if (w == 0) ok = ok && mbar_wait(&S.xfull[xsl], (uint32_t)((it / XSLOTS) & 1));
+        if (!ok) S.abort_flag = 1;           // seen by everyone at the barrier below
+
+        const uint32_t* gs = tab + (size_t)r * P.nseg;
+#pragma unroll
+        for (int k = 0; k < GP; ++k) {
+            const uint32_t g = tile * (TILE / GROUP) + warp * GP + k;
+            const uint32_t q = (warp * GP + k) * GROUP + lane * 4;   // offset inside the tile
+            const uint32_t e0 = tile * TILE + q;
+            if (w == 0 && P.nseg > 1) {
+                int sq = g < P.ngroups ? (int)P.grp_seg[g] : 0;
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    while (sq + 1 < P.nseg && e0 + jj >= seg_off[sq + 1]) ++sq;
+                    sg[k][jj] = sq;
+                }
+            }
+            const float4 xq = *reinterpret_cast<const float4*>(&S.xs[xsl][q]);
+            const float4 wq = *reinterpret_cast<const float4*>(&S.stage[s][0][q]);
+            const float4 mq = *reinterpret_cast<const float4*>(&S.stage[s][1][q]);
+            float4 u;
+            u.x = mq.x + (xq.x - wq.x);
+            u.y = mq.y + (xq.y - wq.y);
+            u.z = mq.z + (xq.z - wq.z);
+            u.w = mq.w + (xq.w - wq.w);
+            *reinterpret_cast<float4*>(&S.stage[s][1][q]) = u;
+            const bool in = e0 < P.d;                            // d is a multiple of 4: whole quads
+            const uint32_t key[4] = {topk_key(u.x), topk_key(u.y), topk_key(u.z), topk_key(u.w)};
+            uint32_t sk[4] = {key[0], key[1], key[2], key[3]};
+            if (RANDK) {
+                const uint4 h = philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
+                sk[0] = ~h.x; sk[1] = ~h.y; sk[2] = ~h.z; sk[3] = ~h.w;
+            }
+            uint32_t fl[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) fl[jj] = in && sk[jj] >= gs[sg[k][jj]];
+            if (in) bad |= (key[0] >= 0xFF000000u) | (key[1] >= 0xFF000000u) | (key[2] >= 0xFF000000u) | (key[3] >= 0xFF000000u);
+            const uint32_t b0 = __ballot_sync(0xffffffffu, fl[0]);
+            const uint32_t b1 = __ballot_sync(0xffffffffu, fl[1]);
+            const uint32_t b2 = __ballot_sync(0xffffffffu, fl[2]);
+            const uint32_t b3 = __ballot_sync(0xffffffffu, fl[3]);
+            if (lane == 0 && g < P.ngroups) {
+                reinterpret_cast<uint4*>(P.bitmap)[(size_t)r * P.ngroups + g] = make_uint4(b0, b1, b2, b3);
+                const uint32_t cnt = __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+                if (cnt) atomicAdd(&P.blk_count[(size_t)r * P.nblk + g / EMIT_GROUPS], cnt);
+            }
+        }
+        fence_async_smem();                  // the tile written above must be visible to the bulk store
+        __syncthreads();
+        if (S.abort_flag) break;
+        if (threadIdx.x == 0) {
+            const uint32_t t0 = tile * TILE;
+            const uint32_t bytes = (P.d - t0 < TILE ? P.d - t0 : TILE) * 4u;
+            bulk_store(P.mem + (size_t)r * P.d + t0, S.stage[s][1], bytes);
+            bulk_commit();
+        }
+    }
+    if (threadIdx.x == 0) {
+        if (S.abort_flag) {
+            // give the loads already issued a bounded chance to land before the block leaves
+            for (uint64_t jj = j; jj < nitems && jj < j + (uint64_t)prefetch; ++jj)
+                mbar_wait(&S.full[jj % STAGES], (uint32_t)((jj / STAGES) & 1));
+            set_status(P, QS_TIMEOUT);
+        }
+        bulk_wait_all();                     // nothing of this block may still be reading shared memory
+    }
+    if (bad) set_status(P, QS_NONFINITE);
+}
+
+size_t pass_a_tma_smem(const Plan& P) { return sizeof(TmaSmem) + ((size_t)P.R * P.nseg + P.nseg + 1) * 4; }
+
+bool pass_a_tma_usable(const Plan& P, bool aligned) {
+    return aligned && !P.anchors && pass_a_tma_smem(P) <= 100 * 1024;
+}
+
+cudaError_t launch_pass_a_tma(const Plan& P, const Active& act, int sms, cudaStream_t st) {
+    const size_t smem = pass_a_tma_smem(P);
+    const bool rk = P.sp == QS_RANDK;
+    cudaError_t e = rk ? cudaFuncSetAttribute(pass_a_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                       : cudaFuncSetAttribute(pass_a_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const uint32_t ntiles = (P.d + TILE - 1) / TILE;
+    const uint32_t cap = (uint32_t)sms * (uint32_t)QS_TMA_PER_SM;
+    const int grid = (int)(ntiles < cap ? ntiles : cap);
+    int prefetch = STAGES - 2;
+    if (prefetch > (XSLOTS - 1) * act.n) prefetch = (XSLOTS - 1) * act.n;   // an x slot is refilled only after its tile is done
+    if (rk) pass_a_tma_kernel<true><<<grid, 256, smem, st>>>(P, act, prefetch);
+    else pass_a_tma_kernel<false><<<grid, 256, smem, st>>>(P, act, prefetch);
+    return cudaGetLastError();
+}
+
+}  // namespace qs

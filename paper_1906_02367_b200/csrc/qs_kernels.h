@@ -9,10 +9,14 @@ void launch_pass_a(const Plan& P, const Active& act, int mode, bool aligned, int
 void launch_broadcast(const Plan& P, const Active& act, bool aligned, int sms, cudaStream_t st);
 void launch_local_step(const Plan& P, const Active& act, const float* grad, float eta, bool aligned,
                        int sms, cudaStream_t st);
+// qs_dense_tma.cu: the dense pass fed by bulk copies (aligned rows, synchronous algorithm)
+bool pass_a_tma_usable(const Plan& P, bool aligned);
+cudaError_t launch_pass_a_tma(const Plan& P, const Active& act, int sms, cudaStream_t st);
 // qs_mid.cu: the persistent kernel that runs every stage after the dense pass
 int mid_blocks_per_sm(bool randk);
 cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode, int patch,
-                       uint32_t* wire, long long stride, long long* bits_out, int grid, cudaStream_t st);
+                       int do_broadcast, int aligned, uint32_t* wire, long long stride, long long* bits_out, int grid,
+                       cudaStream_t st);
 void launch_export(const Plan& P, long long* sel_idx, int* level, uint8_t* sign, float* norm, long long* n,
                    int sms, cudaStream_t st);
 

@@ -29,7 +29,7 @@ constexpr uint32_t SPIN_LIMIT = 1u << 22;  // barrier polls before giving up (ab
 struct MidArgs {
     Plan P;
     Active act;
-    int do_compress, do_pack, do_decode, patch;
+    int do_compress, do_pack, do_decode, patch, do_broadcast, aligned;
     uint32_t* wire;
     long long stride;
     long long* bits_out;
@@ -47,6 +47,12 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
 __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, int* sh_abort) {
     target += gridDim.x;
     __syncthreads();
+    if (P.trace && blockIdx.x == 0 && threadIdx.x == 0) {     // stage boundaries as block 0 sees them
+        const uint32_t slot = target / gridDim.x;
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        if (slot < TRACE_SLOTS) P.trace[slot] = t;
+    }
     if (threadIdx.x == 0) {
         __threadfence();
         atomicAdd(P.bar, 1u);
@@ -895,6 +901,31 @@ __device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t
     }
 }
 
+// xw_r <- x (and the anchors) for the active workers: the closing dense stage of a fused round
+template <bool ALIGNED>
+__device__ void stage_broadcast(const Plan& P, const Active& act) {
+    const int lane = threadIdx.x & 31;
+    for (uint32_t g = blockIdx.x * (BT / 32) + (threadIdx.x >> 5); g < P.ngroups; g += gridDim.x * (BT / 32)) {
+        const uint32_t e0 = g * (uint32_t)GROUP + (uint32_t)lane * 4u;
+        if (e0 >= P.d) continue;
+        if (ALIGNED) {
+            const float4 v = *reinterpret_cast<const float4*>(P.x + e0);
+            for (int w = 0; w < act.n; ++w) {
+                __stcs(reinterpret_cast<float4*>(P.xw + (size_t)act.r[w] * P.d + e0), v);
+                if (P.anchors) __stcs(reinterpret_cast<float4*>(P.anchors + (size_t)act.r[w] * P.d + e0), v);
+            }
+        } else {
+            for (uint32_t j = 0; j < 4 && e0 + j < P.d; ++j) {
+                const float v = P.x[e0 + j];
+                for (int w = 0; w < act.n; ++w) {
+                    P.xw[(size_t)act.r[w] * P.d + e0 + j] = v;
+                    if (P.anchors) P.anchors[(size_t)act.r[w] * P.d + e0 + j] = v;
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------ the persistent kernel
 template <bool RANDK>
 __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
@@ -908,6 +939,12 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     uint32_t* bins = reinterpret_cast<uint32_t*>(sh_big);
     if (threadIdx.x == 0) sh_abort = 0;
     uint32_t target = 0;
+    if (P.trace && blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        P.trace[0] = t;
+        for (int i = 1; i < TRACE_SLOTS; ++i) P.trace[i] = 0;
+    }
 #define QS_BARRIER() do { if (!grid_barrier(P, target, &sh_abort)) return; } while (0)
 
     if (a.do_compress) {
@@ -960,9 +997,19 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
         QS_BARRIER();
         stage_dec_apply(P, act, a.wire, a.stride, a.patch);
     }
+    if (a.do_broadcast) {
+        QS_BARRIER();
+        if (a.aligned) stage_broadcast<true>(P, act);
+        else stage_broadcast<false>(P, act);
+    }
 #undef QS_BARRIER
     // the last block to leave resets the barrier for the next launch
     __syncthreads();
+    if (P.trace && blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        P.trace[TRACE_SLOTS - 1] = t;
+    }
     if (threadIdx.x == 0) {
         if (atomicAdd(P.bar + 1, 1u) == gridDim.x - 1) {
             P.bar[0] = 0;
@@ -995,10 +1042,12 @@ int mid_blocks_per_sm(bool randk) {
 }
 
 cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode, int patch,
-                       uint32_t* wire, long long stride, long long* bits_out, int grid, cudaStream_t st) {
+                       int do_broadcast, int aligned, uint32_t* wire, long long stride, long long* bits_out, int grid,
+                       cudaStream_t st) {
     MidArgs a;
     a.P = P; a.act = act;
     a.do_compress = do_compress; a.do_pack = do_pack; a.do_decode = do_decode; a.patch = patch;
+    a.do_broadcast = do_broadcast; a.aligned = aligned;
     a.wire = wire; a.stride = stride; a.bits_out = bits_out;
     void* params[] = {&a};
     const void* fn = P.sp == QS_RANDK ? (const void*)mid_kernel<true> : (const void*)mid_kernel<false>;
