@@ -57,7 +57,8 @@ enum {
     QS_CAPACITY = -4,    /* caller's wire stride is smaller than qs_wire_words         */
     QS_NONFINITE = -5,   /* an inf or NaN reached the compressor (device status)       */
     QS_STATE = -6,       /* call out of order (no buffers bound, nothing compressed)   */
-    QS_TIMEOUT = -7      /* a bounded device-side wait ran out (device status)         */
+    QS_TIMEOUT = -7,     /* a bounded device-side wait ran out (device status)         */
+    QS_TOO_LARGE = -8    /* d beyond QS_STATIC_MAX_D (qs_unpack_accumulate_static only) */
 };
 
 /* Sparsifiers of Section 2.2. */
@@ -228,6 +229,39 @@ int qs_get_phase_timing(qs_ctx* ctx, double* ms, int n);
  * Writes min(n, 32) values.
  */
 int qs_get_stage_trace(qs_ctx* ctx, double* us, int n);
+
+/*
+ * qs_unpack_accumulate_static — the master update of qs_unpack_accumulate for callers that
+ * must not allocate.  (The paper has no counterpart: this entry point exists for deployment,
+ * not for the method.)
+ *
+ * Who needs it: code that cannot call cudaMalloc when the update has to run — a serving or
+ * training loop in which an allocation would synchronise the whole device, a process whose
+ * device memory is owned and handed out by another component, a job whose memory budget is
+ * already spent.  qs_init allocates, so this call takes no context: the operator is described
+ * by plain arguments, and the one piece of scratch the decode needs (a word per coordinate
+ * recording which workers sent it) lives in a fixed array inside the library image.  Every GPU
+ * that loads the library therefore holds QS_STATIC_MAX_D words (4 MiB) until the process ends.
+ *
+ *   R, d, k, s, quantizer   as in qs_init, one segment [0, d); d <= QS_STATIC_MAX_D, else
+ *                           QS_TOO_LARGE is returned and nothing is enqueued.
+ *   x (device, d)           updated in place: acc = 0; acc += g_r in increasing r;
+ *                           x <- x - acc / R, at every index some masked worker sent.
+ *   wire (device), stride_words, worker_mask (host, R bytes or NULL)
+ *                           records in the format of qs_pack; QS_CAPACITY if stride_words is
+ *                           below the size of a full record.  A record whose count exceeds k,
+ *                           or an index >= d, is skipped, never followed.
+ *   cuda_stream             the work (one memset, two kernels) is enqueued there.
+ * It calls no allocator.  The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current): make that first call outside any stream
+ * capture.  The array is shared by all calls on a device and keeps the last call's contents;
+ * each call clears the d words it uses before use, and calls that overlap in time on one GPU
+ * (two streams, two threads) race on it — issue them one after another.
+ */
+#define QS_STATIC_MAX_D (1 << 20)
+int qs_unpack_accumulate_static(int R, int64_t d, int64_t k, int s, int quantizer, float* x,
+                                const uint32_t* wire, int64_t stride_words,
+                                const uint8_t* worker_mask, void* cuda_stream);
 
 /* Frees the scratch and the context (NULL is allowed). */
 void qs_destroy(qs_ctx* ctx);

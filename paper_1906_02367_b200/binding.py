@@ -14,6 +14,8 @@ from . import build as _build
 
 QS_OK = 0
 QS_INVALID_ARG, QS_ALLOC, QS_CUDA, QS_CAPACITY, QS_NONFINITE, QS_STATE, QS_TIMEOUT = -1, -2, -3, -4, -5, -6, -7
+QS_TOO_LARGE = -8
+QS_STATIC_MAX_D = 1 << 20
 QS_TOPK, QS_RANDK = 0, 1
 QS_QSGD, QS_QSGD_SCALED, QS_SIGN_L1 = 0, 1, 2
 QS_ROUND_AUTO = 2**64 - 1
@@ -22,7 +24,8 @@ EXPORTS = [
     "qs_init", "qs_set_segments", "qs_bind", "qs_local_step", "qs_compress_feedback", "qs_pack",
     "qs_unpack_accumulate", "qs_broadcast", "qs_sync_round", "qs_export_selection", "qs_wire_words",
     "qs_record_bits", "qs_total_k", "qs_sync_status", "qs_last_error", "qs_get_round", "qs_set_round",
-    "qs_get_stats", "qs_enable_phase_timing", "qs_get_phase_timing", "qs_get_stage_trace", "qs_destroy",
+    "qs_get_stats", "qs_enable_phase_timing", "qs_get_phase_timing", "qs_get_stage_trace", "qs_unpack_accumulate_static",
+    "qs_destroy",
 ]
 
 _lib = None
@@ -67,6 +70,7 @@ def lib():
         L.qs_enable_phase_timing.argtypes = [vp, C.c_int]
         L.qs_get_phase_timing.argtypes = [vp, vp, C.c_int]
         L.qs_get_stage_trace.argtypes = [vp, vp, C.c_int]
+        L.qs_unpack_accumulate_static.argtypes = [C.c_int, i64, i64, C.c_int, C.c_int, vp, vp, i64, vp, vp]
         L.qs_destroy.argtypes = [vp]
         L.qs_destroy.restype = None
         _lib = L
@@ -89,6 +93,15 @@ def _mask(mask, R):
     m = np.ascontiguousarray(mask, dtype=np.uint8)
     assert m.size == R
     return m, m.ctypes.data_as(C.c_void_p)
+
+
+def unpack_accumulate_static(R, d, k, s, quantizer, x, wire, mask=None, stream=None):
+    """qs_unpack_accumulate_static: the master update without a context and without allocating.
+    Returns the status code (0 on success) instead of raising, so that callers can test limits."""
+    m, mp = _mask(mask, R)
+    st = stream if stream is not None else torch.cuda.current_stream()
+    return int(lib().qs_unpack_accumulate_static(int(R), int(d), int(k), int(s), int(quantizer), _ptr(x), _ptr(wire),
+                                                 int(wire.shape[1]), mp, C.c_void_p(st.cuda_stream)))
 
 
 class Context:
