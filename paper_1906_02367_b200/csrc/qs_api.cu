@@ -141,6 +141,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     const int64_t d = (int64_t)P.d;
     if (nseg < 1 || !offsets || !kseg || offsets[0] != 0 || offsets[nseg] != d)
         return fail(c, QS_INVALID_ARG, "segments must start at 0 and end at d");
+    if ((int64_t)P.R * nseg > UT_MAX) return fail(c, QS_INVALID_ARG, "R x nseg exceeds the unit table (2048)");
     for (int g = 0; g < nseg; ++g) {
         const int64_t n = offsets[g + 1] - offsets[g];
         if (n < 1 || kseg[g] < 1 || kseg[g] > n) return fail(c, QS_INVALID_ARG, "need 1 <= k_seg <= segment length");
@@ -155,7 +156,9 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.nseg = nseg;
     P.U = (uint32_t)R * nseg;
     P.ngroups = (uint32_t)((d + GROUP - 1) / GROUP);
-    P.nblk = (P.ngroups + EMIT_GROUPS - 1) / EMIT_GROUPS;
+    P.ntile = (uint32_t)((d + STILE - 1) / STILE);
+    P.nblk = (P.ntile + BLK_TILES - 1) / BLK_TILES;
+    P.nsup = (P.nblk + SUP_BLOCKS - 1) / SUP_BLOCKS;
     P.cap = (uint64_t)d;
     P.bl = std::max(1, ceil_log2((uint64_t)P.s));
     P.maxchunks = (uint32_t)R * (uint32_t)((d + CHUNK - 1) / CHUNK + nseg);
@@ -213,10 +216,12 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     if ((rc = dev_upload(c, &g_up, h_guess)) != QS_OK) return rc;
     P.guess = const_cast<uint32_t*>(g_up);
 #define AL(field, count, zero) if ((rc = dev_alloc(c, &P.field, (size_t)(count), zero)) != QS_OK) return rc
-    AL(bitmap, (size_t)R * P.ngroups * 4, true);
+    AL(stage_idx, (size_t)R * P.cap, false);
+    AL(stage_val, (size_t)R * P.cap, false);
+    AL(tile_cnt, (size_t)R * P.ntile, true);
     AL(blk_count, (size_t)R * P.nblk, true);
-    AL(blk_base, (size_t)R * P.nblk, true);
-    AL(ncand, R, true);
+    AL(sup_count, (size_t)R * P.nsup, true);
+    AL(seg_start, (size_t)R * (nseg + 1), true);
     AL(fail, R, true);
     AL(units, P.U, true);
     AL(total_chunks, 1, true);
@@ -257,6 +262,7 @@ int rezero(qs_ctx* c) {
     QS_CUDA_TRY(c, cudaMemsetAsync(P.status, 0, sizeof(int), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 2 * sizeof(uint32_t), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.blk_count, 0, sizeof(uint32_t) * P.R * P.nblk, c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.sup_count, 0, sizeof(uint32_t) * P.R * P.nsup, c->st));
     return QS_OK;
 }
 

@@ -8,9 +8,13 @@
 namespace qs {
 
 constexpr int MAX_R = 32;            // decode keeps one bit per worker in a 32-bit word
-constexpr int GROUP = 128;           // coordinates per candidate-bitmap group (one warp, 4 each)
-constexpr int EMIT_GROUPS = 256;     // groups per candidate-emission block (32768 coordinates)
+constexpr int GROUP = 128;           // coordinates one warp handles at a time (4 per lane)
+constexpr int GPW = 2;               // groups per warp in a tile
+constexpr int STILE = 8 * GPW * GROUP;   // coordinates per tile: 8 warps x GPW groups = 2048
+constexpr int BLK_TILES = 16;        // tiles per candidate block (32768 coordinates)
+constexpr int SUP_BLOCKS = 64;       // blocks per super-block of the two-level candidate counts
 constexpr int CHUNK = 2048;          // candidates per selection chunk (256 threads x 8)
+constexpr int UT_MAX = 2048;         // units whose table fits in the persistent kernel's shared memory
 constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (top 11 key bits)
 constexpr int FB_SHIFT = 21;
 constexpr int FB_CHUNK = 65536;      // coordinates per fallback-histogram block
@@ -45,7 +49,7 @@ struct FbBlock {         // fallback histogram work item: one stretch of one seg
 
 struct Plan {
     int R, nseg, s, sp, qz, bl;
-    uint32_t d, ngroups, nblk, K, U, nfb, maxchunks;
+    uint32_t d, ngroups, ntile, nblk, nsup, K, U, nfb, maxchunks;
     uint32_t seed_lo, seed_hi, round_lo, round_hi;
     uint64_t cap;
     // tables (device)
@@ -61,10 +65,12 @@ struct Plan {
     float* x; float* xw; float* mem; float* anchors;
     // scratch
     uint32_t* guess;           // R x nseg, sort-key space
-    uint32_t* bitmap;          // R x ngroups x 4
-    uint32_t* blk_count;       // R x nblk
-    uint32_t* blk_base;        // R x nblk
-    uint32_t* ncand;           // R
+    uint32_t* stage_idx;       // R x cap: candidates as the dense pass left them, tile t at t * STILE
+    float* stage_val;          // R x cap
+    uint32_t* tile_cnt;        // R x ntile
+    uint32_t* blk_count;       // R x nblk, zero between rounds
+    uint32_t* sup_count;       // R x nsup, zero between rounds
+    uint32_t* seg_start;       // R x (nseg + 1): first candidate of each segment in the ordered list
     uint32_t* fail;            // R
     Unit* units;               // U = R x nseg
     uint32_t* total_chunks;    // 1
@@ -116,6 +122,53 @@ __device__ __forceinline__ uint32_t philox_word(const Plan& P, uint32_t worker, 
     const uint4 o = philox_quad(P, worker, e >> 2, stream);
     const uint32_t j = e & 3u;
     return j == 0 ? o.x : j == 1 ? o.y : j == 2 ? o.z : o.w;
+}
+
+// Candidates of one tile, written by the block that just formed u for it (8 warps, warp w owns
+// groups GPW w .. GPW w + GPW - 1).  bal[k][j]: ballot of "coordinate 4 lane + j of group k is a
+// candidate".  Phase 1 publishes the group counts; after a block-wide barrier phase 2 writes the
+// tile's candidates in ascending coordinate order at the tile's fixed place, and the counts.
+__device__ __forceinline__ void tile_counts(uint32_t* sh_cnt, int warp, int lane, const uint32_t bal[GPW][4]) {
+    if (lane == 0) {
+#pragma unroll
+        for (int k = 0; k < GPW; ++k)
+            sh_cnt[warp * GPW + k] = __popc(bal[k][0]) + __popc(bal[k][1]) + __popc(bal[k][2]) + __popc(bal[k][3]);
+    }
+}
+
+__device__ __forceinline__ void tile_write(const Plan& P, int r, uint32_t tile, const uint32_t* sh_cnt, int warp,
+                                           int lane, const uint32_t bal[GPW][4], const float u[GPW][4]) {
+    uint32_t base = 0, total = 0;
+#pragma unroll
+    for (int i = 0; i < 8 * GPW; ++i) {
+        const uint32_t c = sh_cnt[i];
+        if (i < warp * GPW) base += c;
+        total += c;
+    }
+    if (total == 0) {
+        if (threadIdx.x == 0) P.tile_cnt[(size_t)r * P.ntile + tile] = 0;
+        return;
+    }
+    const size_t off = (size_t)r * P.cap + (size_t)tile * STILE;
+    const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+    for (int k = 0; k < GPW; ++k) {
+        uint32_t pos = base + __popc(bal[k][0] & lt) + __popc(bal[k][1] & lt) + __popc(bal[k][2] & lt) + __popc(bal[k][3] & lt);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if ((bal[k][j] >> lane) & 1u) {
+                P.stage_idx[off + pos] = tile * (uint32_t)STILE + (uint32_t)((warp * GPW + k) * GROUP + lane * 4 + j);
+                P.stage_val[off + pos] = u[k][j];
+                ++pos;
+            }
+        base += sh_cnt[warp * GPW + k];
+    }
+    if (threadIdx.x == 0) {
+        P.tile_cnt[(size_t)r * P.ntile + tile] = total;
+        const uint32_t blk = tile / BLK_TILES;
+        atomicAdd(&P.blk_count[(size_t)r * P.nblk + blk], total);
+        atomicAdd(&P.sup_count[(size_t)r * P.nsup + blk / SUP_BLOCKS], total);
+    }
 }
 
 // Sort key: larger = kept first.  Top_k: |u| bit pattern (shifted up by the spare sign bit);

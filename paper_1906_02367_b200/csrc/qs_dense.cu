@@ -1,13 +1,13 @@
 // Dense passes of the sync round: everything that touches all R x d coordinates.
 //
-//   pass_a      u = mem + (anchor - xw) written over mem, candidate bitmap against the
-//               predicted threshold with per-block candidate counts, and (fused round) the
-//               broadcast of the old model
+//   pass_a      u = mem + (anchor - xw) written over mem, and the candidates (coordinates whose
+//               key passes the predicted threshold) written out per tile, in order
 //   broadcast   xw_r <- x,   local_step  xw_r <- xw_r - eta grad_r
 //
-// One warp owns a group of 128 consecutive coordinates (4 per lane, one 128-bit access
-// per array) and loops over the workers with the model quad held in registers, so x is
-// read once for all R workers.
+// One warp owns groups of 128 consecutive coordinates (4 per lane, one 128-bit access per
+// array) and loops over the workers with the model quads held in registers, so x is read once
+// for all R workers.  This file holds the general path; the aligned synchronous case runs the
+// bulk-copy version of the pass.
 #include "qs_kernels.h"
 
 namespace qs {
@@ -37,36 +37,18 @@ __device__ __forceinline__ void store_quad(float* __restrict__ row, uint32_t e0,
     }
 }
 
-// Store that asks the L2 to keep the line: used for the few quads that hold a candidate, which
-// the selection stages read back right after this pass.
-template <bool ALIGNED>
-__device__ __forceinline__ void store_quad_keep(float* __restrict__ row, uint32_t e0, uint32_t d, const float v[4],
-                                                uint64_t policy) {
-    if (ALIGNED) {
-        if (e0 < d)
-            asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(row + e0), "f"(v[0]),
-                         "f"(v[1]), "f"(v[2]), "f"(v[3]), "l"(policy)
-                         : "memory");
-    } else {
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (e0 + j < d)
-                asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(row + e0 + j), "f"(v[j]), "l"(policy)
-                             : "memory");
-    }
-}
-
-constexpr int WB = 4;            // workers whose loads are issued together
 constexpr int TAB_MAX = 11 * 1024;   // words of shared memory for the threshold and offset tables
 
-// mode 0: compress only; mode 1: fused round (xw_r, and anchors_r if bound, receive x).
-// Shared memory holds the candidate thresholds of all workers and the segment offsets when
-// they fit (tab != 0), so that the inner loop never waits on global memory for them.
+// General dense pass: any alignment, either algorithm (anchors bound or not).  A block handles a
+// tile of 2048 coordinates (warp w owns groups 2w and 2w+1) for the active workers in turn:
+// plain loads, u = mem + (anchor - xw) written over mem, candidate flags voted per group and the
+// tile's candidates written out in order.  mode 1 also writes x into xw_r (and anchors_r).
+// Shared memory holds the thresholds of all workers and the segment offsets when they fit.
 template <bool ALIGNED, bool RANDK, bool ANCH>
 __global__ void __launch_bounds__(256) pass_a_kernel(const Plan P, const Active act, const int mode, const int tab) {
     extern __shared__ uint32_t sh_tab[];
-    const int lane = threadIdx.x & 31;
-    const uint32_t nwarps = gridDim.x * 8u;
+    __shared__ uint32_t sh_cnt[2][8 * GPW];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t* guess = P.guess;
     const uint32_t* seg_off = P.seg_off;
     if (tab) {
@@ -78,71 +60,64 @@ __global__ void __launch_bounds__(256) pass_a_kernel(const Plan P, const Active 
         seg_off = sh_tab + ng;
     }
     bool bad = false;
-    uint64_t keep;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
-    for (uint32_t g = blockIdx.x * 8u + (threadIdx.x >> 5); g < P.ngroups; g += nwarps) {
-        const uint32_t e0 = g * (uint32_t)GROUP + (uint32_t)lane * 4u;
-        int sg[4] = {0, 0, 0, 0};
-        if (P.nseg > 1) {
-            int sq = (int)P.grp_seg[g];
+    uint32_t item = 0;
+    for (uint32_t tile = blockIdx.x; tile < P.ntile; tile += gridDim.x) {
+        int sg[GPW][4] = {};
+        float xq[GPW][4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                while (sq + 1 < P.nseg && e0 + j >= seg_off[sq + 1]) ++sq;
-                sg[j] = sq;
-            }
-        }
-        float xq[4];
-        load_quad<ALIGNED>(P.x, e0, P.d, xq);
-        for (int w0 = 0; w0 < act.n; w0 += WB) {
-            float xw[WB][4], mm[WB][4], an[ANCH ? WB : 1][4];
+        for (int k = 0; k < GPW; ++k) {
+            const uint32_t g = tile * (uint32_t)(STILE / GROUP) + warp * GPW + k;
+            const uint32_t e0 = g * (uint32_t)GROUP + (uint32_t)lane * 4u;
+            if (P.nseg > 1) {
+                int sq = g < P.ngroups ? (int)P.grp_seg[g] : 0;
 #pragma unroll
-            for (int b = 0; b < WB; ++b) {
-                if (w0 + b < act.n) {
-                    const size_t row = (size_t)act.r[w0 + b] * P.d;
-                    load_quad<ALIGNED>(P.xw + row, e0, P.d, xw[b]);
-                    load_quad<ALIGNED>(P.mem + row, e0, P.d, mm[b]);
-                    if (ANCH) load_quad<ALIGNED>(P.anchors + row, e0, P.d, an[ANCH ? b : 0]);
+                for (int j = 0; j < 4; ++j) {
+                    while (sq + 1 < P.nseg && e0 + j >= seg_off[sq + 1]) ++sq;
+                    sg[k][j] = sq;
                 }
             }
+            load_quad<ALIGNED>(P.x, e0, P.d, xq[k]);
+        }
+        for (int w = 0; w < act.n; ++w, ++item) {
+            const int r = act.r[w];
+            const size_t row = (size_t)r * P.d;
+            const uint32_t* gs = guess + (size_t)r * P.nseg;
+            float xw[GPW][4], mm[GPW][4], an[ANCH ? GPW : 1][4];
 #pragma unroll
-            for (int b = 0; b < WB; ++b) {
-                if (w0 + b >= act.n) break;
-                const int r = act.r[w0 + b];
-                const size_t row = (size_t)r * P.d;
-                const uint32_t* gs = guess + (size_t)r * P.nseg;
+            for (int k = 0; k < GPW; ++k) {
+                const uint32_t e0 = (tile * (uint32_t)(STILE / GROUP) + warp * GPW + k) * (uint32_t)GROUP + (uint32_t)lane * 4u;
+                load_quad<ALIGNED>(P.xw + row, e0, P.d, xw[k]);
+                load_quad<ALIGNED>(P.mem + row, e0, P.d, mm[k]);
+                if (ANCH) load_quad<ALIGNED>(P.anchors + row, e0, P.d, an[ANCH ? k : 0]);
+            }
+            uint32_t bal[GPW][4];
+            float u[GPW][4];
+#pragma unroll
+            for (int k = 0; k < GPW; ++k) {
+                const uint32_t e0 = (tile * (uint32_t)(STILE / GROUP) + warp * GPW + k) * (uint32_t)GROUP + (uint32_t)lane * 4u;
                 uint4 h = make_uint4(0, 0, 0, 0);
                 if (RANDK) h = philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
                 const uint32_t hh[4] = {h.x, h.y, h.z, h.w};
-                float u[4];
-                uint32_t fl[4];
-                const uint32_t g0 = gs[sg[0]];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const float anchor = ANCH ? an[ANCH ? b : 0][j] : xq[j];
-                    const float diff = anchor - xw[b][j];
-                    u[j] = mm[b][j] + diff;
-                    const uint32_t key = topk_key(u[j]);
-                    bad |= key >= 0xFF000000u;
-                    const uint32_t gj = (sg[j] == sg[0]) ? g0 : gs[sg[j]];
+                    const float anchor = ANCH ? an[ANCH ? k : 0][j] : xq[k][j];
+                    const float diff = anchor - xw[k][j];
+                    u[k][j] = mm[k][j] + diff;
+                    const uint32_t key = topk_key(u[k][j]);
+                    const bool in = e0 + j < P.d;
+                    if (in) bad |= key >= 0xFF000000u;
                     const uint32_t sk = RANDK ? ~hh[j] : key;
-                    fl[j] = (e0 + j < P.d) && (sk >= gj);
+                    bal[k][j] = __ballot_sync(0xffffffffu, in && sk >= gs[sg[k][j]]);
                 }
-                if (fl[0] | fl[1] | fl[2] | fl[3]) store_quad_keep<ALIGNED>(P.mem + row, e0, P.d, u, keep);
-                else store_quad<ALIGNED>(P.mem + row, e0, P.d, u);
+                store_quad<ALIGNED>(P.mem + row, e0, P.d, u[k]);
                 if (mode == 1) {
-                    store_quad<ALIGNED>(P.xw + row, e0, P.d, xq);
-                    if (ANCH) store_quad<ALIGNED>(P.anchors + row, e0, P.d, xq);
-                }
-                const uint32_t b0 = __ballot_sync(0xffffffffu, fl[0]);
-                const uint32_t b1 = __ballot_sync(0xffffffffu, fl[1]);
-                const uint32_t b2 = __ballot_sync(0xffffffffu, fl[2]);
-                const uint32_t b3 = __ballot_sync(0xffffffffu, fl[3]);
-                if (lane == 0) {
-                    reinterpret_cast<uint4*>(P.bitmap)[(size_t)r * P.ngroups + g] = make_uint4(b0, b1, b2, b3);
-                    const uint32_t cnt = __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
-                    if (cnt) atomicAdd(&P.blk_count[(size_t)r * P.nblk + g / EMIT_GROUPS], cnt);
+                    store_quad<ALIGNED>(P.xw + row, e0, P.d, xq[k]);
+                    if (ANCH) store_quad<ALIGNED>(P.anchors + row, e0, P.d, xq[k]);
                 }
             }
+            tile_counts(sh_cnt[item & 1], warp, lane, bal);
+            __syncthreads();
+            tile_write(P, r, tile, sh_cnt[item & 1], warp, lane, bal, u);
         }
     }
     if (bad) set_status(P, QS_NONFINITE);
@@ -199,7 +174,8 @@ static void pass_a_dispatch(const Plan& P, const Active& act, int mode, int grid
 }
 
 void launch_pass_a(const Plan& P, const Active& act, int mode, bool aligned, int sms, cudaStream_t st) {
-    const int grid = dense_grid(P, sms, 2);
+    const uint32_t cap = (uint32_t)sms * 4u;
+    const int grid = (int)(P.ntile < cap ? P.ntile : cap);
     const size_t words = (size_t)P.R * P.nseg + P.nseg + 1;
     const int tab = words <= (size_t)TAB_MAX;
     const size_t smem = tab ? words * 4 : 0;

@@ -4,8 +4,8 @@
 // tile, the active workers in turn.  One thread keeps a ring of (xw, mem) tile pairs filling
 // with cp.async.bulk loads several items ahead; each arrival is announced on an mbarrier.  The
 // eight warps read their quads from shared memory, form u = mem + (x - xw), overwrite the mem
-// tile in place, vote the candidate flags into the bitmap, and the finished tile goes back to
-// global memory as one bulk store.  Loads and stores never pass through registers of the
+// tile in place, vote the candidate flags, and the finished tile goes back to global memory as
+// one bulk store while the tile's few candidates (index, value) are written out in order.  Loads and stores never pass through registers of the
 // computing warps, so the depth of the ring, not the occupancy, sets the bytes in flight.
 //
 // Every wait is bounded: a barrier that does not complete records QS_TIMEOUT, the block waits
@@ -14,17 +14,14 @@
 
 namespace qs {
 
-#ifndef QS_TMA_GP
-#define QS_TMA_GP 2
-#endif
 #ifndef QS_TMA_STAGES
 #define QS_TMA_STAGES 3
 #endif
 #ifndef QS_TMA_PER_SM
 #define QS_TMA_PER_SM 3
 #endif
-constexpr int GP = QS_TMA_GP;              // groups of 128 coordinates per warp and tile
-constexpr int TILE = 1024 * GP;            // coordinates per tile: 8 warps x GP groups
+constexpr int GP = GPW;                    // groups of 128 coordinates per warp and tile
+constexpr int TILE = STILE;                // coordinates per tile: 8 warps x GP groups
 constexpr int STAGES = QS_TMA_STAGES;      // (xw, mem) tile pairs in the ring
 #ifndef QS_TMA_XSLOTS
 #define QS_TMA_XSLOTS 2
@@ -87,6 +84,7 @@ struct TmaSmem {
     float xs[XSLOTS][TILE];
     uint64_t full[STAGES];
     uint64_t xfull[XSLOTS];
+    uint32_t cnt[2][8 * GPW];              // candidates per group of the current tile (double-buffered)
     int abort_flag;
 };
 
@@ -155,6 +153,8 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
         if (!ok) S.abort_flag = 1;           // seen by everyone at the barrier below
 
         const uint32_t* gs = tab + (size_t)r * P.nseg;
+        uint32_t bal[GPW][4];
+        float uu[GPW][4];
 #pragma unroll
         for (int k = 0; k < GP; ++k) {
             const uint32_t g = tile * (TILE / GROUP) + warp * GP + k;
@@ -171,33 +171,27 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
             const float4 xq = *reinterpret_cast<const float4*>(&S.xs[xsl][q]);
             const float4 wq = *reinterpret_cast<const float4*>(&S.stage[s][0][q]);
             const float4 mq = *reinterpret_cast<const float4*>(&S.stage[s][1][q]);
-            float4 u;
-            u.x = mq.x + (xq.x - wq.x);
-            u.y = mq.y + (xq.y - wq.y);
-            u.z = mq.z + (xq.z - wq.z);
-            u.w = mq.w + (xq.w - wq.w);
-            *reinterpret_cast<float4*>(&S.stage[s][1][q]) = u;
+            uu[k][0] = mq.x + (xq.x - wq.x);
+            uu[k][1] = mq.y + (xq.y - wq.y);
+            uu[k][2] = mq.z + (xq.z - wq.z);
+            uu[k][3] = mq.w + (xq.w - wq.w);
+            *reinterpret_cast<float4*>(&S.stage[s][1][q]) = make_float4(uu[k][0], uu[k][1], uu[k][2], uu[k][3]);
             const bool in = e0 < P.d;                            // d is a multiple of 4: whole quads
-            const uint32_t key[4] = {topk_key(u.x), topk_key(u.y), topk_key(u.z), topk_key(u.w)};
-            uint32_t sk[4] = {key[0], key[1], key[2], key[3]};
+            uint32_t sk[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                sk[jj] = topk_key(uu[k][jj]);
+                if (in) bad |= sk[jj] >= 0xFF000000u;
+            }
             if (RANDK) {
                 const uint4 h = philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
                 sk[0] = ~h.x; sk[1] = ~h.y; sk[2] = ~h.z; sk[3] = ~h.w;
             }
-            uint32_t fl[4];
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj) fl[jj] = in && sk[jj] >= gs[sg[k][jj]];
-            if (in) bad |= (key[0] >= 0xFF000000u) | (key[1] >= 0xFF000000u) | (key[2] >= 0xFF000000u) | (key[3] >= 0xFF000000u);
-            const uint32_t b0 = __ballot_sync(0xffffffffu, fl[0]);
-            const uint32_t b1 = __ballot_sync(0xffffffffu, fl[1]);
-            const uint32_t b2 = __ballot_sync(0xffffffffu, fl[2]);
-            const uint32_t b3 = __ballot_sync(0xffffffffu, fl[3]);
-            if (lane == 0 && g < P.ngroups) {
-                reinterpret_cast<uint4*>(P.bitmap)[(size_t)r * P.ngroups + g] = make_uint4(b0, b1, b2, b3);
-                const uint32_t cnt = __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
-                if (cnt) atomicAdd(&P.blk_count[(size_t)r * P.nblk + g / EMIT_GROUPS], cnt);
-            }
+            for (int jj = 0; jj < 4; ++jj)
+                bal[k][jj] = __ballot_sync(0xffffffffu, in && sk[jj] >= gs[sg[k][jj]]);
         }
+        tile_counts(S.cnt[j & 1], warp, lane, bal);
         fence_async_smem();                  // the tile written above must be visible to the bulk store
         __syncthreads();
         if (S.abort_flag) break;
@@ -207,6 +201,7 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
             bulk_store(P.mem + (size_t)r * P.d + t0, S.stage[s][1], bytes);
             bulk_commit();
         }
+        tile_write(P, r, tile, S.cnt[j & 1], warp, lane, bal, uu);
     }
     if (threadIdx.x == 0) {
         if (S.abort_flag) {

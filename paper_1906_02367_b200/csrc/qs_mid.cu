@@ -5,10 +5,11 @@
 // gaps and cold starts than in work, so they run here as stages of one cooperative launch
 // (every block resident), separated by grid-wide barriers with a bounded wait:
 //
-//   candidates  scan of the per-block candidate counts left by the dense pass, candidate
-//               range of every (worker, segment) unit, the exact fallback for workers whose
-//               predicted threshold left a unit short (histogram of the top key bits, new
-//               threshold, bitmap rebuilt from the stored u), ordered emission (index, value)
+//   candidates  the per-tile candidate runs left by the dense pass are gathered into each worker's
+//               ordered list (index, value) with the first select histogram and the segment
+//               boundaries; the exact fallback for workers whose predicted threshold left a unit
+//               short (histogram of the top key bits, new threshold, candidates found again from
+//               the stored u)
 //   select      radix select over the 32-bit sort key (4 levels of 8 bits), tie cut by lower
 //               index, next round's prediction
 //   quantize    exact norm of the kept values, levels and signs (Philox stream 0), m <- u - g,
@@ -71,89 +72,147 @@ __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, in
     return *sh_abort == 0;
 }
 
-__device__ __forceinline__ uint32_t popc4(const uint4 w) {
-    return __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
-}
-
 template <bool RANDK>
 __device__ __forceinline__ uint32_t sort_key(const Plan& P, size_t pos) {
     return RANDK ? P.cand_key[pos] : topk_key(P.cand_val[pos]);
 }
 
+// Unit table: where each (worker, segment) unit's candidates start, how many there are, and the
+// number of chunks before it.  Every block builds it for itself in shared memory.
+struct Tab {
+    const uint32_t* start;
+    const uint32_t* c;
+    const uint32_t* cb;      // U + 1 entries
+    uint32_t total_chunks;
+};
+
+__device__ __forceinline__ uint32_t segment_of(const Plan& P, uint32_t e) {
+    if (P.nseg == 1) return 0;
+    uint32_t sq = P.grp_seg[e >> 7];
+    while (sq + 1 < (uint32_t)P.nseg && e >= P.seg_off[sq + 1]) ++sq;
+    return sq;
+}
+
 // ------------------------------------------------------------------ candidates
-// exclusive prefix of the per-block candidate counts of each worker; clears the counts
-__device__ void stage_scan(const Plan& P, const Active& act, bool only_failed, uint32_t* sh) {
-    for (int w = blockIdx.x; w < act.n; w += gridDim.x) {
-        const int r = act.r[w];
-        if (only_failed && !P.fail[r]) continue;
-        uint32_t carry = 0;
-        for (uint32_t base = 0; base < P.nblk; base += BT) {
-            const uint32_t i = base + threadIdx.x;
-            uint32_t v = 0;
-            if (i < P.nblk) {
-                v = P.blk_count[(size_t)r * P.nblk + i];
-                P.blk_count[(size_t)r * P.nblk + i] = 0;
-            }
-            uint32_t total;
-            const uint32_t ex = block_excl_scan(v, sh, &total);
-            if (i < P.nblk) P.blk_base[(size_t)r * P.nblk + i] = carry + ex;
-            carry += total;
-        }
-        if (threadIdx.x == 0) P.ncand[r] = carry;
-    }
-}
-
-// candidates of worker r among coordinates below p (warp-cooperative, every lane gets it)
-__device__ uint32_t cand_prefix(const Plan& P, int r, uint32_t p, int lane) {
-    if (p >= P.d) return P.ncand[r];
-    const uint32_t g = p >> 7, blk = g / EMIT_GROUPS;
-    const uint4* bm = reinterpret_cast<const uint4*>(P.bitmap) + (size_t)r * P.ngroups;
-    uint32_t c = 0;
-    for (uint32_t gg = blk * EMIT_GROUPS + lane; gg < g; gg += 32) c += popc4(bm[gg]);
-    if (lane == 0) {
-        const uint4 w = bm[g];
-        const uint32_t pl = p & 127u;
-        const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (uint32_t j = 0; j < 4; ++j) {
-            const uint32_t nl = pl > j ? (pl - j + 3u) >> 2 : 0u;      // lanes l with 4 l + j < pl
-            const uint32_t mask = nl >= 32u ? 0xffffffffu : ((1u << nl) - 1u);
-            c += __popc(ws[j] & mask);
-        }
-        c += P.blk_base[(size_t)r * P.nblk + blk];
-    }
-    return warp_sum(c);
-}
-
-// one warp per unit: its candidate range; a unit with fewer candidates than k marks its worker
-__device__ void stage_bounds(const Plan& P, const Active& act, bool only_failed) {
+// One candidate block (BLK_TILES tiles of one worker): its candidates are copied from the tiles'
+// fixed places into the worker's ordered list, their top key digit is counted for the select,
+// and the list positions of the segment boundaries inside the block are recorded.
+template <bool RANDK>
+__device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask, uint32_t* sh, uint32_t* sh_tp) {
     const int lane = threadIdx.x & 31;
-    const uint32_t nunits = (uint32_t)act.n * P.nseg;
-    for (uint32_t wu = blockIdx.x * (BT / 32) + (threadIdx.x >> 5); wu < nunits; wu += gridDim.x * (BT / 32)) {
-        const int r = act.r[wu / P.nseg];
-        const uint32_t seg = wu % P.nseg;
-        if (only_failed && !P.fail[r]) continue;
-        const uint32_t lo = cand_prefix(P, r, P.seg_off[seg], lane);
-        const uint32_t hi = cand_prefix(P, r, P.seg_off[seg + 1], lane);
-        if (lane == 0) {
-            Unit& un = P.units[(size_t)r * P.nseg + seg];
-            un.start = lo;
-            un.c = hi - lo;
-            if (hi - lo < P.kseg[seg]) {
-                if (only_failed) set_status(P, QS_STATE);      // the exact pass cannot miss
-                else atomicExch(&P.fail[r], 1u);
+    const uint32_t items = P.nblk * (uint32_t)act.n;
+    for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
+        const int r = act.r[item / P.nblk];
+        if (only_mask && !((only_mask >> r) & 1u)) continue;
+        const uint32_t blk = item % P.nblk;
+        const uint32_t sup = blk / SUP_BLOCKS;
+        // candidates of this worker in earlier blocks: whole super-blocks, then blocks of this one
+        uint32_t part = 0;
+        for (uint32_t i = threadIdx.x; i < sup; i += BT) part += P.sup_count[(size_t)r * P.nsup + i];
+        for (uint32_t i = sup * SUP_BLOCKS + threadIdx.x; i < blk; i += BT) part += P.blk_count[(size_t)r * P.nblk + i];
+        uint32_t base;
+        block_excl_scan(part, sh, &base);
+        const uint32_t n = P.blk_count[(size_t)r * P.nblk + blk];
+        const uint32_t t0 = blk * BLK_TILES;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t run = 0;
+            for (int t = 0; t < BLK_TILES; ++t) {
+                sh_tp[t] = run;
+                run += (t0 + t < P.ntile) ? P.tile_cnt[(size_t)r * P.ntile + t0 + t] : 0u;
+            }
+            sh_tp[BLK_TILES] = run;
+        }
+        __syncthreads();
+        const size_t row = (size_t)r * P.cap;
+        for (uint32_t eb = 0; eb < n; eb += BT) {
+            const uint32_t e = eb + threadIdx.x;
+            const bool valid = e < n;
+            uint32_t idx = 0, sk = 0, seg = 0;
+            if (valid) {
+                int t = 0;
+                while (t + 1 < BLK_TILES && sh_tp[t + 1] <= e) ++t;
+                const size_t src = row + (size_t)(t0 + t) * STILE + (e - sh_tp[t]);
+                idx = P.stage_idx[src];
+                const float val = P.stage_val[src];
+                sk = RANDK ? ~philox_word(P, (uint32_t)r, idx, 1u) : topk_key(val);
+                P.cand_idx[row + base + e] = idx;
+                P.cand_val[row + base + e] = val;
+                if (RANDK) P.cand_key[row + base + e] = sk;
+                seg = segment_of(P, idx);
+            }
+            // level 0 of the radix select: count the top key byte per unit
+            const uint32_t tag = (seg << 8) | (sk >> 24);
+            const uint32_t live = __ballot_sync(0xffffffffu, valid);
+            if (valid) {
+                const uint32_t peers = __match_any_sync(live, tag);
+                if (lane == __ffs(peers) - 1)
+                    atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
             }
         }
+        __syncthreads();                          // the block's part of the ordered list is written
+        // segment boundaries inside this block: position of the first candidate at or after each
+        const uint32_t lo = blk * (uint32_t)(BLK_TILES * STILE);
+        const uint64_t hi64 = (uint64_t)lo + BLK_TILES * STILE;
+        const uint32_t hi = hi64 < P.d ? (uint32_t)hi64 : P.d;
+        uint32_t s_lo = 0;
+        if (P.nseg > 1) {
+            const uint32_t sc = P.grp_seg[lo >> 7];
+            s_lo = P.seg_off[sc] == lo ? sc : sc + 1;
+        } else if (blk != 0) {
+            s_lo = 1;
+        }
+        uint32_t* ss = P.seg_start + (size_t)r * (P.nseg + 1);
+        for (uint32_t sgm = s_lo + threadIdx.x; sgm < (uint32_t)P.nseg && P.seg_off[sgm] < hi; sgm += BT) {
+            const uint32_t bound = P.seg_off[sgm];
+            uint32_t a = 0, b = n;               // first entry of the block with index >= bound
+            while (a < b) {
+                const uint32_t m = (a + b) >> 1;
+                if (P.cand_idx[row + base + m] < bound) a = m + 1; else b = m;
+            }
+            ss[sgm] = base + a;
+        }
+        if (blk == P.nblk - 1 && threadIdx.x == 0) ss[P.nseg] = base + n;
     }
+}
+
+// Builds the unit table; returns the workers (bit mask) that have a unit with fewer candidates
+// than k.  Every block computes the same thing from the same data.
+__device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_start, uint32_t* t_c, uint32_t* t_cb,
+                                uint32_t* sh, uint32_t* sh_flag, Tab* tab) {
+    if (threadIdx.x == 0) *sh_flag = 0;
+    __syncthreads();
+    uint32_t carry = 0;
+    for (uint32_t ub = 0; ub < P.U; ub += BT) {
+        const uint32_t u = ub + threadIdx.x;
+        uint32_t start = 0, c = 0;
+        if (u < P.U) {
+            const uint32_t r = u / P.nseg, seg = u % P.nseg;
+            if ((act.bits >> r) & 1u) {
+                const uint32_t* ss = P.seg_start + (size_t)r * (P.nseg + 1);
+                start = ss[seg];
+                c = ss[seg + 1] - start;
+                if (c < P.kseg[seg]) atomicOr(sh_flag, 1u << r);
+            }
+        }
+        uint32_t total;
+        const uint32_t ex = block_excl_scan((c + CHUNK - 1) / CHUNK, sh, &total);
+        if (u < P.U) { t_start[u] = start; t_c[u] = c; t_cb[u] = carry + ex; }
+        carry += total;
+    }
+    if (threadIdx.x == 0) t_cb[P.U] = carry;
+    __syncthreads();
+    tab->start = t_start; tab->c = t_c; tab->cb = t_cb; tab->total_chunks = carry;
+    return *sh_flag;
 }
 
 // histogram of the top 11 key bits of one stretch of one segment, for missed workers
 template <bool RANDK>
-__device__ void stage_fb_hist(const Plan& P, const Active& act, uint32_t* sh_bins) {
+__device__ void stage_fb_hist(const Plan& P, const Active& act, uint32_t missed, uint32_t* sh_bins) {
     const uint32_t items = P.nfb * (uint32_t)act.n;
     for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
         const int r = act.r[item / P.nfb];
-        if (!P.fail[r]) continue;
+        if (!((missed >> r) & 1u)) continue;
         const FbBlock blk = P.fb_tab[item % P.nfb];
         for (int i = threadIdx.x; i < FB_BINS; i += BT) sh_bins[i] = 0;
         __syncthreads();
@@ -178,28 +237,30 @@ __device__ void stage_fb_hist(const Plan& P, const Active& act, uint32_t* sh_bin
     }
 }
 
-// new threshold of each segment of a missed worker: the lowest bin edge that still leaves
-// `target` coordinates at or above it; clears the histogram
-__device__ void stage_fb_guess(const Plan& P, const Active& act, uint32_t* sh, uint32_t* sh_best) {
+// New threshold of each segment of a missed worker: the lowest bin edge that still leaves
+// `target` coordinates at or above it.  Clears the histogram, the worker's candidate counts and
+// the select histogram its first attempt filled.
+__device__ void stage_fb_guess(const Plan& P, const Active& act, uint32_t missed, uint32_t* sh, uint32_t* sh_best) {
     const uint32_t items = (uint32_t)P.nseg * act.n;
     for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
         const int r = act.r[item / P.nseg];
-        if (!P.fail[r]) continue;
+        if (!((missed >> r) & 1u)) continue;
         const uint32_t seg = item % P.nseg;
         uint32_t* hist = P.fb_hist + ((size_t)r * P.nseg + seg) * FB_BINS;
-        uint32_t v[8], s = 0;                    // thread t owns bins 2047 - 8t .. 2040 - 8t
+        uint32_t v[8], sum = 0;                  // thread t owns bins 2047 - 8t .. 2040 - 8t
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int bin = FB_BINS - 1 - 8 * (int)threadIdx.x - i;
             v[i] = hist[bin];
             hist[bin] = 0;
-            s += v[i];
+            sum += v[i];
         }
+        P.hist[((size_t)r * P.nseg + seg) * 256 + threadIdx.x] = 0;
         if (threadIdx.x == 0) *sh_best = 0;
         uint32_t total;
-        const uint32_t excl = block_excl_scan(s, sh, &total);
+        const uint32_t excl = block_excl_scan(sum, sh, &total);
         const uint32_t target = P.target[seg];
-        if (excl < target && excl + s >= target) {
+        if (excl < target && excl + sum >= target) {
             uint32_t run = excl;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -211,132 +272,56 @@ __device__ void stage_fb_guess(const Plan& P, const Active& act, uint32_t* sh, u
         if (threadIdx.x == 0) P.guess[(size_t)r * P.nseg + seg] = *sh_best << FB_SHIFT;
         __syncthreads();
     }
-}
-
-// segment of each coordinate of a quad
-__device__ __forceinline__ void quad_segments(const Plan& P, uint32_t g, uint32_t e0, int sg[4]) {
-    if (P.nseg == 1) { sg[0] = sg[1] = sg[2] = sg[3] = 0; return; }
-    int sq = (int)P.grp_seg[g];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        while (sq + 1 < P.nseg && e0 + j >= P.seg_off[sq + 1]) ++sq;
-        sg[j] = sq;
-    }
-}
-
-// bitmap and block counts of the missed workers rebuilt from the stored u
-template <bool RANDK>
-__device__ void stage_reflag(const Plan& P, const Active& act) {
-    const int lane = threadIdx.x & 31;
     for (int w = 0; w < act.n; ++w) {
         const int r = act.r[w];
-        if (!P.fail[r]) continue;
+        if (!((missed >> r) & 1u)) continue;
+        for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < P.nblk; i += gridDim.x * BT) P.blk_count[(size_t)r * P.nblk + i] = 0;
+        for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < P.nsup; i += gridDim.x * BT) P.sup_count[(size_t)r * P.nsup + i] = 0;
+    }
+}
+
+// candidates of the missed workers found again from the stored u with the new thresholds
+template <bool RANDK>
+__device__ void stage_reflag(const Plan& P, const Active& act, uint32_t missed, uint32_t* sh_cnt) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t item = 0;
+    for (int w = 0; w < act.n; ++w) {
+        const int r = act.r[w];
+        if (!((missed >> r) & 1u)) continue;
         const size_t row = (size_t)r * P.d;
         const uint32_t* gs = P.guess + (size_t)r * P.nseg;
-        for (uint32_t g = blockIdx.x * (BT / 32) + (threadIdx.x >> 5); g < P.ngroups; g += gridDim.x * (BT / 32)) {
-            const uint32_t e0 = g * (uint32_t)GROUP + (uint32_t)lane * 4u;
-            int sg[4];
-            quad_segments(P, g, e0, sg);
-            uint4 h = make_uint4(0, 0, 0, 0);
-            if (RANDK) h = philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
-            const uint32_t hh[4] = {h.x, h.y, h.z, h.w};
-            uint32_t fl[4];
+        for (uint32_t tile = blockIdx.x; tile < P.ntile; tile += gridDim.x, ++item) {
+            uint32_t bal[GPW][4];
+            float u[GPW][4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                fl[j] = 0;
-                if (e0 + j < P.d) {
-                    const uint32_t sk = RANDK ? ~hh[j] : topk_key(P.mem[row + e0 + j]);
-                    fl[j] = sk >= gs[sg[j]];
+            for (int k = 0; k < GPW; ++k) {
+                const uint32_t e0 = (tile * (uint32_t)(STILE / GROUP) + warp * GPW + k) * (uint32_t)GROUP + (uint32_t)lane * 4u;
+                uint4 h = make_uint4(0, 0, 0, 0);
+                if (RANDK) h = philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
+                const uint32_t hh[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool in = e0 + j < P.d;
+                    u[k][j] = in ? P.mem[row + e0 + j] : 0.0f;
+                    const uint32_t sk = RANDK ? ~hh[j] : topk_key(u[k][j]);
+                    bal[k][j] = __ballot_sync(0xffffffffu, in && sk >= gs[segment_of(P, in ? e0 + j : 0u)]);
                 }
             }
-            const uint32_t b0 = __ballot_sync(0xffffffffu, fl[0]);
-            const uint32_t b1 = __ballot_sync(0xffffffffu, fl[1]);
-            const uint32_t b2 = __ballot_sync(0xffffffffu, fl[2]);
-            const uint32_t b3 = __ballot_sync(0xffffffffu, fl[3]);
-            if (lane == 0) {
-                reinterpret_cast<uint4*>(P.bitmap)[(size_t)r * P.ngroups + g] = make_uint4(b0, b1, b2, b3);
-                const uint32_t cnt = __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
-                if (cnt) atomicAdd(&P.blk_count[(size_t)r * P.nblk + g / EMIT_GROUPS], cnt);
-            }
+            uint32_t* cnt = sh_cnt + (item & 1u) * (8 * GPW);
+            tile_counts(cnt, warp, lane, bal);
+            __syncthreads();
+            tile_write(P, r, tile, cnt, warp, lane, bal, u);
         }
-    }
-}
-
-// candidates of one emission block, in ascending coordinate order
-template <bool RANDK>
-__device__ void stage_emit(const Plan& P, const Active& act, uint32_t* sh) {
-    const uint32_t items = P.nblk * (uint32_t)act.n;
-    for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
-        const int r = act.r[item / P.nblk];
-        const uint32_t blk = item % P.nblk;
-        const uint32_t g = blk * (uint32_t)EMIT_GROUPS + threadIdx.x;
-        uint4 w = make_uint4(0, 0, 0, 0);
-        if (g < P.ngroups) w = reinterpret_cast<const uint4*>(P.bitmap)[(size_t)r * P.ngroups + g];
-        uint32_t total;
-        const uint32_t ex = block_excl_scan(popc4(w), sh, &total);
-        if (total == 0) continue;
-        size_t pos = (size_t)r * P.cap + P.blk_base[(size_t)r * P.nblk + blk] + ex;
-        const float* mem = P.mem + (size_t)r * P.d;
-        while (w.x | w.y | w.z | w.w) {
-            uint32_t best = 0xffffffffu;               // lowest coordinate 4 l + j still set
-            if (w.x) best = min(best, (uint32_t)(__ffs(w.x) - 1) * 4u + 0u);
-            if (w.y) best = min(best, (uint32_t)(__ffs(w.y) - 1) * 4u + 1u);
-            if (w.z) best = min(best, (uint32_t)(__ffs(w.z) - 1) * 4u + 2u);
-            if (w.w) best = min(best, (uint32_t)(__ffs(w.w) - 1) * 4u + 3u);
-            const uint32_t j = best & 3u;
-            if (j == 0) w.x &= w.x - 1u; else if (j == 1) w.y &= w.y - 1u;
-            else if (j == 2) w.z &= w.z - 1u; else w.w &= w.w - 1u;
-            const uint32_t e = g * (uint32_t)GROUP + best;
-            P.cand_idx[pos] = e;
-            P.cand_val[pos] = mem[e];
-            if (RANDK) P.cand_key[pos] = ~philox_word(P, (uint32_t)r, e, 1u);
-            ++pos;
-        }
-    }
-}
-
-// block 0: chunk numbering over the units of the active workers, in (worker, segment) order
-__device__ void stage_setup(const Plan& P, const Active& act, uint32_t* sh) {
-    if (blockIdx.x != 0) return;
-    uint32_t carry = 0;
-    for (uint32_t base = 0; base < P.U; base += BT) {
-        const uint32_t u = base + threadIdx.x;
-        uint32_t nch = 0, cands = 0;
-        if (u < P.U) {
-            Unit& un = P.units[u];
-            if (!((act.bits >> (u / P.nseg)) & 1u)) un.c = 0;
-            cands = un.c;
-            nch = (cands + CHUNK - 1) / CHUNK;
-        }
-        uint32_t total;
-        const uint32_t ex = block_excl_scan(nch, sh, &total);
-        if (u < P.U) {
-            Unit& un = P.units[u];
-            un.chunk_base = carry + ex;
-            un.nchunks = nch;
-            un.n = 0;
-            un.emin = 255u;
-            un.emax = 0u;
-            un.norm = 0.0f;
-            if (cands) atomicAdd((unsigned long long*)&P.stats[1], (unsigned long long)cands);
-        }
-        carry += total;
-    }
-    if (threadIdx.x == 0) {
-        *P.total_chunks = carry;
-        uint32_t nf = 0;
-        for (int w = 0; w < act.n; ++w) { nf += P.fail[act.r[w]] ? 1u : 0u; P.fail[act.r[w]] = 0; }
-        if (nf) atomicAdd((unsigned long long*)&P.stats[0], (unsigned long long)nf);
     }
 }
 
 // ------------------------------------------------------------------ select
 // unit owning a chunk: the last unit whose first chunk is not after it
-__device__ __forceinline__ uint32_t unit_of_chunk(const Plan& P, uint32_t chunk) {
+__device__ __forceinline__ uint32_t unit_of_chunk(const Plan& P, const Tab& tab, uint32_t chunk) {
     uint32_t lo = 0, hi = P.U;
     while (hi - lo > 1) {
         const uint32_t mid = (lo + hi) >> 1;
-        if (P.units[mid].chunk_base <= chunk) lo = mid; else hi = mid;
+        if (tab.cb[mid] <= chunk) lo = mid; else hi = mid;
     }
     return lo;
 }
@@ -379,36 +364,38 @@ __device__ void derive_prefix(const Plan& P, uint32_t u, uint32_t k, int level, 
     *above_total = at;
 }
 
-struct ChunkCtx { uint32_t u, r, seg, first; Unit un; size_t base; };
+struct ChunkCtx { uint32_t u, r, seg, first, c, cb; Unit un; size_t base; };
 
 // which unit a chunk belongs to (one search per block, shared through sh_u)
-__device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, uint32_t chunk, uint32_t* sh_u) {
+__device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, const Tab& tab, uint32_t chunk, uint32_t* sh_u) {
     __syncthreads();
-    if (threadIdx.x == 0) *sh_u = unit_of_chunk(P, chunk);
+    if (threadIdx.x == 0) *sh_u = unit_of_chunk(P, tab, chunk);
     __syncthreads();
     ChunkCtx c;
     c.u = *sh_u;
     c.un = P.units[c.u];
     c.r = c.u / P.nseg;
     c.seg = c.u % P.nseg;
-    c.first = (chunk - c.un.chunk_base) * CHUNK;
-    c.base = (size_t)c.r * P.cap + c.un.start;
+    c.c = tab.c[c.u];
+    c.cb = tab.cb[c.u];
+    c.first = (chunk - c.cb) * CHUNK;
+    c.base = (size_t)c.r * P.cap + tab.start[c.u];
     return c;
 }
 
 // one level of the radix select: histogram of the level's digit among keys matching the prefix
 template <bool RANDK>
-__device__ void stage_hist(const Plan& P, int level, uint32_t* sh_hist, uint32_t* sh_u, uint32_t* sh_prefix) {
+__device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* sh_hist, uint32_t* sh_u, uint32_t* sh_prefix) {
     const int lane = threadIdx.x & 31;
-    const uint32_t total = *P.total_chunks;
+    const uint32_t total = tab.total_chunks;
     const int shift = 24 - 8 * level;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, chunk, sh_u);
+        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
         uint32_t sk[PER];
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            sk[i] = off < c.un.c ? sort_key<RANDK>(P, c.base + off) : 0u;
+            sk[i] = off < c.c ? sort_key<RANDK>(P, c.base + off) : 0u;
         }
         if (threadIdx.x < 32) {
             uint32_t prefix, at;
@@ -421,7 +408,7 @@ __device__ void stage_hist(const Plan& P, int level, uint32_t* sh_hist, uint32_t
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            const bool valid = off < c.un.c && (level == 0 || (sk[i] >> (32 - 8 * level)) == prefix);
+            const bool valid = off < c.c && (level == 0 || (sk[i] >> (32 - 8 * level)) == prefix);
             const uint32_t digit = (sk[i] >> shift) & 255u;
             const uint32_t live = __ballot_sync(0xffffffffu, valid);
             if (valid) {
@@ -437,11 +424,11 @@ __device__ void stage_hist(const Plan& P, int level, uint32_t* sh_hist, uint32_t
 
 // threshold key, tie cut and next prediction of each unit; clears its histograms
 template <bool RANDK>
-__device__ void stage_final(const Plan& P, uint32_t* sh4, uint32_t* sh_w) {
+__device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     for (uint32_t u = blockIdx.x; u < P.U; u += gridDim.x) {
-        const Unit un = P.units[u];
-        if (un.c == 0) continue;
+        const uint32_t uc = tab.c[u];
+        if (uc == 0) continue;
         const uint32_t seg = u % P.nseg, r = u / P.nseg, k = P.kseg[seg];
         __syncthreads();
         if (wid == 0) {
@@ -461,10 +448,10 @@ __device__ void stage_final(const Plan& P, uint32_t* sh4, uint32_t* sh_w) {
         uint32_t tie_max = 0xffffffffu;
         if (ceq > t) {
             // more equal keys than slots: the t lowest coordinates win; walk the list in order
-            const size_t base = (size_t)r * P.cap + un.start;
-            for (uint32_t first = 0; first < un.c; first += BT) {
+            const size_t base = (size_t)r * P.cap + tab.start[u];
+            for (uint32_t first = 0; first < uc; first += BT) {
                 const uint32_t off = first + threadIdx.x;
-                const bool eq = off < un.c && sort_key<RANDK>(P, base + off) == tau;
+                const bool eq = off < uc && sort_key<RANDK>(P, base + off) == tau;
                 const uint32_t bal = __ballot_sync(0xffffffffu, eq);
                 if (lane == 0) sh_w[wid] = __popc(bal);
                 __syncthreads();
@@ -483,6 +470,10 @@ __device__ void stage_final(const Plan& P, uint32_t* sh4, uint32_t* sh_w) {
             Unit& out = P.units[u];
             out.tau = tau;
             out.tie_max = tie_max;
+            out.n = 0;
+            out.emin = 255u;
+            out.emax = 0u;
+            out.norm = 0.0f;
             if (!RANDK) {
                 // prediction for the next round: move the candidate floor so that about `target`
                 // coordinates pass it, assuming the tail keeps its shape (log-linear in the count)
@@ -490,11 +481,11 @@ __device__ void stage_final(const Plan& P, uint32_t* sh4, uint32_t* sh_w) {
                 const float tk = __uint_as_float(tau >> 1), tg = __uint_as_float(*gp >> 1);
                 const float target = (float)P.target[seg];
                 float tn = tg;
-                if (un.c > k && tk > tg) {
-                    float ratio = __logf(target / (float)k) / __logf((float)un.c / (float)k);
+                if (uc > k && tk > tg) {
+                    float ratio = __logf(target / (float)k) / __logf((float)uc / (float)k);
                     ratio = fminf(fmaxf(ratio, 0.25f), 4.0f);
                     tn = tk - (tk - tg) * ratio;
-                } else if (un.c <= k) {
+                } else if (uc <= k) {
                     tn = tk * 0.75f;
                 }
                 tn = fminf(fmaxf(tn, tk * 0.25f), tk);
@@ -514,18 +505,18 @@ __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t id
 // products are summed as two 24-bit halves (QSGD), or the 24-bit mantissas themselves (Sign).
 // A 64-bit sum cannot overflow below 2^32 terms.
 template <bool RANDK>
-__device__ void stage_norm_accum(const Plan& P, unsigned long long (*acc)[2], uint32_t* sh_u) {
+__device__ void stage_norm_accum(const Plan& P, const Tab& tab, unsigned long long (*acc)[2], uint32_t* sh_u) {
     const int lane = threadIdx.x & 31;
-    const uint32_t total = *P.total_chunks;
+    const uint32_t total = tab.total_chunks;
     const bool l1 = P.qz == QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, chunk, sh_u);
+        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
         float val[PER];
         uint32_t idx[PER], key[PER];
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            const bool in = off < c.un.c;
+            const bool in = off < c.c;
             val[i] = in ? P.cand_val[c.base + off] : 0.0f;
             idx[i] = in ? P.cand_idx[c.base + off] : 0xffffffffu;
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
@@ -536,7 +527,7 @@ __device__ void stage_norm_accum(const Plan& P, unsigned long long (*acc)[2], ui
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            const bool kept = off < c.un.c && is_kept<RANDK>(c.un, key[i], idx[i]);
+            const bool kept = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
             const uint32_t live = __ballot_sync(0xffffffffu, kept);
             if (kept) {
                 const uint32_t b = __float_as_uint(val[i]);
@@ -585,10 +576,10 @@ __device__ void big_add(uint32_t* dig, int ndig, unsigned long long v, int bitpo
 }
 
 // one thread per unit: exact sum -> fp64 (round to nearest even) -> norm in fp32
-__device__ void stage_norm_final(const Plan& P) {
+__device__ void stage_norm_final(const Plan& P, const Tab& tab) {
     for (uint32_t u = blockIdx.x * BT + threadIdx.x; u < P.U; u += gridDim.x * BT) {
         Unit& un = P.units[u];
-        if (un.c == 0 || un.emin > un.emax) continue;
+        if (tab.c[u] == 0 || un.emin > un.emax) continue;
         constexpr int ND = 24;                      // 768 bits
         uint32_t dig[ND];
         for (int j = 0; j < ND; ++j) dig[j] = 0;
@@ -628,12 +619,12 @@ __device__ void stage_norm_final(const Plan& P) {
 
 // levels, signs, memory update; kept and sent counts per chunk
 template <bool RANDK>
-__device__ void stage_quant(const Plan& P, uint32_t* sh_u, uint32_t* sh_w) {
+__device__ void stage_quant(const Plan& P, const Tab& tab, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const uint32_t total = *P.total_chunks;
+    const uint32_t total = tab.total_chunks;
     const bool sign_op = P.qz == QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, chunk, sh_u);
+        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
         const float N = c.un.norm, cs = P.cscale[c.seg];
         const uint32_t k = P.kseg[c.seg];
         float* mem = P.mem + (size_t)c.r * P.d;
@@ -642,7 +633,7 @@ __device__ void stage_quant(const Plan& P, uint32_t* sh_u, uint32_t* sh_w) {
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            const bool in = off < c.un.c;
+            const bool in = off < c.c;
             val[i] = in ? P.cand_val[c.base + off] : 0.0f;
             idx[i] = in ? P.cand_idx[c.base + off] : 0xffffffffu;
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
@@ -651,7 +642,7 @@ __device__ void stage_quant(const Plan& P, uint32_t* sh_u, uint32_t* sh_w) {
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            if (off >= c.un.c) continue;
+            if (off >= c.c) continue;
             uint32_t q = 0;
             if (is_kept<RANDK>(c.un, key[i], idx[i])) {
                 const bool neg = val[i] < 0.0f;
@@ -679,9 +670,9 @@ __device__ void stage_quant(const Plan& P, uint32_t* sh_u, uint32_t* sh_w) {
 
 // block 0: exclusive sums of kept / sent over the chunks, entries per unit, stream offsets,
 // bit counts; writes the directory when a wire is given
-__device__ void stage_chunk_scan(const Plan& P, const Active& act, uint32_t* sh) {
+__device__ void stage_chunk_scan(const Plan& P, const Tab& tab, const Active& act, uint32_t* sh) {
     if (blockIdx.x != 0) return;
-    const uint32_t total = *P.total_chunks;
+    const uint32_t total = tab.total_chunks;
     uint32_t carry_k = 0, carry_s = 0;
     for (uint32_t base = 0; base <= total; base += BT) {
         const uint32_t i = base + threadIdx.x;
@@ -696,8 +687,9 @@ __device__ void stage_chunk_scan(const Plan& P, const Active& act, uint32_t* sh)
     for (uint32_t u = threadIdx.x; u < P.U; u += BT) {
         Unit& un = P.units[u];
         if (!((act.bits >> (u / P.nseg)) & 1u)) continue;
-        const uint32_t kept = P.chunk_sel[un.chunk_base + un.nchunks] - P.chunk_sel[un.chunk_base];
-        un.n = P.chunk_nz[un.chunk_base + un.nchunks] - P.chunk_nz[un.chunk_base];
+        const uint32_t c0 = tab.cb[u], c1 = tab.cb[u + 1];
+        const uint32_t kept = P.chunk_sel[c1] - P.chunk_sel[c0];
+        un.n = P.chunk_nz[c1] - P.chunk_nz[c0];
         if (kept != P.kseg[u % P.nseg]) set_status(P, QS_STATE);
     }
     __syncthreads();
@@ -747,13 +739,13 @@ __device__ void stage_pack_dir(const Plan& P, const Active& act, uint32_t* wire,
 }
 
 // streams of every segment, and the ordered kept list kept for inspection
-__device__ void stage_pack(const Plan& P, uint32_t* wire, long long stride, uint32_t* sh_u, uint32_t* sh) {
-    const uint32_t total = *P.total_chunks;
+__device__ void stage_pack(const Plan& P, const Tab& tab, uint32_t* wire, long long stride, uint32_t* sh_u, uint32_t* sh) {
+    const uint32_t total = tab.total_chunks;
     const bool has_lvl = P.qz != QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, chunk, sh_u);
-        uint32_t run_k = P.chunk_sel[chunk] - P.chunk_sel[c.un.chunk_base];
-        uint32_t run_s = P.chunk_nz[chunk] - P.chunk_nz[c.un.chunk_base];
+        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+        uint32_t run_k = P.chunk_sel[chunk] - P.chunk_sel[c.cb];
+        uint32_t run_s = P.chunk_nz[chunk] - P.chunk_nz[c.cb];
         const uint32_t bi = P.bidx[c.seg], lo = P.seg_off[c.seg];
         uint32_t* w_idx = wire + (size_t)c.r * stride + P.pay_off[c.u];
         uint32_t* w_sgn = w_idx + words_for(c.un.n, bi);
@@ -764,8 +756,8 @@ __device__ void stage_pack(const Plan& P, uint32_t* wire, long long stride, uint
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            q[i] = off < c.un.c ? P.cand_q[c.base + off] : 0u;
-            e[i] = off < c.un.c ? P.cand_idx[c.base + off] : 0u;
+            q[i] = off < c.c ? P.cand_q[c.base + off] : 0u;
+            e[i] = off < c.c ? P.cand_idx[c.base + off] : 0u;
         }
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
@@ -932,7 +924,11 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_scan[33];
     __shared__ uint32_t sh_small[8];              // unit id, prefix, select scratch
     __shared__ uint32_t sh_w[BT / 32];
+    __shared__ uint32_t sh_tp[BLK_TILES + 1];
+    __shared__ uint32_t sh_cnt[2 * 8 * GPW];
+    __shared__ uint32_t sh_flag;
     __shared__ int sh_abort;
+    __shared__ uint32_t t_start[UT_MAX], t_c[UT_MAX], t_cb[UT_MAX + 1];
     __shared__ __align__(16) unsigned char sh_big[FB_BINS * 4];   // fallback bins / radix bins / exponent sums
     const Plan& P = a.P;
     const Active& act = a.act;
@@ -947,47 +943,51 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     }
 #define QS_BARRIER() do { if (!grid_barrier(P, target, &sh_abort)) return; } while (0)
 
+    Tab tab;
     if (a.do_compress) {
-        stage_scan(P, act, false, sh_scan);
+        stage_order<RANDK>(P, act, 0u, sh_scan, sh_tp);
         QS_BARRIER();
-        stage_bounds(P, act, false);
-        QS_BARRIER();
-        int missed = 0;
-        for (int w = 0; w < act.n; ++w) missed |= (int)P.fail[act.r[w]];
-        if (missed) {                              // same value in every block
-            QS_BARRIER();                          // nobody may clear a flag before all have read it
-            stage_fb_hist<RANDK>(P, act, bins);
+        const uint32_t missed = build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
+        if (missed) {                              // the same value in every block
+            stage_fb_hist<RANDK>(P, act, missed, bins);
             QS_BARRIER();
-            stage_fb_guess(P, act, sh_scan, &sh_small[0]);
+            stage_fb_guess(P, act, missed, sh_scan, &sh_small[0]);
             QS_BARRIER();
-            stage_reflag<RANDK>(P, act);
+            stage_reflag<RANDK>(P, act, missed, sh_cnt);
             QS_BARRIER();
-            stage_scan(P, act, true, sh_scan);
+            stage_order<RANDK>(P, act, missed, sh_scan, sh_tp);
             QS_BARRIER();
-            stage_bounds(P, act, true);
+            if (build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab)) set_status(P, QS_STATE);   // the exact pass cannot miss
+            if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd((unsigned long long*)&P.stats[0], (unsigned long long)__popc(missed));
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            unsigned long long cands = 0;
+            for (int w = 0; w < act.n; ++w) cands += P.seg_start[(size_t)act.r[w] * (P.nseg + 1) + P.nseg];
+            atomicAdd((unsigned long long*)&P.stats[1], cands);
+        }
+        // the candidate counts have been consumed: clear them for the next dense pass
+        for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nblk; i += gridDim.x * BT) P.blk_count[i] = 0;
+        for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nsup; i += gridDim.x * BT) P.sup_count[i] = 0;
+        for (int level = 1; level < 4; ++level) {
+            stage_hist<RANDK>(P, tab, level, bins, &sh_small[0], &sh_small[1]);
             QS_BARRIER();
         }
-        stage_emit<RANDK>(P, act, sh_scan);
-        stage_setup(P, act, sh_scan);
+        stage_final<RANDK>(P, tab, &sh_small[2], sh_w);
         QS_BARRIER();
-        for (int level = 0; level < 4; ++level) {
-            stage_hist<RANDK>(P, level, bins, &sh_small[0], &sh_small[1]);
-            QS_BARRIER();
-        }
-        stage_final<RANDK>(P, &sh_small[2], sh_w);
+        stage_norm_accum<RANDK>(P, tab, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0]);
         QS_BARRIER();
-        stage_norm_accum<RANDK>(P, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0]);
+        stage_norm_final(P, tab);
         QS_BARRIER();
-        stage_norm_final(P);
+        stage_quant<RANDK>(P, tab, &sh_small[0], sh_w);
         QS_BARRIER();
-        stage_quant<RANDK>(P, &sh_small[0], sh_w);
+        stage_chunk_scan(P, tab, act, sh_scan);
         QS_BARRIER();
-        stage_chunk_scan(P, act, sh_scan);
-        QS_BARRIER();
+    } else if (a.do_pack) {
+        build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
     }
     if (a.do_pack) {
         stage_pack_dir(P, act, a.wire, a.stride, a.bits_out);
-        stage_pack(P, a.wire, a.stride, &sh_small[0], sh_scan);
+        stage_pack(P, tab, a.wire, a.stride, &sh_small[0], sh_scan);
         if (a.do_decode) QS_BARRIER();
     }
     if (a.do_decode) {
