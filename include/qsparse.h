@@ -224,7 +224,7 @@ int qs_get_phase_timing(qs_ctx* ctx, double* ms, int n);
 
 /*
  * qs_get_stage_trace — measurement aid: microseconds, from the start of the last persistent
- * kernel of this context, at which its block 0 reached each grid barrier (us[1], us[2], ...,
+ * kernel of this context, at which each of its grid barriers completed (us[1], us[2], ...,
  * -1 = not reached) and left the kernel (us[31]); us[0] = 0.  Synchronises the stream.
  * Writes min(n, 32) values.
  */

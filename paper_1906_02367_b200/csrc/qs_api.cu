@@ -216,8 +216,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     if ((rc = dev_upload(c, &g_up, h_guess)) != QS_OK) return rc;
     P.guess = const_cast<uint32_t*>(g_up);
 #define AL(field, count, zero) if ((rc = dev_alloc(c, &P.field, (size_t)(count), zero)) != QS_OK) return rc
-    AL(stage_idx, (size_t)R * P.cap, false);
-    AL(stage_val, (size_t)R * P.cap, false);
+    AL(stage, (size_t)R * P.cap, false);
     AL(tile_cnt, (size_t)R * P.ntile, true);
     AL(blk_count, (size_t)R * P.nblk, true);
     AL(sup_count, (size_t)R * P.nsup, true);
@@ -353,7 +352,9 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     }
     const int per_sm = mid_blocks_per_sm(sp == QS_RANDK);
     if (per_sm < 1) { delete c; return QS_CUDA; }
-    c->mid_grid = c->sms * (per_sm < 2 ? per_sm : 2);
+    int want = 4;                                  // blocks of the persistent kernel per SM
+    if (const char* e = std::getenv("QSPARSE_MID_PER_SM")) want = std::atoi(e) > 0 ? std::atoi(e) : want;
+    c->mid_grid = c->sms * (per_sm < want ? per_sm : want);
     Plan& P = c->P;
     P.R = R; P.d = (uint32_t)d; P.s = s; P.sp = sp; P.qz = qz;
     P.seed_lo = (uint32_t)seed; P.seed_hi = (uint32_t)(seed >> 32);

@@ -65,8 +65,7 @@ struct Plan {
     float* x; float* xw; float* mem; float* anchors;
     // scratch
     uint32_t* guess;           // R x nseg, sort-key space
-    uint32_t* stage_idx;       // R x cap: candidates as the dense pass left them, tile t at t * STILE
-    float* stage_val;          // R x cap
+    uint2* stage;              // R x cap (index, value bits): candidates as the dense pass left them, tile t at t * STILE
     uint32_t* tile_cnt;        // R x ntile
     uint32_t* blk_count;       // R x nblk, zero between rounds
     uint32_t* sup_count;       // R x nsup, zero between rounds
@@ -124,6 +123,8 @@ __device__ __forceinline__ uint32_t philox_word(const Plan& P, uint32_t worker, 
     return j == 0 ? o.x : j == 1 ? o.y : j == 2 ? o.z : o.w;
 }
 
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v);
+
 // Candidates of one tile, written by the block that just formed u for it (8 warps, warp w owns
 // groups GPW w .. GPW w + GPW - 1).  bal[k][j]: ballot of "coordinate 4 lane + j of group k is a
 // candidate".  Phase 1 publishes the group counts; after a block-wide barrier phase 2 writes the
@@ -138,17 +139,25 @@ __device__ __forceinline__ void tile_counts(uint32_t* sh_cnt, int warp, int lane
 
 __device__ __forceinline__ void tile_write(const Plan& P, int r, uint32_t tile, const uint32_t* sh_cnt, int warp,
                                            int lane, const uint32_t bal[GPW][4], const float u[GPW][4]) {
-    uint32_t base = 0, total = 0;
+    // the last warp owes the tile's total (warp 0 is the one that keeps the copies going); a warp
+    // without candidates has nothing else to do
+    uint32_t mine = 0;
 #pragma unroll
-    for (int i = 0; i < 8 * GPW; ++i) {
-        const uint32_t c = sh_cnt[i];
-        if (i < warp * GPW) base += c;
-        total += c;
+    for (int k = 0; k < GPW; ++k) mine |= bal[k][0] | bal[k][1] | bal[k][2] | bal[k][3];
+    if (warp == 7) {
+        const uint32_t total = warp_sum(lane < 8 * GPW ? sh_cnt[lane] : 0u);
+        if (lane == 0) {
+            P.tile_cnt[(size_t)r * P.ntile + tile] = total;
+            if (total) {
+                const uint32_t blk = tile / BLK_TILES;
+                atomicAdd(&P.blk_count[(size_t)r * P.nblk + blk], total);
+                atomicAdd(&P.sup_count[(size_t)r * P.nsup + blk / SUP_BLOCKS], total);
+            }
+        }
     }
-    if (total == 0) {
-        if (threadIdx.x == 0) P.tile_cnt[(size_t)r * P.ntile + tile] = 0;
-        return;
-    }
+    if (!mine) return;
+    uint32_t base = 0;
+    for (int i = 0; i < warp * GPW; ++i) base += sh_cnt[i];
     const size_t off = (size_t)r * P.cap + (size_t)tile * STILE;
     const uint32_t lt = (1u << lane) - 1u;
 #pragma unroll
@@ -157,17 +166,11 @@ __device__ __forceinline__ void tile_write(const Plan& P, int r, uint32_t tile, 
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             if ((bal[k][j] >> lane) & 1u) {
-                P.stage_idx[off + pos] = tile * (uint32_t)STILE + (uint32_t)((warp * GPW + k) * GROUP + lane * 4 + j);
-                P.stage_val[off + pos] = u[k][j];
+                P.stage[off + pos] = make_uint2(tile * (uint32_t)STILE + (uint32_t)((warp * GPW + k) * GROUP + lane * 4 + j),
+                                                __float_as_uint(u[k][j]));
                 ++pos;
             }
         base += sh_cnt[warp * GPW + k];
-    }
-    if (threadIdx.x == 0) {
-        P.tile_cnt[(size_t)r * P.ntile + tile] = total;
-        const uint32_t blk = tile / BLK_TILES;
-        atomicAdd(&P.blk_count[(size_t)r * P.nblk + blk], total);
-        atomicAdd(&P.sup_count[(size_t)r * P.nsup + blk / SUP_BLOCKS], total);
     }
 }
 

@@ -48,12 +48,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
 __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, int* sh_abort) {
     target += gridDim.x;
     __syncthreads();
-    if (P.trace && blockIdx.x == 0 && threadIdx.x == 0) {     // stage boundaries as block 0 sees them
-        const uint32_t slot = target / gridDim.x;
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        if (slot < TRACE_SLOTS) P.trace[slot] = t;
-    }
     if (threadIdx.x == 0) {
         __threadfence();
         atomicAdd(P.bar, 1u);
@@ -67,6 +61,12 @@ __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, in
             __nanosleep(32);
         }
         __threadfence();
+        if (P.trace && blockIdx.x == 0) {          // time at which every block has finished the stage
+            const uint32_t slot = target / gridDim.x;
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+            if (slot < TRACE_SLOTS - 1) P.trace[slot] = t;
+        }
     }
     __syncthreads();
     return *sh_abort == 0;
@@ -98,59 +98,76 @@ __device__ __forceinline__ uint32_t segment_of(const Plan& P, uint32_t e) {
 // fixed places into the worker's ordered list, their top key digit is counted for the select,
 // and the list positions of the segment boundaries inside the block are recorded.
 template <bool RANDK>
-__device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask, uint32_t* sh, uint32_t* sh_tp) {
+__device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask, uint32_t* sh_bins) {
     const int lane = threadIdx.x & 31;
+    // one segment and few workers: the top-byte counts, which pile up on two or three bins per
+    // worker, are gathered per block in shared memory (8 workers x 256 bins) and flushed once
+    const bool local_bins = P.nseg == 1 && act.n <= 8;
+    if (local_bins) {
+        for (int i = threadIdx.x; i < FB_BINS; i += BT) sh_bins[i] = 0;
+        __syncthreads();
+    }
     const uint32_t items = P.nblk * (uint32_t)act.n;
-    for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
-        const int r = act.r[item / P.nblk];
+    const uint32_t nwarps = gridDim.x * (BT / 32);
+    for (uint32_t item = blockIdx.x * (BT / 32) + (threadIdx.x >> 5); item < items; item += nwarps) {
+        const uint32_t wslot = item / P.nblk;
+        const int r = act.r[wslot];
         if (only_mask && !((only_mask >> r) & 1u)) continue;
         const uint32_t blk = item % P.nblk;
         const uint32_t sup = blk / SUP_BLOCKS;
         // candidates of this worker in earlier blocks: whole super-blocks, then blocks of this one
         uint32_t part = 0;
-        for (uint32_t i = threadIdx.x; i < sup; i += BT) part += P.sup_count[(size_t)r * P.nsup + i];
-        for (uint32_t i = sup * SUP_BLOCKS + threadIdx.x; i < blk; i += BT) part += P.blk_count[(size_t)r * P.nblk + i];
-        uint32_t base;
-        block_excl_scan(part, sh, &base);
-        const uint32_t n = P.blk_count[(size_t)r * P.nblk + blk];
+        for (uint32_t i = lane; i < sup; i += 32) part += P.sup_count[(size_t)r * P.nsup + i];
+        for (uint32_t i = sup * SUP_BLOCKS + lane; i < blk; i += 32) part += P.blk_count[(size_t)r * P.nblk + i];
+        const uint32_t base = warp_sum(part);
         const uint32_t t0 = blk * BLK_TILES;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t run = 0;
-            for (int t = 0; t < BLK_TILES; ++t) {
-                sh_tp[t] = run;
-                run += (t0 + t < P.ntile) ? P.tile_cnt[(size_t)r * P.ntile + t0 + t] : 0u;
-            }
-            sh_tp[BLK_TILES] = run;
-        }
-        __syncthreads();
+        const uint32_t tc = (lane < BLK_TILES && t0 + lane < P.ntile) ? P.tile_cnt[(size_t)r * P.ntile + t0 + lane] : 0u;
+        const uint32_t incl = warp_incl_scan(tc, lane);          // lanes >= BLK_TILES repeat the total
+        const uint32_t n = __shfl_sync(0xffffffffu, incl, 31);
         const size_t row = (size_t)r * P.cap;
-        for (uint32_t eb = 0; eb < n; eb += BT) {
-            const uint32_t e = eb + threadIdx.x;
-            const bool valid = e < n;
-            uint32_t idx = 0, sk = 0, seg = 0;
-            if (valid) {
-                int t = 0;
-                while (t + 1 < BLK_TILES && sh_tp[t + 1] <= e) ++t;
-                const size_t src = row + (size_t)(t0 + t) * STILE + (e - sh_tp[t]);
-                idx = P.stage_idx[src];
-                const float val = P.stage_val[src];
-                sk = RANDK ? ~philox_word(P, (uint32_t)r, idx, 1u) : topk_key(val);
-                P.cand_idx[row + base + e] = idx;
-                P.cand_val[row + base + e] = val;
-                if (RANDK) P.cand_key[row + base + e] = sk;
-                seg = segment_of(P, idx);
+        constexpr int OB = 4;                     // entries per lane whose reads are issued together
+        for (uint32_t eb = 0; eb < n; eb += 32 * OB) {
+            uint2 ent[OB];
+#pragma unroll
+            for (int q = 0; q < OB; ++q) {
+                const uint32_t e = eb + q * 32 + lane;
+                // tile of entry e: the number of tiles whose inclusive count is <= e
+                uint32_t t = 0, before = 0;
+#pragma unroll
+                for (int i = 0; i < BLK_TILES; ++i) {
+                    const uint32_t inc_i = __shfl_sync(0xffffffffu, incl, i);
+                    if (e >= inc_i) { t = i + 1; before = inc_i; }
+                }
+                ent[q] = make_uint2(0u, 0u);
+                if (e < n) ent[q] = P.stage[row + (size_t)(t0 + t) * STILE + (e - before)];
             }
-            // level 0 of the radix select: count the top key byte per unit
-            const uint32_t tag = (seg << 8) | (sk >> 24);
-            const uint32_t live = __ballot_sync(0xffffffffu, valid);
-            if (valid) {
-                const uint32_t peers = __match_any_sync(live, tag);
-                if (lane == __ffs(peers) - 1)
-                    atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
+#pragma unroll
+            for (int q = 0; q < OB; ++q) {
+                const uint32_t e = eb + q * 32 + lane;
+                const bool valid = e < n;
+                const uint32_t idx = ent[q].x;
+                uint32_t sk = 0, seg = 0;
+                if (valid) {
+                    const float val = __uint_as_float(ent[q].y);
+                    sk = RANDK ? ~philox_word(P, (uint32_t)r, idx, 1u) : topk_key(val);
+                    P.cand_idx[row + base + e] = idx;
+                    P.cand_val[row + base + e] = val;
+                    if (RANDK) P.cand_key[row + base + e] = sk;
+                    seg = segment_of(P, idx);
+                }
+                // level 0 of the radix select: count the top key byte per unit
+                const uint32_t tag = (seg << 8) | (sk >> 24);
+                const uint32_t live = __ballot_sync(0xffffffffu, valid);
+                if (valid) {
+                    const uint32_t peers = __match_any_sync(live, tag);
+                    if (lane == __ffs(peers) - 1) {
+                        if (local_bins) atomicAdd(&sh_bins[wslot * 256 + (sk >> 24)], __popc(peers));
+                        else atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
+                    }
+                }
             }
         }
-        __syncthreads();                          // the block's part of the ordered list is written
+        __syncwarp();                             // the block's part of the ordered list is written
         // segment boundaries inside this block: position of the first candidate at or after each
         const uint32_t lo = blk * (uint32_t)(BLK_TILES * STILE);
         const uint64_t hi64 = (uint64_t)lo + BLK_TILES * STILE;
@@ -163,7 +180,7 @@ __device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask
             s_lo = 1;
         }
         uint32_t* ss = P.seg_start + (size_t)r * (P.nseg + 1);
-        for (uint32_t sgm = s_lo + threadIdx.x; sgm < (uint32_t)P.nseg && P.seg_off[sgm] < hi; sgm += BT) {
+        for (uint32_t sgm = s_lo + lane; sgm < (uint32_t)P.nseg && P.seg_off[sgm] < hi; sgm += 32) {
             const uint32_t bound = P.seg_off[sgm];
             uint32_t a = 0, b = n;               // first entry of the block with index >= bound
             while (a < b) {
@@ -172,7 +189,13 @@ __device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask
             }
             ss[sgm] = base + a;
         }
-        if (blk == P.nblk - 1 && threadIdx.x == 0) ss[P.nseg] = base + n;
+        if (blk == P.nblk - 1 && lane == 0) ss[P.nseg] = base + n;
+    }
+    if (local_bins) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < act.n * 256; i += BT)
+            if (sh_bins[i]) atomicAdd(&P.hist[(size_t)act.r[i >> 8] * 256 + (i & 255)], sh_bins[i]);
+        __syncthreads();
     }
 }
 
@@ -598,18 +621,22 @@ __device__ void stage_norm_final(const Plan& P, const Tab& tab) {
                 big_add(dig, ND, a1, 2 * (ee - 1) + 24);
             }
         }
-        int top = -1;
-        for (int j = ND - 1; j >= 0 && top < 0; --j)
-            if (dig[j]) top = j * 32 + 31 - __clz(dig[j]);
+        int tw = ND - 1;
+        while (tw >= 0 && dig[tw] == 0) --tw;
         double sum = 0.0;
-        if (top >= 0) {
-            unsigned long long mant = 0;
-            for (int p = top; p > top - 53; --p)
-                mant = (mant << 1) | (p >= 0 ? (dig[p >> 5] >> (p & 31)) & 1u : 0u);
-            const int gp = top - 53;
-            const uint32_t guard = gp >= 0 ? (dig[gp >> 5] >> (gp & 31)) & 1u : 0u;
-            uint32_t sticky = 0;
-            for (int p = gp - 1; p >= 0 && !sticky; --p) sticky = (dig[p >> 5] >> (p & 31)) & 1u;
+        if (tw >= 0) {
+            const int top = tw * 32 + 31 - __clz(dig[tw]);
+            // the 64 bits that start at the top bit (zeros below bit 0), then the 53-bit mantissa
+            const int sh = 31 - (top & 31);                       // left shift that puts the top bit at bit 31
+            const uint32_t w0 = dig[tw], w1 = tw >= 1 ? dig[tw - 1] : 0u, w2 = tw >= 2 ? dig[tw - 2] : 0u;
+            const unsigned long long hi64 = ((unsigned long long)w0 << 32) | w1;
+            const unsigned long long bits = sh ? ((hi64 << sh) | ((unsigned long long)w2 >> (32 - sh))) : hi64;
+            unsigned long long mant = bits >> 11;
+            const uint32_t guard = (uint32_t)(bits >> 10) & 1u;
+            uint32_t sticky = (bits & 0x3ffull) != 0;
+            if (sh && (w2 << sh)) sticky = 1;                     // bits of the third word not shifted in
+            if (!sh && w2) sticky = 1;
+            for (int j = tw - 3; j >= 0 && !sticky; --j) sticky = dig[j] != 0;
             if (guard && (sticky || (mant & 1ull))) mant += 1ull;
             sum = ldexp((double)mant, top - 52 - (l1 ? 149 : 298));
         }
@@ -694,18 +721,35 @@ __device__ void stage_chunk_scan(const Plan& P, const Tab& tab, const Active& ac
     }
     __syncthreads();
     const bool has_lvl = P.qz != QS_SIGN_L1;
-    for (int w = threadIdx.x; w < act.n; w += BT) {
+    for (int w = 0; w < act.n; ++w) {
         const int r = act.r[w];
-        uint32_t pay = 2u * P.nseg;
+        uint32_t carry = 2u * P.nseg;
         long long bits = 0;
-        for (int g = 0; g < P.nseg; ++g) {
-            const uint32_t n = P.units[(size_t)r * P.nseg + g].n;
-            const uint32_t bi = P.bidx[g];
-            P.pay_off[(size_t)r * P.nseg + g] = pay;
-            pay += words_for(n, bi) + words_for(n, 1) + (has_lvl ? words_for(n, P.bl) : 0u);
-            bits += 64 + (long long)n * (bi + 1 + (has_lvl ? P.bl : 0));
+        for (uint32_t gb = 0; gb < (uint32_t)P.nseg; gb += BT) {
+            const uint32_t g = gb + threadIdx.x;
+            uint32_t words = 0, n = 0, bi = 0;
+            if (g < (uint32_t)P.nseg) {
+                n = P.units[(size_t)r * P.nseg + g].n;
+                bi = P.bidx[g];
+                words = words_for(n, bi) + words_for(n, 1) + (has_lvl ? words_for(n, P.bl) : 0u);
+                bits += 64 + (long long)n * (bi + 1 + (has_lvl ? P.bl : 0));
+            }
+            uint32_t total;
+            const uint32_t ex = block_excl_scan(words, sh, &total);
+            if (g < (uint32_t)P.nseg) P.pay_off[(size_t)r * P.nseg + g] = carry + ex;
+            carry += total;
         }
-        P.bits[r] = bits;
+        // sum of the per-thread bit counts
+        for (int o = 16; o; o >>= 1) bits += __shfl_xor_sync(0xffffffffu, bits, o);
+        __shared__ long long sh_bits[BT / 32];
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) sh_bits[threadIdx.x >> 5] = bits;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            long long t = 0;
+            for (int i = 0; i < BT / 32; ++i) t += sh_bits[i];
+            P.bits[r] = t;
+        }
     }
 }
 
@@ -924,7 +968,6 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_scan[33];
     __shared__ uint32_t sh_small[8];              // unit id, prefix, select scratch
     __shared__ uint32_t sh_w[BT / 32];
-    __shared__ uint32_t sh_tp[BLK_TILES + 1];
     __shared__ uint32_t sh_cnt[2 * 8 * GPW];
     __shared__ uint32_t sh_flag;
     __shared__ int sh_abort;
@@ -945,7 +988,7 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
 
     Tab tab;
     if (a.do_compress) {
-        stage_order<RANDK>(P, act, 0u, sh_scan, sh_tp);
+        stage_order<RANDK>(P, act, 0u, bins);
         QS_BARRIER();
         const uint32_t missed = build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
         if (missed) {                              // the same value in every block
@@ -955,7 +998,7 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
             QS_BARRIER();
             stage_reflag<RANDK>(P, act, missed, sh_cnt);
             QS_BARRIER();
-            stage_order<RANDK>(P, act, missed, sh_scan, sh_tp);
+            stage_order<RANDK>(P, act, missed, bins);
             QS_BARRIER();
             if (build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab)) set_status(P, QS_STATE);   // the exact pass cannot miss
             if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd((unsigned long long*)&P.stats[0], (unsigned long long)__popc(missed));
