@@ -144,6 +144,19 @@ def compress_feedback(plan, rnd, x, xw, mem, anchors=None, mask=None, mode=SORT,
     return out
 
 
+def compress_worker(plan, rnd, worker, anchor, xw_r, mem_r, mode=NTH):
+    """Worker half for the single worker `worker` on its own rows (mem_r updated in place)."""
+    stride = plan.wire_words()
+    wire = np.zeros(stride, dtype=np.uint32)
+    bits = np.zeros(1, dtype=np.int64)
+    rc = lib().qso_compress_worker(
+        C.c_int64(plan.d), C.c_int(plan.nseg), _p(plan.offsets, C.c_int64), _p(plan.kseg, C.c_int64),
+        C.c_int(plan.s), C.c_int(plan.sparsifier), C.c_int(plan.quantizer), C.c_uint64(plan.seed), C.c_uint64(rnd),
+        C.c_int(worker), _f32(anchor), _f32(xw_r), _f32(mem_r), _p(wire, C.c_uint32), C.c_int64(stride),
+        _p(bits, C.c_int64), C.c_int(mode))
+    return {"rc": rc, "wire": wire, "bits": int(bits[0])}
+
+
 def unpack_accumulate(plan, x, wire, mask=None):
     m = _mask(mask)
     wire = np.ascontiguousarray(wire, dtype=np.uint32)

@@ -494,6 +494,18 @@ int qso_compress_feedback(int R, int64_t d, int nseg, const int64_t* off, const 
     return ERR_OK;
 }
 
+// Worker half for one worker given by its id (the id enters the Philox counter), on that
+// worker's own rows: used where only some workers of a large configuration are replayed.
+int qso_compress_worker(int64_t d, int nseg, const int64_t* off, const int64_t* kseg, int s, int sparsifier,
+                        int quantizer, uint64_t seed, uint64_t round, int worker, const float* anchor,
+                        const float* xw_r, float* mem_r, uint32_t* wire, int64_t stride_words,
+                        int64_t* bits_out, int mode) {
+    Plan P = {worker + 1, d, nseg, off, kseg, s, sparsifier, quantizer, seed};
+    if (worker < 0 || !valid_plan(P)) return ERR_ARG;
+    if (stride_words < wire_words(P)) return ERR_CAPACITY;
+    return worker_compress(P, round, worker, anchor, xw_r, mem_r, wire, bits_out, mode, 0, 0, 0, 0, 0);
+}
+
 // Master half: decode the records of the workers in mask from the wire words,
 // accumulate in worker order, update x; the divisor is R whatever the mask.
 int qso_unpack_accumulate(int R, int64_t d, int nseg, const int64_t* off, const int64_t* kseg,

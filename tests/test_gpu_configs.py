@@ -1,0 +1,239 @@
+"""The five workload configurations at their full sizes, in the launch configuration bench.py times.
+
+Where the oracle can run the whole configuration in seconds (configs 1, 2, 4) everything is compared
+bit for bit.  At the sizes of configs 3 and 5 the oracle runs a subset of the workers in full
+(their records and memories are compared bit for bit) and the master update is checked at every
+index against an independent numpy decode of all the records the library wrote.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_1906_02367_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+B = None
+
+
+def setup_module(module):
+    global B
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_1906_02367_b200 import binding
+    B = binding
+
+
+def u32(a):
+    return np.ascontiguousarray(a).view(np.uint32)
+
+
+def clog2(v):
+    return max(1, (int(v) - 1).bit_length())
+
+
+def fields(words, count, width):
+    """count fixed-width LSB-first fields from a uint32 stream, vectorised."""
+    bitpos = np.arange(count, dtype=np.int64) * width
+    q, o = bitpos >> 5, (bitpos & 31).astype(np.uint64)
+    w = words.astype(np.uint64)
+    lo = w[q] >> o
+    hi = np.where(o + width > 32, w[np.minimum(q + 1, len(w) - 1)] << (np.uint64(32) - o), 0)
+    return ((lo | hi) & np.uint64((1 << width) - 1)).astype(np.int64)
+
+
+def numpy_master(x, wire, R, d, k, s, quantizer, workers):
+    """x - (1/R) sum of the decoded records, one segment, fp32 adds in worker order."""
+    acc = np.zeros(d, np.float32)
+    bi, bl = clog2(d), clog2(s)
+    beta = min(k / s**2, math.sqrt(k) / s)
+    c = np.float32(1.0 / (1.0 + beta))
+    for r in workers:
+        row = wire[r]
+        n = int(row[0])
+        N = row[1:2].view(np.float32)[0]
+        wi, ws = -(-n * bi // 32), -(-n // 32)
+        idx = fields(row[2:], n, bi)
+        sgn = fields(row[2 + wi:], n, 1)
+        if quantizer == O.SIGN_L1:
+            mag = np.full(n, N / np.float32(k), np.float32)
+        else:
+            lvl = fields(row[2 + wi + ws:], n, bl) + 1
+            mag = (N * lvl.astype(np.float32)) / np.float32(s)
+            if quantizer == O.QSGD_SCALED:
+                mag = (mag * c).astype(np.float32)
+        acc[idx] = acc[idx] + np.where(sgn == 1, -mag, mag).astype(np.float32)
+    return (x - acc / np.float32(R)).astype(np.float32)
+
+
+def test_config2_resnet50_shape_full_size():
+    # R = 8, d = 25,557,032 in 161 tensors, Laplace drift per tensor, memory carried; Top_k 0.1% flat and
+    # per tensor with the sign/l1 quantizer; two rounds each, everything compared with the oracle
+    sizes = I.resnet50_tensor_sizes()
+    off = I.segments_from_sizes(sizes)
+    d, R = int(off[-1]), 8
+    scales = I.tensor_scales(len(sizes), seed=0)
+    x0 = I.model_init(d, seed=0)
+    for kw in (dict(k=I.k_from_ratio(d, 1, 1000)), dict(offsets=off, kseg=I.k_per_tensor_ratio(sizes))):
+        plan = O.Plan(R, d, s=1, quantizer=O.SIGN_L1, seed=2, **kw)
+        x, xw, mem = x0.copy(), np.broadcast_to(x0, (R, d)).copy(), np.zeros((R, d), np.float32)
+        gx, gxw, gmem = (torch.from_numpy(a).cuda() for a in (x, xw, mem))
+        ctx = B.Context(R, d, int(plan.kseg[0]), 1, B.QS_TOPK, B.QS_SIGN_L1, seed=2)
+        if plan.nseg > 1:
+            ctx.set_segments(plan.offsets, plan.kseg)
+        ctx.bind(gx, gxw, gmem)
+        wire = ctx.new_wire()
+        bits = torch.zeros(R, dtype=torch.int64, device="cuda")
+        for rnd in range(2):
+            drift = I.laplace_drift(R, off, scales, 0, rnd)
+            xw += drift
+            gxw += torch.from_numpy(drift).cuda()
+            del drift
+            ref = O.sync_round(plan, rnd, x, xw, mem, mode=O.NTH, nthreads=8)
+            assert ref["rc"] == 0
+            ctx.sync_round(wire, rnd, bits_out=bits)
+            assert ctx.sync_status() == 0, ctx.last_error()
+            assert np.array_equal(u32(wire.cpu().numpy()), ref["wire"]), f"records, round {rnd}"
+            assert np.array_equal(bits.cpu().numpy(), ref["bits"])
+            assert np.array_equal(u32(gmem.cpu().numpy()), u32(mem)), f"memory, round {rnd}"
+            assert np.array_equal(u32(gx.cpu().numpy()), u32(x)), f"x, round {rnd}"
+            assert np.array_equal(u32(gxw.cpu().numpy()), u32(xw)), f"workers' copies, round {rnd}"
+        ctx.destroy()
+        del gx, gxw, gmem
+        torch.cuda.empty_cache()
+
+
+def check_large(R, d, k, s, sparsifier, quantizer, drift_kw, oracle_workers, rounds=2, seed=3):
+    """Full-size round with a subset of the workers replayed by the oracle."""
+    x0 = I.model_init(d, seed=1)
+    gx = torch.from_numpy(x0).cuda()
+    gxw = gx.expand(R, d).contiguous()
+    gmem = torch.zeros((R, d), dtype=torch.float32, device="cuda")
+    ctx = B.Context(R, d, k, s, sparsifier, quantizer, seed=seed)
+    ctx.bind(gx, gxw, gmem)
+    wire = ctx.new_wire()
+    bits = torch.zeros(R, dtype=torch.int64, device="cuda")
+    sub = np.zeros(R, np.uint8)
+    sub[oracle_workers] = 1
+    plan = O.Plan(R, d, k=k, s=s, sparsifier=sparsifier, quantizer=quantizer, seed=seed)
+    for rnd in range(rounds):
+        for r in range(R):                                   # drift drawn row by row to bound host memory
+            gxw[r] += torch.from_numpy(I.gaussian_drift(1, d, 100 + r, rnd, **drift_kw)[0]).cuda()
+        x_before = gx.cpu().numpy()
+        xw_sub = {r: gxw[r].cpu().numpy() for r in oracle_workers}
+        mem_sub = {r: gmem[r].cpu().numpy() for r in oracle_workers}
+        ctx.sync_round(wire, rnd, bits_out=bits)
+        assert ctx.sync_status() == 0, ctx.last_error()
+        w = u32(wire.cpu().numpy())
+        n_sent = w[:, 0].astype(np.int64)
+        assert np.all(n_sent <= k) and np.all(n_sent > 0)
+        has_lvl = quantizer != O.SIGN_L1
+        assert np.array_equal(bits.cpu().numpy(), 64 + n_sent * (clog2(d) + 1 + (clog2(s) if has_lvl else 0)))
+        # oracle replay of the chosen workers, one at a time (the other rows are never read)
+        for r in oracle_workers:
+            m1 = mem_sub[r].copy()
+            ref = O.compress_worker(plan, rnd, r, x_before, xw_sub[r], m1)
+            assert ref["rc"] == 0
+            assert np.array_equal(w[r, :ref["wire"].size], ref["wire"]), f"record of worker {r}, round {rnd}"
+            assert int(bits[r]) == ref["bits"]
+            assert np.array_equal(u32(gmem[r].cpu().numpy()), u32(m1)), f"memory of worker {r}, round {rnd}"
+        # master update at every index against an independent decode of all records
+        want = numpy_master(x_before, w, R, d, k, s, quantizer, range(R))
+        assert np.array_equal(u32(gx.cpu().numpy()), u32(want)), f"x, round {rnd}"
+        assert bool((gxw == gx[None, :]).all()), "broadcast"
+        for idxs in (fields(w[0, 2:], int(n_sent[0]), clog2(d)),):
+            assert np.all(np.diff(idxs) > 0) and idxs[-1] < d            # ascending, in range
+    st = ctx.stats()
+    ctx.destroy()
+    return st
+
+
+def test_config3_randk_full_size():
+    # R = 16, d = 2^26, Gaussian drift N(0, 1e-3), Rand_k 1% by keyed-hash rank, QSGD s = 4
+    d = 1 << 26
+    st = check_large(16, d, I.k_from_ratio(d, 1, 100), 4, O.RANDK, O.QSGD, dict(std=1e-3), [0, 11])
+    assert st["fallback_worker_rounds"] == 0
+
+
+@pytest.mark.parametrize("ratio,s", [((1, 10000), 2), ((1, 100), 16), ((1, 10), 256)])
+def test_config5_large_d_points(ratio, s):
+    # R = 4, d = 2^28, drift N(0, 1e-3) with 0.1% outliers x100, Top_k at several ratios, QSGD
+    d = 1 << 28
+    check_large(4, d, I.k_from_ratio(d, *ratio), s, O.TOPK, O.QSGD, dict(std=1e-3, outlier_frac=1e-3), [2],
+                rounds=2 if ratio[1] == 10000 else 1)
+
+
+def softmax_grads(xw, data, labels, parts, rng, batch=64, features=1024, classes=100):
+    """Minibatch gradient of softmax regression (weights then one bias per class) for every worker,
+    computed once on the host in fp32 and handed to both sides."""
+    R = xw.shape[0]
+    g = np.zeros_like(xw)
+    for r in range(R):
+        pick = parts[r][rng.integers(0, len(parts[r]), batch)]
+        A = torch.from_numpy(data[pick])
+        y = torch.from_numpy(labels[pick])
+        W = torch.from_numpy(xw[r, :features * classes]).reshape(features, classes)
+        b = torch.from_numpy(xw[r, features * classes:])
+        p = torch.softmax(A @ W + b, dim=1)
+        p[torch.arange(batch), y] -= 1.0
+        g[r, :features * classes] = ((A.T @ p) / batch).reshape(-1).numpy()
+        g[r, features * classes:] = p.mean(dim=0).numpy()
+    return g
+
+
+@pytest.mark.parametrize("asynchronous", [False, True])
+def test_config4_end_to_end_trajectory(asynchronous):
+    # softmax regression 1024 x 100 (+100 biases): d = 102,500, R = 8, minibatch 64, H = 8, eta = 0.05,
+    # Top_k 1% with QSGD s = 16, 500 synchronisations (sync) or 4000 steps of per-worker schedules (async).
+    # The data are a seeded Gaussian mixture split by class (40,000 samples stand in for the 400,000 of the
+    # configuration: the trajectory only ever sees minibatches).  Both sides receive the same gradients, so
+    # the trajectories must coincide bit for bit.
+    R, F, Cn, H, eta = 8, 1024, 100, 8, 0.05
+    d = F * Cn + Cn
+    k = I.k_from_ratio(d, 1, 100)
+    data, labels = I.gaussian_mixture(40000, F, Cn, seed=4)
+    parts = I.split_by_class(labels, R)
+    rng = np.random.default_rng(11)
+    T = 500 * H
+    sched = I.async_schedule(R, T, H, seed=8) if asynchronous else None
+    x = np.zeros(d, np.float32)
+    xw = np.zeros((R, d), np.float32)
+    mem = np.zeros((R, d), np.float32)
+    anchors = np.zeros((R, d), np.float32) if asynchronous else None
+    gx, gxw, gmem = (torch.from_numpy(a.copy()).cuda() for a in (x, xw, mem))
+    ganchors = torch.from_numpy(anchors.copy()).cuda() if asynchronous else None
+    plan = O.Plan(R, d, k=k, s=16, quantizer=O.QSGD, seed=6)
+    ctx = B.Context(R, d, k, 16, B.QS_TOPK, B.QS_QSGD, seed=6)
+    ctx.bind(gx, gxw, gmem, ganchors)
+    wire = ctx.new_wire()
+    rounds = 0
+    for t in range(T):
+        grad = softmax_grads(xw, data, labels, parts, rng)
+        O.local_step(plan, xw, grad, eta)
+        ctx.local_step(torch.from_numpy(grad).cuda(), eta)
+        if asynchronous:
+            mask = sched[t]
+            if not mask.any():
+                continue
+        else:
+            if (t + 1) % H:
+                continue
+            mask = None
+        assert O.sync_round(plan, t, x, xw, mem, anchors=anchors, mask=mask, mode=O.NTH)["rc"] == 0
+        ctx.sync_round(wire, t, mask)
+        rounds += 1
+        assert np.array_equal(u32(gx.cpu().numpy()), u32(x)), f"x after step {t}"
+    assert ctx.sync_status() == 0, ctx.last_error()
+    assert rounds >= 500
+    assert np.array_equal(u32(gxw.cpu().numpy()), u32(xw)) and np.array_equal(u32(gmem.cpu().numpy()), u32(mem))
+    if asynchronous:
+        assert np.array_equal(u32(ganchors.cpu().numpy()), u32(anchors))
+    # the run learned something: training loss of the global model on a sample is below log(classes)
+    A, y = torch.from_numpy(data[:4000]), torch.from_numpy(labels[:4000])
+    W, b = torch.from_numpy(x[:F * Cn]).reshape(F, Cn), torch.from_numpy(x[F * Cn:])
+    loss = float(torch.nn.functional.cross_entropy(A @ W + b, y))
+    assert loss < 0.9 * math.log(Cn), loss
+    ctx.destroy()

@@ -544,3 +544,16 @@ def test_resnet50_table_matches_the_paper():
     assert sum(sizes) == int(want["elements"])
     assert int(I.k_per_tensor_capped(sizes).sum()) == int(want["sum_min_dt_1000"])
     assert I.k_from_ratio(65536, 1, 100) == 655
+
+
+def test_single_worker_entry_equals_the_batch_entry():
+    R, d, k = 3, 5000, 50
+    x, xw, mem = I.gaussian_round(R, d, seed=1)
+    plan = O.Plan(R, d, k=k, s=4, sparsifier=O.RANDK, quantizer=O.QSGD, seed=9)
+    m2 = mem.copy()
+    out = O.compress_feedback(plan, 5, x, xw, m2)
+    for r in range(R):
+        mr = mem[r].copy()
+        one = O.compress_worker(plan, 5, r, x, xw[r].copy(), mr)
+        assert one["rc"] == 0 and np.array_equal(one["wire"], out["wire"][r])
+        assert np.array_equal(mr, m2[r]) and one["bits"] == out["bits"][r]
