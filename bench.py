@@ -30,6 +30,9 @@ R = 8
 METRIC = "sync_round_effective_bandwidth"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dense pass on the bench workload, from the
+# ncu capture summarised in profiles/, scaled from the half-size capture (traffic grows with d)
+DENSE_TRAFFIC_BYTES = 2479600000   # 1239.8 MB measured at half size (profiles/pass_a_tma_kernel_resnet50_half_size.txt) x 2
 
 
 def workload(variant, shrink=1):
@@ -89,6 +92,22 @@ class ClockSampler:
         reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
         return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons,
                 "power_w_max": max(float(r[2]) for r in rows), "samples": len(rows)}
+
+
+def max_over_ranks(ms, device):
+    """Slowest rank's time: the replicas are independent, the job is as slow as the slowest."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(bytes_per_round, steps, total_ms, world):
+    """Whole-job GB/s: every rank moved bytes_per_round per step in total_ms (max over ranks)."""
+    return world * bytes_per_round * steps / (total_ms * 1e-3) / 1e9
 
 
 def run_ours(args):
@@ -161,12 +180,9 @@ def run_ours(args):
     ctx.enable_phase_timing(False)
     st1 = ctx.stats()
     wire_bytes = int(bits.sum().item() + 7) // 8
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev)
     bmin = min_bytes(d, wire_bytes)
-    value = world * bmin * args.steps / (total_ms * 1e-3) / 1e9
+    value = aggregate_value(bmin, args.steps, total_ms, world)
     peak, peak_src = peak_hbm()
 
     result = {
@@ -188,12 +204,13 @@ def run_ours(args):
         "kernels_per_round": (st1["launches"] - st0["launches"]) / max(1, args.steps),
         "clocks": clocks,
     }
-    # roofline of the dominant kernel (the dense pass): 16 B per worker coordinate + 4 B per coordinate
+    # roofline of the dominant kernel (the dense pass: reads xw, mem, writes mem, reads x once):
+    # 12 B per worker coordinate + 4 B per coordinate
     dense_ms = phases["dense_pass"] / max(1, phases["rounds"])
-    dense_bytes = 16 * R * d + 4 * d
+    dense_bytes = 12 * R * d + 4 * d
     achieved = dense_bytes / (dense_ms * 1e-3) / 1e9 if dense_ms > 0 else 0.0
-    result["roofline"] = {"kernel": "pass_a_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                          "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+    result["roofline"] = {"kernel": "pass_a_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                          "frac": achieved / peak, "peak_source": peak_src, "traffic": DENSE_TRAFFIC_BYTES if args.shrink == 1 and args.variant == "flat" else None,
                           "algorithmic_bytes_per_launch": dense_bytes, "ms_per_launch": dense_ms}
 
     if rank == 0 and world == 1 and not args.no_e2e:
@@ -287,6 +304,69 @@ def run_reference(args):
     }))
 
 
+def run_sweep5(args):
+    """Large-d sweep: R = 4, d = 2^28, Gaussian drift N(0, 1e-3) with 0.1% outliers x100, Top_k ratio in
+    {1e-4, 1e-3, 1e-2, 1e-1} x QSGD s in {2, 16, 256}.  One JSON line with the twelve points."""
+    import torch
+    from paper_1906_02367_b200 import binding as B
+    R5, d = 4, 1 << 28
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+    x = torch.from_numpy(I.model_init(d, seed=1)).to(dev)
+    xw = x.expand(R5, d).contiguous()
+    mem = torch.zeros((R5, d), dtype=torch.float32, device=dev)
+    e1 = torch.empty(d, dtype=torch.float32, device=dev)
+    hit = torch.empty(d, dtype=torch.float32, device=dev)
+
+    def drift():
+        for r in range(R5):
+            e1.normal_(0.0, 1e-3, generator=gen)
+            hit.uniform_(generator=gen)
+            e1.mul_(torch.where(hit < 1e-3, 100.0, 1.0))
+            xw[r].add_(e1)
+
+    peak, peak_src = peak_hbm()
+    points = []
+    for den in (10000, 1000, 100, 10):
+        for s in (2, 16, 256):
+            k = I.k_from_ratio(d, 1, den)
+            mem.zero_()
+            xw.copy_(x.expand(R5, d))
+            ctx = B.Context(R5, d, k, s, B.QS_TOPK, B.QS_QSGD, seed=den + s)
+            ctx.bind(x, xw, mem)
+            wire = ctx.new_wire()
+            bits = torch.zeros(R5, dtype=torch.int64, device=dev)
+            for _ in range(max(3, args.warmup // 4)):
+                drift()
+                ctx.sync_round(wire, bits_out=bits)
+            st0 = ctx.stats()
+            times = []
+            for _ in range(max(3, args.steps // 20)):
+                drift()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                ctx.sync_round(wire, bits_out=bits)
+                b.record()
+                torch.cuda.synchronize()
+                times.append(a.elapsed_time(b))
+            assert ctx.sync_status() == 0, ctx.last_error()
+            st1 = ctx.stats()
+            ms = float(np.median(times))
+            bmin = 16 * R5 * d + 8 * d + 2 * (int(bits.sum().item() + 7) // 8)
+            gbs = bmin / (ms * 1e-3) / 1e9
+            points.append({"ratio": 1.0 / den, "k": k, "s": s, "ms_per_round": ms, "GBps": gbs,
+                           "pct_of_nominal_8TBps": 100 * gbs / NOMINAL_HBM_GBS, "pct_of_measured_copy": 100 * gbs / peak,
+                           "worker_elements_per_s": R5 * d / (ms * 1e-3),
+                           "fallback_worker_rounds": st1["fallback_worker_rounds"] - st0["fallback_worker_rounds"]})
+            ctx.destroy()
+            del wire
+            torch.cuda.empty_cache()
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "config": {"workload": "large-d sweep: R=4, d=2^28, Top_k x QSGD"},
+                      "peak_source": peak_src, "points": points}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -295,11 +375,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor"])
     ap.add_argument("--shrink", type=int, default=1, help="divide every tensor size (profiling on a small case)")
+    ap.add_argument("--sweep5", action="store_true", help="run the d = 2^28 ratio x s sweep instead of the headline workload")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    if args.impl == "reference":
+    if args.sweep5:
+        run_sweep5(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
