@@ -175,7 +175,8 @@ int qs_sync_round(qs_ctx* ctx, uint64_t round, const uint8_t* worker_mask, uint3
                   int64_t stride_words, int64_t* bits_out);
 
 /*
- * qs_export_selection — copies the result of the last compression out of scratch, for
+ * qs_export_selection — copies the result of the last compression, after it has been packed
+ * (qs_pack or qs_sync_round), out of scratch, for
  * checking against a reference (all device, any may be NULL):
  *   sel_idx  R x K int64, global indices of the kept sets, ascending, segments in order
  *            (K = sum of k_seg);  level R x K int32 (Sign: 1);  sign R x K bytes (1 = u < 0);

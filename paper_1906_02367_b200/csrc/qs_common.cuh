@@ -34,7 +34,7 @@ struct Active {          // workers taking part in a call, ascending
 struct Unit {            // one (worker, segment) pair
     uint32_t start;      // first candidate, position in the worker's list
     uint32_t c;          // number of candidates
-    uint32_t chunk_base; // first chunk in the global chunk numbering
+    uint32_t done;       // chunks of the unit that have added their part of the norm (back to 0 after use)
     uint32_t nchunks;
     uint32_t tau;        // sort key of the last kept coordinate
     uint32_t tie_max;    // largest index kept among keys equal to tau

@@ -84,6 +84,7 @@ struct Tab {
     const uint32_t* c;
     const uint32_t* cb;      // U + 1 entries
     uint32_t total_chunks;
+    bool fast;               // one segment and few chunks per unit: pack finds its own positions
 };
 
 __device__ __forceinline__ uint32_t segment_of(const Plan& P, uint32_t e) {
@@ -226,6 +227,9 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
     if (threadIdx.x == 0) t_cb[P.U] = carry;
     __syncthreads();
     tab->start = t_start; tab->c = t_c; tab->cb = t_cb; tab->total_chunks = carry;
+    bool fast = P.nseg == 1;
+    for (uint32_t u = 0; fast && u < P.U; ++u) fast = t_cb[u + 1] - t_cb[u] <= 1024u;
+    tab->fast = fast;
     return *sh_flag;
 }
 
@@ -524,6 +528,8 @@ __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t id
     return sk > un.tau || (sk == un.tau && idx <= un.tie_max);
 }
 
+__device__ void unit_norm(const Plan& P, uint32_t u);
+
 // Per-exponent integer sums of the kept values: for exponent e the squares' 48-bit mantissa
 // products are summed as two 24-bit halves (QSGD), or the 24-bit mantissas themselves (Sign).
 // A 64-bit sum cannot overflow below 2^32 terms.
@@ -578,6 +584,17 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, unsigned long lo
             atomicMin(&P.units[c.u].emin, threadIdx.x);
             atomicMax(&P.units[c.u].emax, threadIdx.x);
         }
+        // the chunk that completes its unit turns the sums into the norm
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const uint32_t nch = tab.cb[c.u + 1] - c.cb;
+            if (atomicAdd(&P.units[c.u].done, 1u) == nch - 1) {
+                __threadfence();
+                unit_norm(P, c.u);
+                P.units[c.u].done = 0;
+            }
+        }
     }
 }
 
@@ -598,19 +615,21 @@ __device__ void big_add(uint32_t* dig, int ndig, unsigned long long v, int bitpo
     }
 }
 
-// one thread per unit: exact sum -> fp64 (round to nearest even) -> norm in fp32
-__device__ void stage_norm_final(const Plan& P, const Tab& tab) {
-    for (uint32_t u = blockIdx.x * BT + threadIdx.x; u < P.U; u += gridDim.x * BT) {
+// one thread, once per unit, after every chunk has added its sums: exact sum -> fp64 (round to
+// nearest even) -> norm in fp32.  The sums were built with atomics in the L2: read them there.
+__device__ void unit_norm(const Plan& P, uint32_t u) {
+    {
         Unit& un = P.units[u];
-        if (tab.c[u] == 0 || un.emin > un.emax) continue;
+        const uint32_t emin = __ldcg(&un.emin), emax = __ldcg(&un.emax);
+        if (emin > emax) return;
         constexpr int ND = 24;                      // 768 bits
         uint32_t dig[ND];
         for (int j = 0; j < ND; ++j) dig[j] = 0;
         const bool l1 = P.qz == QS_SIGN_L1;
         // bit 0 stands for 2^-298 (squares) or 2^-149 (magnitudes)
-        for (uint32_t e = un.emin; e <= un.emax; ++e) {
+        for (uint32_t e = emin; e <= emax; ++e) {
             unsigned long long* g = P.eacc + ((size_t)u * 256 + e) * 2;
-            const unsigned long long a0 = g[0], a1 = g[1];
+            const unsigned long long a0 = __ldcg(g), a1 = __ldcg(g + 1);
             if (!(a0 | a1)) continue;
             g[0] = 0ull; g[1] = 0ull;
             const int ee = e ? (int)e : 1;          // subnormals share the exponent of e = 1
@@ -783,17 +802,45 @@ __device__ void stage_pack_dir(const Plan& P, const Active& act, uint32_t* wire,
 }
 
 // streams of every segment, and the ordered kept list kept for inspection
-__device__ void stage_pack(const Plan& P, const Tab& tab, uint32_t* wire, long long stride, uint32_t* sh_u, uint32_t* sh) {
+__device__ void stage_pack(const Plan& P, const Tab& tab, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
     const uint32_t total = tab.total_chunks;
     const bool has_lvl = P.qz != QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
-        uint32_t run_k = P.chunk_sel[chunk] - P.chunk_sel[c.cb];
-        uint32_t run_s = P.chunk_nz[chunk] - P.chunk_nz[c.cb];
+        uint32_t run_k, run_s, unit_n, pay;
         const uint32_t bi = P.bidx[c.seg], lo = P.seg_off[c.seg];
-        uint32_t* w_idx = wire + (size_t)c.r * stride + P.pay_off[c.u];
-        uint32_t* w_sgn = w_idx + words_for(c.un.n, bi);
-        uint32_t* w_lvl = w_sgn + words_for(c.un.n, 1);
+        if (tab.fast) {
+            // positions from the chunk counts of the unit directly (no scan stage ran)
+            const uint32_t c1 = tab.cb[c.u + 1];
+            uint32_t bk = 0, bs = 0, ak = 0, as = 0;
+            for (uint32_t i = c.cb + threadIdx.x; i < c1; i += BT) {
+                const uint32_t v = P.chunk_cnt[i];
+                ak += v & 0xffffu; as += v >> 16;
+                if (i < chunk) { bk += v & 0xffffu; bs += v >> 16; }
+            }
+            uint32_t t0, t1, t2, t3;
+            block_excl_scan(bk, sh, &t0); block_excl_scan(bs, sh, &t1);
+            block_excl_scan(ak, sh, &t2); block_excl_scan(as, sh, &t3);
+            run_k = t0; run_s = t1; unit_n = t3; pay = 2u;
+            if (chunk == c.cb && threadIdx.x == 0) {          // the unit's first chunk writes its directory entry
+                P.units[c.u].n = unit_n;
+                if (t2 != P.kseg[c.seg]) set_status(P, QS_STATE);
+                uint32_t* row = wire + (size_t)c.r * stride;
+                row[0] = unit_n;
+                row[1] = __float_as_uint(c.un.norm);
+                const long long bits = 64 + (long long)unit_n * (bi + 1 + (has_lvl ? P.bl : 0));
+                P.bits[c.r] = bits;
+                if (bits_out) bits_out[c.r] = bits;
+            }
+        } else {
+            run_k = P.chunk_sel[chunk] - P.chunk_sel[c.cb];
+            run_s = P.chunk_nz[chunk] - P.chunk_nz[c.cb];
+            unit_n = c.un.n;
+            pay = P.pay_off[c.u];
+        }
+        uint32_t* w_idx = wire + (size_t)c.r * stride + pay;
+        uint32_t* w_sgn = w_idx + words_for(unit_n, bi);
+        uint32_t* w_lvl = w_sgn + words_for(unit_n, 1);
         uint32_t* o_idx = P.sel_idx + (size_t)c.r * P.K + P.kprefix[c.seg];
         uint32_t* o_q = P.sel_q + (size_t)c.r * P.K + P.kprefix[c.seg];
         uint32_t q[PER], e[PER];
@@ -808,11 +855,11 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, uint32_t* wire, long l
             const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
             uint32_t tot;
             const uint32_t ex = block_excl_scan(kept | (sent << 16), sh, &tot);
-            if (kept) {
+            if (kept && run_k + (ex & 0xffffu) < P.kseg[c.seg]) {      // (the bound holds by construction)
                 const uint32_t jk = run_k + (ex & 0xffffu);
                 o_idx[jk] = e[i];
                 o_q[jk] = q[i];
-                if (sent) {
+                if (sent && run_s + (ex >> 16) < unit_n) {
                     const uint64_t js = run_s + (ex >> 16);
                     or_bits(w_idx, js * bi, bi, e[i] - lo);
                     if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
@@ -856,8 +903,31 @@ __device__ void stage_dec_prep(const Plan& P, const Active& act, const uint32_t*
 
 struct Entry { uint32_t seg, j, n, coord; const uint32_t* w_idx; };
 
+// entries and stream offset of one segment of worker r's record
+__device__ __forceinline__ void record_segment(const Plan& P, const uint32_t* wire, long long stride, int r,
+                                               uint32_t seg, uint32_t* n, uint32_t* pay) {
+    if (P.nseg == 1) {                           // read straight from the record: no offsets to look up
+        const uint32_t v = wire[(size_t)r * stride];
+        *n = v <= P.kseg[0] ? v : 0u;
+        *pay = 2u;
+    } else {
+        const uint32_t* eb = P.dec_ent + (size_t)r * (P.nseg + 1);
+        *n = eb[seg + 1] - eb[seg];
+        *pay = P.dec_pay[(size_t)r * P.nseg + seg];
+    }
+}
+
 __device__ __forceinline__ bool locate_entry(const Plan& P, const uint32_t* wire, long long stride, int r,
                                              uint32_t ent, Entry* out) {
+    if (P.nseg == 1) {
+        uint32_t n, pay;
+        record_segment(P, wire, stride, r, 0u, &n, &pay);
+        if (ent >= n) return false;
+        out->seg = 0; out->j = ent; out->n = n;
+        out->w_idx = wire + (size_t)r * stride + pay;
+        out->coord = get_bits(out->w_idx, (uint64_t)ent * P.bidx[0], P.bidx[0]);
+        return true;
+    }
     const uint32_t* eb = P.dec_ent + (size_t)r * (P.nseg + 1);
     if (ent >= eb[P.nseg]) return false;
     uint32_t lo = 0, hi = P.nseg;                // eb[lo] <= ent < eb[hi]
@@ -887,6 +957,7 @@ __device__ void stage_dec_mark(const Plan& P, const Active& act, const uint32_t*
     for (uint64_t id = (uint64_t)blockIdx.x * BT + threadIdx.x; id < total; id += (uint64_t)gridDim.x * BT) {
         const int r = act.r[id / P.K];
         Entry en;
+        if (P.nseg == 1 && id % P.K == 0 && wire[(size_t)r * stride] > P.kseg[0]) set_status(P, QS_INVALID_ARG);
         if (!locate_entry(P, wire, stride, r, (uint32_t)(id % P.K), &en)) continue;
         if (en.coord < P.d) atomicOr(&P.touch[en.coord], 1u << r);
         else set_status(P, QS_INVALID_ARG);
@@ -911,11 +982,11 @@ __device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t
         while (rest) {
             const int r2 = __ffs(rest) - 1;
             rest &= rest - 1u;
-            const uint32_t* eb = P.dec_ent + (size_t)r2 * (P.nseg + 1);
             Entry e2;
+            uint32_t pay2;
             e2.seg = en.seg;
-            e2.n = eb[en.seg + 1] - eb[en.seg];
-            e2.w_idx = wire + (size_t)r2 * stride + P.dec_pay[(size_t)r2 * P.nseg + en.seg];
+            record_segment(P, wire, stride, r2, en.seg, &e2.n, &pay2);
+            e2.w_idx = wire + (size_t)r2 * stride + pay2;
             uint32_t lo = 0, hi = e2.n;              // first position with index >= local
             while (lo < hi) {
                 const uint32_t mid = (lo + hi) >> 1;
@@ -1019,23 +1090,25 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
         QS_BARRIER();
         stage_norm_accum<RANDK>(P, tab, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0]);
         QS_BARRIER();
-        stage_norm_final(P, tab);
-        QS_BARRIER();
         stage_quant<RANDK>(P, tab, &sh_small[0], sh_w);
         QS_BARRIER();
-        stage_chunk_scan(P, tab, act, sh_scan);
-        QS_BARRIER();
+        if (!tab.fast) {
+            stage_chunk_scan(P, tab, act, sh_scan);
+            QS_BARRIER();
+        }
     } else if (a.do_pack) {
         build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
     }
     if (a.do_pack) {
-        stage_pack_dir(P, act, a.wire, a.stride, a.bits_out);
-        stage_pack(P, tab, a.wire, a.stride, &sh_small[0], sh_scan);
+        if (!tab.fast) stage_pack_dir(P, act, a.wire, a.stride, a.bits_out);
+        stage_pack(P, tab, a.wire, a.stride, a.bits_out, &sh_small[0], sh_scan);
         if (a.do_decode) QS_BARRIER();
     }
     if (a.do_decode) {
-        stage_dec_prep(P, act, a.wire, a.stride, sh_scan);
-        QS_BARRIER();
+        if (P.nseg > 1) {
+            stage_dec_prep(P, act, a.wire, a.stride, sh_scan);
+            QS_BARRIER();
+        }
         stage_dec_mark(P, act, a.wire, a.stride);
         QS_BARRIER();
         stage_dec_apply(P, act, a.wire, a.stride, a.patch);
