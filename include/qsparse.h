@@ -30,7 +30,7 @@
  *     word that qs_sync_status reads after synchronising the stream.
  *   - Status codes: QS_OK = 0, negative = error.  Nothing is printed, nothing aborts.
  *   - worker_mask: host array of R bytes, non-zero = worker takes part; NULL = all.
- *   - R <= 32, 1 <= k <= d < 2^32, 1 <= s <= 65535, round < 2^56.
+ *   - R <= 32, 1 <= k <= d < 2^32, 1 <= s <= 65535, round < 2^56, R x nseg <= 2048.
  *
  * Arithmetic (identical, operation for operation, to the CPU checker under oracle/):
  *   fp32 with no fused multiply-add; u = mem + (x - xw); Top_k orders by the bit
@@ -87,7 +87,8 @@ enum {
  *                (round_hi << 8) | stream) and output word element & 3; stream 0 feeds
  *                the quantizer, stream 1 the Rand_k subset.
  *   cuda_stream  a cudaStream_t (NULL = the legacy default stream).
- * Allocates all scratch (about 8 R d bytes of candidate storage plus small tables); one
+ * Allocates all scratch (candidate storage sized for the worst case, 20 R d bytes, 24 for
+ * Rand_k, plus 4 d bytes of sender bits and small tables); one
  * segment [0, d) with k is installed.  Returns QS_INVALID_ARG, QS_ALLOC or QS_CUDA on
  * failure, in which case *out is NULL.
  */
@@ -165,11 +166,11 @@ int qs_unpack_accumulate(qs_ctx* ctx, const uint32_t* wire, int64_t stride_words
 int qs_broadcast(qs_ctx* ctx, const uint8_t* worker_mask);
 
 /*
- * qs_sync_round — the whole synchronisation for the masked workers, with the same
- * final bytes in x, xw, mem, anchors, wire and bits_out as qs_compress_feedback,
- * qs_pack, qs_unpack_accumulate, qs_broadcast in that order, but with the broadcast
- * folded into the pass that forms u and the few changed coordinates patched after the
- * decode.  wire / stride_words / bits_out as in qs_pack.
+ * qs_sync_round — the whole synchronisation for the masked workers, with the same final
+ * bytes in x, xw, mem, anchors, wire and bits_out as qs_compress_feedback, qs_pack,
+ * qs_unpack_accumulate, qs_broadcast in that order, in two kernel launches: the dense pass
+ * that forms u, and one persistent kernel that runs every later step and ends with the
+ * broadcast.  wire / stride_words / bits_out as in qs_pack.
  */
 int qs_sync_round(qs_ctx* ctx, uint64_t round, const uint8_t* worker_mask, uint32_t* wire,
                   int64_t stride_words, int64_t* bits_out);

@@ -32,8 +32,8 @@ struct Active {          // workers taking part in a call, ascending
 };
 
 struct Unit {            // one (worker, segment) pair
-    uint32_t start;      // first candidate, position in the worker's list
-    uint32_t c;          // number of candidates
+    uint32_t tie_t;      // non-zero while a large unit waits for its tie cut: equal keys to keep
+    uint32_t spare;
     uint32_t done;       // chunks of the unit that have added their part of the norm (back to 0 after use)
     uint32_t nchunks;
     uint32_t tau;        // sort key of the last kept coordinate

@@ -472,8 +472,12 @@ __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32
         __syncthreads();
         for (int L = 0; L < 4; ++L) P.hist[((size_t)L * P.U + u) * 256 + threadIdx.x] = 0;
         const uint32_t tau = sh4[0], t = sh4[1], ceq = sh4[2];
-        uint32_t tie_max = 0xffffffffu;
-        if (ceq > t) {
+        uint32_t tie_max = 0xffffffffu, tie_t = 0;
+        if (ceq > t && uc > 16u * BT) {
+            // more equal keys than slots in a long list: the cut is found by all blocks together
+            tie_t = t;
+            if (threadIdx.x == 0) atomicOr(&P.fail[0], 1u);
+        } else if (ceq > t) {
             // more equal keys than slots: the t lowest coordinates win; walk the list in order
             const size_t base = (size_t)r * P.cap + tab.start[u];
             for (uint32_t first = 0; first < uc; first += BT) {
@@ -497,6 +501,7 @@ __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32
             Unit& out = P.units[u];
             out.tau = tau;
             out.tie_max = tie_max;
+            out.tie_t = tie_t;
             out.n = 0;
             out.emin = 255u;
             out.emax = 0u;
@@ -520,6 +525,86 @@ __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32
             }
         }
     }
+}
+
+// Tie cut of long lists, step 1: keys equal to the threshold in every chunk of a waiting unit
+template <bool RANDK>
+__device__ void stage_tie_count(const Plan& P, const Tab& tab, uint32_t* sh_u, uint32_t* sh_w) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (uint32_t chunk = blockIdx.x; chunk < tab.total_chunks; chunk += gridDim.x) {
+        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+        if (c.un.tie_t == 0) continue;
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const uint32_t off = c.first + i * BT + threadIdx.x;
+            if (off < c.c && sort_key<RANDK>(P, c.base + off) == c.un.tau) ++cnt;
+        }
+        cnt = warp_sum(cnt);
+        if (lane == 0) sh_w[wid] = cnt;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t t = 0;
+            for (int w = 0; w < BT / 32; ++w) t += sh_w[w];
+            P.chunk_cnt[chunk] = t;
+        }
+    }
+}
+
+// step 2: the chunk that holds the last kept tie, then the coordinate itself
+template <bool RANDK>
+__device__ void stage_tie_find(const Plan& P, const Tab& tab, uint32_t* sh, uint32_t* sh4, uint32_t* sh_w) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (uint32_t u = blockIdx.x; u < P.U; u += gridDim.x) {
+        const Unit un = P.units[u];
+        if (un.tie_t == 0) continue;
+        const uint32_t c0 = tab.cb[u], c1 = tab.cb[u + 1], t = un.tie_t;
+        __syncthreads();
+        if (threadIdx.x == 0) { sh4[0] = 0xffffffffu; sh4[1] = 0; sh4[3] = 0xffffffffu; sh4[4] = 0; }
+        __syncthreads();
+        uint32_t carry = 0;
+        for (uint32_t cb = c0; cb < c1; cb += BT) {
+            const uint32_t i = cb + threadIdx.x;
+            const uint32_t v = i < c1 ? P.chunk_cnt[i] : 0u;
+            uint32_t total;
+            const uint32_t ex = block_excl_scan(v, sh, &total);
+            if (carry + ex < t && carry + ex + v >= t) { sh4[0] = i; sh4[1] = carry + ex; }
+            carry += total;
+            __syncthreads();
+            if (sh4[0] != 0xffffffffu) break;
+        }
+        const uint32_t chunk = sh4[0], before_chunk = sh4[1];
+        uint32_t tie_max = 0xffffffffu;
+        if (chunk != 0xffffffffu) {
+            const uint32_t uc = tab.c[u];
+            const size_t base = (size_t)(u / P.nseg) * P.cap + tab.start[u];
+            const uint32_t first0 = (chunk - c0) * CHUNK;
+            if (threadIdx.x == 0) sh4[4] = before_chunk;
+            __syncthreads();
+            for (uint32_t first = first0; first < first0 + CHUNK; first += BT) {
+                const uint32_t off = first + threadIdx.x;
+                const bool eq = off < uc && sort_key<RANDK>(P, base + off) == un.tau;
+                const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+                if (lane == 0) sh_w[wid] = __popc(bal);
+                __syncthreads();
+                uint32_t before = sh4[4];
+                for (int w = 0; w < wid; ++w) before += sh_w[w];
+                const uint32_t mine = before + __popc(bal & ((1u << lane) - 1u));
+                if (eq && mine == t - 1) sh4[3] = P.cand_idx[base + off];
+                __syncthreads();
+                if (threadIdx.x == 0) { uint32_t s2 = 0; for (int w = 0; w < BT / 32; ++w) s2 += sh_w[w]; sh4[4] += s2; }
+                __syncthreads();
+                if (sh4[3] != 0xffffffffu) break;
+            }
+            tie_max = sh4[3];
+        }
+        if (threadIdx.x == 0) {
+            if (tie_max == 0xffffffffu) set_status(P, QS_STATE);      // the counts said it is there
+            P.units[u].tie_max = tie_max;
+            P.units[u].tie_t = 0;
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) P.fail[0] = 0;
 }
 
 // ------------------------------------------------------------------ quantize
@@ -1088,6 +1173,12 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
         }
         stage_final<RANDK>(P, tab, &sh_small[2], sh_w);
         QS_BARRIER();
+        if (P.fail[0]) {                           // some long list has more equal keys than slots (same in every block)
+            stage_tie_count<RANDK>(P, tab, &sh_small[0], sh_w);
+            QS_BARRIER();
+            stage_tie_find<RANDK>(P, tab, sh_scan, &sh_small[2], sh_w);
+            QS_BARRIER();
+        }
         stage_norm_accum<RANDK>(P, tab, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0]);
         QS_BARRIER();
         stage_quant<RANDK>(P, tab, &sh_small[0], sh_w);

@@ -156,6 +156,21 @@ def test_ties_zeros_and_equal_values():
             p.close()
 
 
+def test_ties_in_long_candidate_lists():
+    # many equal keys at the threshold of a long list: the cut by lower index is found by all blocks together
+    R, d = 3, 200000
+    g = np.random.default_rng(5)
+    z = np.zeros((R, d), np.float32)
+    few = g.choice(np.array([0.5, 1.0, -1.0, 2.0, -0.25], np.float32), size=(R, d)).astype(np.float32)
+    for xw, k in ((few, 70000), (few, 150000), (z.copy(), 30000)):
+        for sp in (O.TOPK,):
+            p = Pair(R, d, k=k, s=16, sparsifier=sp, quantizer=O.QSGD, seed=2, x=np.zeros(d, np.float32), xw=xw, mem=z.copy())
+            p.round_split(0)
+            p.drift(few * np.float32(0.5))
+            p.round_fused(1)
+            p.close()
+
+
 def test_per_tensor_and_flat_over_rounds():
     # ResNet-50-shaped table shrunk 64x: 161 segments, many of one element; memory carried over
     # rounds with a fresh Laplace drift each round; Sign/l1 operator; flat and per-tensor
