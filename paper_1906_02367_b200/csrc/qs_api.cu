@@ -241,6 +241,8 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(dec_ent, (size_t)R * (nseg + 1), true);
     AL(dec_pay, P.U, true);
     AL(touch, (size_t)d, true);
+    AL(coll, (size_t)R * P.K, false);
+    AL(ncoll, 1, true);
     AL(status, 1, true);
     AL(bar, 2, true);
     AL(trace, TRACE_SLOTS, true);
@@ -258,6 +260,8 @@ int rezero(qs_ctx* c) {
     QS_CUDA_TRY(c, cudaMemsetAsync(P.fb_hist, 0, sizeof(uint32_t) * P.U * FB_BINS, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.touch, 0, sizeof(uint32_t) * P.d, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.fail, 0, sizeof(uint32_t) * P.R, c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.ncoll, 0, sizeof(uint32_t), c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.units, 0, sizeof(Unit) * P.U, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.status, 0, sizeof(int), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 2 * sizeof(uint32_t), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.blk_count, 0, sizeof(uint32_t) * P.R * P.nblk, c->st));

@@ -90,6 +90,8 @@ struct Plan {
     uint32_t* dec_ent;         // R x (nseg + 1)
     uint32_t* dec_pay;         // R x nseg
     uint32_t* touch;           // d, zero between rounds
+    uint2* coll;               // R x K: (coordinate, unit) of indices several workers sent, fused round
+    uint32_t* ncoll;           // 1, zero between rounds
     int* status;
     uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel
     unsigned long long* trace; // TRACE_SLOTS global-timer stamps of the last persistent launch, or null

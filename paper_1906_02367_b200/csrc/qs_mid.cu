@@ -750,7 +750,7 @@ __device__ void unit_norm(const Plan& P, uint32_t u) {
 
 // levels, signs, memory update; kept and sent counts per chunk
 template <bool RANDK>
-__device__ void stage_quant(const Plan& P, const Tab& tab, uint32_t* sh_u, uint32_t* sh_w) {
+__device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_chunks;
     const bool sign_op = P.qz == QS_SIGN_L1;
@@ -784,6 +784,7 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, uint32_t* sh_u, uint3
                 if (level) {
                     mem[idx[i]] = val[i] - coord_value(P, N, level, neg, cs, k);
                     cnt += 1u << 16;
+                    if (fused) atomicOr(&P.touch[idx[i]], 1u << c.r);     // the master's "who sent this index"
                 }
             }
             P.cand_q[c.base + off] = q;
@@ -887,7 +888,7 @@ __device__ void stage_pack_dir(const Plan& P, const Active& act, uint32_t* wire,
 }
 
 // streams of every segment, and the ordered kept list kept for inspection
-__device__ void stage_pack(const Plan& P, const Tab& tab, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
+__device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
     const uint32_t total = tab.total_chunks;
     const bool has_lvl = P.qz != QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
@@ -928,7 +929,7 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, uint32_t* wire, long l
         uint32_t* w_lvl = w_sgn + words_for(unit_n, 1);
         uint32_t* o_idx = P.sel_idx + (size_t)c.r * P.K + P.kprefix[c.seg];
         uint32_t* o_q = P.sel_q + (size_t)c.r * P.K + P.kprefix[c.seg];
-        uint32_t q[PER], e[PER];
+        uint32_t q[PER], e[PER], sent_mask = 0;
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
@@ -949,10 +950,39 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, uint32_t* wire, long l
                     or_bits(w_idx, js * bi, bi, e[i] - lo);
                     if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
                     if (has_lvl) or_bits(w_lvl, js * P.bl, P.bl, (q[i] & 0xffffu) - 1u);
+                    sent_mask |= 1u << i;
                 }
             }
             run_k += tot & 0xffffu;
             run_s += tot >> 16;
+        }
+        if (fused) {
+            // Master update riding along: an index only this worker sent gets acc = 0 + g,
+            // x <- x - acc / R right here; an index with several senders has each sender leave its
+            // value at (worker, coordinate) and the lowest sender list it for the next stage.
+            // All reads of one kind are issued together: this part is bound by memory latency.
+            uint32_t senders[PER];
+            float xv[PER];
+#pragma unroll
+            for (int i = 0; i < PER; ++i) senders[i] = ((sent_mask >> i) & 1u) ? P.touch[e[i]] : 0u;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) xv[i] = (senders[i] == (1u << c.r)) ? P.x[e[i]] : 0.0f;
+            float* gval = reinterpret_cast<float*>(P.stage);
+#pragma unroll
+            for (int i = 0; i < PER; ++i) {
+                if (!senders[i]) continue;
+                const float g = coord_value(P, c.un.norm, (int)(q[i] & 0xffffu), (q[i] & Q_NEG) != 0, P.cscale[c.seg],
+                                            P.kseg[c.seg]);
+                if (senders[i] == (1u << c.r)) {
+                    float acc = 0.0f;
+                    acc = acc + g;
+                    P.x[e[i]] = xv[i] - acc / (float)P.R;
+                    P.touch[e[i]] = 0u;
+                } else {
+                    gval[(size_t)c.r * P.cap + e[i]] = g;
+                    if ((uint32_t)(__ffs(senders[i]) - 1) == c.r) P.coll[atomicAdd(P.ncoll, 1u)] = make_uint2(e[i], c.u);
+                }
+            }
         }
     }
 }
@@ -1093,6 +1123,25 @@ __device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t
     }
 }
 
+// Fused round: indices that several workers sent.  Their lowest sender listed them and every sender
+// left its value at (worker, coordinate); here they are added in increasing worker order.
+__device__ void stage_coll_apply(const Plan& P) {
+    const uint32_t n = *P.ncoll;
+    const float* gval = reinterpret_cast<const float*>(P.stage);
+    for (uint32_t id = blockIdx.x * BT + threadIdx.x; id < n; id += gridDim.x * BT) {
+        const uint32_t coord = P.coll[id].x;
+        uint32_t rest = P.touch[coord];
+        float acc = 0.0f;
+        while (rest) {
+            const int r2 = __ffs(rest) - 1;
+            rest &= rest - 1u;
+            acc = acc + gval[(size_t)r2 * P.cap + coord];
+        }
+        P.x[coord] = P.x[coord] - acc / (float)P.R;
+        P.touch[coord] = 0u;
+    }
+}
+
 // xw_r <- x (and the anchors) for the active workers: the closing dense stage of a fused round
 template <bool ALIGNED>
 __device__ void stage_broadcast(const Plan& P, const Active& act) {
@@ -1143,6 +1192,7 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
 #define QS_BARRIER() do { if (!grid_barrier(P, target, &sh_abort)) return; } while (0)
 
     Tab tab;
+    const bool fused = a.do_compress && a.do_pack && a.do_decode;   // whole round: the master update rides along
     if (a.do_compress) {
         stage_order<RANDK>(P, act, 0u, bins);
         QS_BARRIER();
@@ -1181,7 +1231,7 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
         }
         stage_norm_accum<RANDK>(P, tab, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0]);
         QS_BARRIER();
-        stage_quant<RANDK>(P, tab, &sh_small[0], sh_w);
+        stage_quant<RANDK>(P, tab, fused, &sh_small[0], sh_w);
         QS_BARRIER();
         if (!tab.fast) {
             stage_chunk_scan(P, tab, act, sh_scan);
@@ -1192,10 +1242,12 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     }
     if (a.do_pack) {
         if (!tab.fast) stage_pack_dir(P, act, a.wire, a.stride, a.bits_out);
-        stage_pack(P, tab, a.wire, a.stride, a.bits_out, &sh_small[0], sh_scan);
+        stage_pack(P, tab, fused, a.wire, a.stride, a.bits_out, &sh_small[0], sh_scan);
         if (a.do_decode) QS_BARRIER();
     }
-    if (a.do_decode) {
+    if (fused) {
+        stage_coll_apply(P);
+    } else if (a.do_decode) {
         if (P.nseg > 1) {
             stage_dec_prep(P, act, a.wire, a.stride, sh_scan);
             QS_BARRIER();
@@ -1221,6 +1273,7 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
         if (atomicAdd(P.bar + 1, 1u) == gridDim.x - 1) {
             P.bar[0] = 0;
             P.bar[1] = 0;
+            *P.ncoll = 0;
         }
     }
 }
