@@ -19,6 +19,7 @@
 //               order, updates x and (fused round) patches the workers' copies
 //
 // Order-dependent results come only from ordered scans, never from the order of atomics.
+#include "qs_bulk.cuh"
 #include "qs_kernels.h"
 
 namespace qs {
@@ -1167,6 +1168,49 @@ __device__ void stage_broadcast(const Plan& P, const Active& act) {
     }
 }
 
+// The same broadcast through the bulk-copy engine (16-byte-aligned rows): one thread per block
+// brings tiles of x into a ring of three shared-memory buffers and sends each out to every active
+// worker's row; no data passes through registers.  Waits are bounded.
+__device__ void stage_broadcast_bulk(const Plan& P, const Active& act, float* buf0, float* buf1, float* buf2,
+                                     uint64_t* mbar, int* sh_abort) {
+    if (threadIdx.x != 0) return;
+    float* buf[3] = {buf0, buf1, buf2};
+    for (int b = 0; b < 3; ++b) mbar_init(&mbar[b], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();                              // the buffers were ordinary shared memory until now
+    const uint32_t ntiles = P.ntile;
+    const uint32_t mine = blockIdx.x < ntiles ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    auto load = [&](uint32_t i) {
+        const uint32_t e0 = (blockIdx.x + i * gridDim.x) * (uint32_t)STILE;
+        const uint32_t bytes = (P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE) * 4u;
+        mbar_expect(&mbar[i % 3], bytes);
+        bulk_load(buf[i % 3], P.x + e0, bytes, &mbar[i % 3]);
+    };
+    for (uint32_t i = 0; i < 2 && i < mine; ++i) load(i);
+    uint32_t done = 0;
+    for (uint32_t i = 0; i < mine; ++i) {
+        if (!mbar_wait(&mbar[i % 3], (i / 3) & 1u)) { *sh_abort = 1; break; }
+        done = i + 1;
+        const uint32_t e0 = (blockIdx.x + i * gridDim.x) * (uint32_t)STILE;
+        const uint32_t bytes = (P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE) * 4u;
+        for (int w = 0; w < act.n; ++w) {
+            bulk_store(P.xw + (size_t)act.r[w] * P.d + e0, buf[i % 3], bytes);
+            if (P.anchors) bulk_store(P.anchors + (size_t)act.r[w] * P.d + e0, buf[i % 3], bytes);
+        }
+        bulk_commit();
+        if (i + 2 < mine) {
+            bulk_wait_read<1>();                     // the buffer of tile i - 1 has been read by its stores
+            load(i + 2);
+        }
+    }
+    if (*sh_abort) {
+        // loads already issued get a bounded chance to land before the block leaves
+        for (uint32_t i = done; i < mine && i < done + 2; ++i) mbar_wait(&mbar[i % 3], (i / 3) & 1u);
+        set_status(P, QS_TIMEOUT);
+    }
+    bulk_wait_all();
+}
+
 // ------------------------------------------------------------------ the persistent kernel
 template <bool RANDK>
 __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
@@ -1176,7 +1220,8 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_cnt[2 * 8 * GPW];
     __shared__ uint32_t sh_flag;
     __shared__ int sh_abort;
-    __shared__ uint32_t t_start[UT_MAX], t_c[UT_MAX], t_cb[UT_MAX + 1];
+    __shared__ __align__(128) uint32_t t_start[UT_MAX], t_c[UT_MAX], t_cb[UT_MAX + 4];
+    __shared__ __align__(8) uint64_t sh_mbar[3];
     __shared__ __align__(16) unsigned char sh_big[FB_BINS * 4];   // fallback bins / radix bins / exponent sums
     const Plan& P = a.P;
     const Active& act = a.act;
@@ -1258,8 +1303,13 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     }
     if (a.do_broadcast) {
         QS_BARRIER();
-        if (a.aligned) stage_broadcast<true>(P, act);
-        else stage_broadcast<false>(P, act);
+        if (a.aligned) {
+            // the unit table is no longer needed: its three arrays are the tile buffers
+            stage_broadcast_bulk(P, act, reinterpret_cast<float*>(t_start), reinterpret_cast<float*>(t_c),
+                                 reinterpret_cast<float*>(t_cb), sh_mbar, &sh_abort);
+        } else {
+            stage_broadcast<false>(P, act);
+        }
     }
 #undef QS_BARRIER
     // the last block to leave resets the barrier for the next launch
