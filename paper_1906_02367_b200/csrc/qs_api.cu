@@ -275,20 +275,10 @@ uint64_t take_round(qs_ctx* c, uint64_t round) {
     return round;
 }
 
-int clear_wire(qs_ctx* c, const Active& act, uint32_t* wire, int64_t stride) {
-    if (act.n == c->P.R) {
-        QS_CUDA_TRY(c, cudaMemset2DAsync(wire, (size_t)stride * 4, 0, (size_t)c->wire_words * 4, (size_t)act.n, c->st));
-    } else {
-        for (int w = 0; w < act.n; ++w)
-            QS_CUDA_TRY(c, cudaMemsetAsync(wire + (size_t)act.r[w] * stride, 0, (size_t)c->wire_words * 4, c->st));
-    }
-    return QS_OK;
-}
-
 int run_mid(qs_ctx* c, const Active& act, int do_compress, int do_pack, int do_decode, int do_broadcast,
             uint32_t* wire, int64_t stride, int64_t* bits_out) {
     const cudaError_t e = launch_mid(c->P, act, do_compress, do_pack, do_decode, 0, do_broadcast, c->aligned ? 1 : 0,
-                                     wire, stride, (long long*)bits_out, c->mid_grid, c->st);
+                                     wire, stride, (long long)c->wire_words, (long long*)bits_out, c->mid_grid, c->st);
     if (e != cudaSuccess) return cuda_fail(c, e, "persistent kernel");
     return after_launch(c, 1, "persistent kernel");
 }
@@ -310,7 +300,6 @@ int round_body(qs_ctx* c, uint64_t round, const Active& act, bool fused, uint32_
     if ((rc = after_launch(c, 1, "pass_a")) != QS_OK) return rc;
     if (fused) {
         mark(c, 1);
-        if ((rc = clear_wire(c, act, wire, stride)) != QS_OK) return rc;
     }
     rc = run_mid(c, act, 1, fused, fused, fused, wire, stride, bits_out);
     if (fused) {
@@ -406,8 +395,6 @@ int qs_pack(qs_ctx* c, uint32_t* wire, int64_t stride_words, int64_t* bits_out) 
     if (!c->compressed) return fail(c, QS_STATE, "nothing compressed yet");
     if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
     if (c->last.n == 0) return QS_OK;
-    const int rc = clear_wire(c, c->last, wire, stride_words);
-    if (rc != QS_OK) return rc;
     return run_mid(c, c->last, 0, 1, 0, 0, wire, stride_words, bits_out);
 }
 

@@ -15,8 +15,8 @@ cudaError_t launch_pass_a_tma(const Plan& P, const Active& act, int sms, cudaStr
 // qs_mid.cu: the persistent kernel that runs every stage after the dense pass
 int mid_blocks_per_sm(bool randk);
 cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode, int patch,
-                       int do_broadcast, int aligned, uint32_t* wire, long long stride, long long* bits_out, int grid,
-                       cudaStream_t st);
+                       int do_broadcast, int aligned, uint32_t* wire, long long stride, long long wire_words,
+                       long long* bits_out, int grid, cudaStream_t st);
 void launch_export(const Plan& P, long long* sel_idx, int* level, uint8_t* sign, float* norm, long long* n,
                    int sms, cudaStream_t st);
 

@@ -33,7 +33,7 @@ struct MidArgs {
     Active act;
     int do_compress, do_pack, do_decode, patch, do_broadcast, aligned;
     uint32_t* wire;
-    long long stride;
+    long long stride, wire_words;
     long long* bits_out;
 };
 
@@ -1236,6 +1236,13 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     }
 #define QS_BARRIER() do { if (!grid_barrier(P, target, &sh_abort)) return; } while (0)
 
+    if (a.do_pack) {
+        // the records are built with OR: start from zero words (a later barrier precedes their use)
+        for (int w = 0; w < act.n; ++w) {
+            uint32_t* row = a.wire + (size_t)act.r[w] * a.stride;
+            for (long long i = (long long)blockIdx.x * BT + threadIdx.x; i < a.wire_words; i += (long long)gridDim.x * BT) row[i] = 0u;
+        }
+    }
     Tab tab;
     const bool fused = a.do_compress && a.do_pack && a.do_decode;   // whole round: the master update rides along
     if (a.do_compress) {
@@ -1284,6 +1291,7 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
         }
     } else if (a.do_pack) {
         build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
+        QS_BARRIER();                              // the zeroed records
     }
     if (a.do_pack) {
         if (!tab.fast) stage_pack_dir(P, act, a.wire, a.stride, a.bits_out);
@@ -1352,13 +1360,13 @@ int mid_blocks_per_sm(bool randk) {
 }
 
 cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode, int patch,
-                       int do_broadcast, int aligned, uint32_t* wire, long long stride, long long* bits_out, int grid,
-                       cudaStream_t st) {
+                       int do_broadcast, int aligned, uint32_t* wire, long long stride, long long wire_words,
+                       long long* bits_out, int grid, cudaStream_t st) {
     MidArgs a;
     a.P = P; a.act = act;
     a.do_compress = do_compress; a.do_pack = do_pack; a.do_decode = do_decode; a.patch = patch;
     a.do_broadcast = do_broadcast; a.aligned = aligned;
-    a.wire = wire; a.stride = stride; a.bits_out = bits_out;
+    a.wire = wire; a.stride = stride; a.wire_words = wire_words; a.bits_out = bits_out;
     void* params[] = {&a};
     const void* fn = P.sp == QS_RANDK ? (const void*)mid_kernel<true> : (const void*)mid_kernel<false>;
     return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(BT), params, 0, st);
