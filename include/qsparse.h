@@ -70,6 +70,10 @@ enum {
 #define QS_QSGD 0
 #define QS_QSGD_SCALED 1
 #define QS_SIGN_L1 2
+/* No quantizer: the sparsifier alone (a compression operator with gamma = k/d, Section 2.2; the
+ * Top_k-SGD scheme the paper compares with).  g = u on the kept set; the record carries the
+ * kept values as 32-bit words in place of the sign and level streams, all k of them. */
+#define QS_NONE 3
 /* op argument of qs_init */
 #define QS_OP(sparsifier, quantizer) ((sparsifier) | ((quantizer) << 4))
 

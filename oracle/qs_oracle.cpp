@@ -38,6 +38,10 @@
 //             in fp64; Sign (Lemma 3, m = 1): g = N1/k.  The sign is applied
 //             last by negation; Sign(0) = +1 (Definition 2), so the sign bit is
 //             (u < 0), not the IEEE sign bit.
+//   [none]    quantizer 3 sends the kept values themselves (the sparsifier alone, a compression
+//             operator with gamma = k/d, Section 2.2; the Top_k-SGD scheme of the comparisons):
+//             g = u on the kept set, so the memory becomes 0 there; the record carries 32-bit
+//             values instead of signs and levels, and all k entries.
 //   [pieces]  Corollary 1: each segment has its own k, norm, beta.
 //   [master]  acc = 0; acc += g_r in worker order; x = x - acc/R; indices no
 //             worker sent are left untouched.
@@ -73,7 +77,7 @@
 namespace {
 
 enum { SP_TOPK = 0, SP_RANDK = 1 };
-enum { QZ_QSGD = 0, QZ_QSGD_SCALED = 1, QZ_SIGN_L1 = 2 };
+enum { QZ_QSGD = 0, QZ_QSGD_SCALED = 1, QZ_SIGN_L1 = 2, QZ_NONE = 3 };
 enum { ERR_OK = 0, ERR_ARG = -1, ERR_CAPACITY = -4, ERR_NONFINITE = -5 };
 
 // ---------------------------------------------------------------- Philox
@@ -278,8 +282,14 @@ uint32_t get_bits(const uint32_t* w, int64_t bitpos, int width) {
     return v;
 }
 
-int64_t payload_words(int64_t n, int bi, int bl, int has_levels) {
-    return words_for(n, bi) + words_for(n, 1) + (has_levels ? words_for(n, bl) : 0);
+// words of the streams of a segment that sends n entries, and bits per entry
+int64_t payload_words(int64_t n, int bi, int bl, int quantizer) {
+    if (quantizer == QZ_NONE) return words_for(n, bi) + n;                 // indices, then 32-bit values
+    return words_for(n, bi) + words_for(n, 1) + (quantizer != QZ_SIGN_L1 ? words_for(n, bl) : 0);
+}
+int entry_bits(int bi, int bl, int quantizer) {
+    if (quantizer == QZ_NONE) return bi + 32;
+    return bi + 1 + (quantizer != QZ_SIGN_L1 ? bl : 0);
 }
 
 struct Plan {
@@ -289,9 +299,8 @@ struct Plan {
 
 int64_t wire_words(const Plan& P) {
     int64_t w = 2 * (int64_t)P.nseg;
-    int has_levels = P.quantizer != QZ_SIGN_L1;
     for (int g = 0; g < P.nseg; ++g)
-        w += payload_words(P.kseg[g], bits_idx(P.off[g + 1] - P.off[g]), bits_lvl(P.s), has_levels);
+        w += payload_words(P.kseg[g], bits_idx(P.off[g + 1] - P.off[g]), bits_lvl(P.s), P.quantizer);
     return w;
 }
 
@@ -309,7 +318,8 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
         u[i] = mem[i] + diff;
         if (!std::isfinite(u[i])) return ERR_NONFINITE;
     }
-    const int has_levels = P.quantizer != QZ_SIGN_L1;
+    const int has_levels = P.quantizer == QZ_QSGD || P.quantizer == QZ_QSGD_SCALED;
+    const int plain = P.quantizer == QZ_NONE;   // sparsifier alone: the kept values travel as they are
     const int bl = bits_lvl(P.s);
     int64_t payload = 2 * (int64_t)P.nseg;  // word offset of the next segment's streams
     int64_t bits = 0, selpos = 0;
@@ -321,9 +331,9 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
         else select_randk(P.seed, round, (uint32_t)r, lo, n_el, k, mode, idx.data());
         std::vector<float> kept(k);
         for (int64_t j = 0; j < k; ++j) kept[j] = u[lo + idx[j]];
-        const float N = has_levels ? norm_l2_exact(kept.data(), k) : norm_l1_exact(kept.data(), k);
+        const float N = plain ? 0.0f : has_levels ? norm_l2_exact(kept.data(), k) : norm_l1_exact(kept.data(), k);
         const float c = (float)(1.0 / (1.0 + beta_qsgd(k, P.s)));
-        std::vector<int64_t> s_idx; std::vector<int> s_lvl, s_neg;
+        std::vector<int64_t> s_idx; std::vector<int> s_lvl, s_neg; std::vector<float> s_val;
         for (int64_t j = 0; j < k; ++j) {
             const int64_t gi = lo + idx[j];
             const float v = u[gi];
@@ -333,6 +343,9 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
                 level = qsgd_level(v, N, P.s, philox_word(P.seed, round, (uint32_t)r, (uint64_t)gi, 0u));
                 gval = value_qsgd(N, level, P.s, P.quantizer == QZ_QSGD_SCALED, c, neg);
                 if (level == 0) gval = 0.0f;
+            } else if (plain) {
+                level = 1;
+                gval = v;
             } else {
                 level = 1;
                 gval = value_sign(N, k, neg);
@@ -341,7 +354,7 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
             if (sel_out) sel_out[selpos + j] = gi;
             if (lvl_out) lvl_out[selpos + j] = level;
             if (sgn_out) sgn_out[selpos + j] = (uint8_t)neg;
-            if (level != 0) { s_idx.push_back(idx[j]); s_lvl.push_back(level); s_neg.push_back(neg); }
+            if (level != 0) { s_idx.push_back(idx[j]); s_lvl.push_back(level); s_neg.push_back(neg); s_val.push_back(v); }
         }
         // coordinates outside the kept set: C(u) = 0 there, so m <- u
         {
@@ -360,11 +373,15 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
         uint32_t* w_lvl = w_sgn + words_for(n, 1);
         for (int64_t j = 0; j < n; ++j) {
             put_bits(w_idx, j * bi, bi, (uint32_t)s_idx[j]);
-            put_bits(w_sgn, j, 1, (uint32_t)s_neg[j]);
-            if (has_levels) put_bits(w_lvl, j * bl, bl, (uint32_t)(s_lvl[j] - 1));
+            if (plain) {
+                std::memcpy(&w_sgn[j], &s_val[j], 4);          // the value stream follows the indices
+            } else {
+                put_bits(w_sgn, j, 1, (uint32_t)s_neg[j]);
+                if (has_levels) put_bits(w_lvl, j * bl, bl, (uint32_t)(s_lvl[j] - 1));
+            }
         }
-        payload += payload_words(n, bi, bl, has_levels);
-        bits += 64 + n * (bi + 1 + (has_levels ? bl : 0));
+        payload += payload_words(n, bi, bl, P.quantizer);
+        bits += 64 + n * entry_bits(bi, bl, P.quantizer);
         if (norm_out) norm_out[g] = N;
         if (n_out) n_out[g] = n;
     }
@@ -375,7 +392,8 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
 // ---------------------------------------------------------------- master side
 // Decodes one worker's record from its wire words and adds it into acc.
 void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
-    const int has_levels = P.quantizer != QZ_SIGN_L1;
+    const int has_levels = P.quantizer == QZ_QSGD || P.quantizer == QZ_QSGD_SCALED;
+    const int plain = P.quantizer == QZ_NONE;
     const int bl = bits_lvl(P.s);
     int64_t payload = 2 * (int64_t)P.nseg;
     for (int g = 0; g < P.nseg; ++g) {
@@ -389,9 +407,11 @@ void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
         const uint32_t* w_lvl = w_sgn + words_for(n, 1);
         for (int64_t j = 0; j < n; ++j) {
             const int64_t i = lo + (int64_t)get_bits(w_idx, j * bi, bi);
-            const int neg = (int)get_bits(w_sgn, j, 1);
+            const int neg = plain ? 0 : (int)get_bits(w_sgn, j, 1);
             float gval;
-            if (has_levels) {
+            if (plain) {
+                std::memcpy(&gval, &w_sgn[j], 4);
+            } else if (has_levels) {
                 const int level = (int)get_bits(w_lvl, j * bl, bl) + 1;
                 gval = value_qsgd(N, level, P.s, P.quantizer == QZ_QSGD_SCALED, c, neg);
             } else {
@@ -399,7 +419,7 @@ void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
             }
             acc[i] = acc[i] + gval;
         }
-        payload += payload_words(n, bi, bl, has_levels);
+        payload += payload_words(n, bi, bl, P.quantizer);
     }
 }
 

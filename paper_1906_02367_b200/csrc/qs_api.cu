@@ -167,7 +167,6 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     std::vector<float> h_c(nseg);
     std::vector<uint8_t> h_bi(nseg);
     std::vector<FbBlock> h_fb;
-    const bool has_lvl = P.qz != QS_SIGN_L1;
     int64_t words = 2 * (int64_t)nseg;
     for (int g = 0; g < nseg; ++g) {
         const uint64_t n = (uint64_t)(offsets[g + 1] - offsets[g]), k = (uint64_t)kseg[g];
@@ -178,7 +177,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
         const double a = (double)k / ((double)P.s * (double)P.s), b = std::sqrt((double)k) / (double)P.s;
         h_c[g] = (float)(1.0 / (1.0 + (a < b ? a : b)));
         h_bi[g] = (uint8_t)std::max(1, ceil_log2(n));
-        words += words_for((uint32_t)k, h_bi[g]) + words_for((uint32_t)k, 1) + (has_lvl ? words_for((uint32_t)k, P.bl) : 0);
+        words += streams_words((uint32_t)k, h_bi[g], (uint32_t)P.bl, P.qz);
         for (uint64_t s0 = 0; s0 < n; s0 += FB_CHUNK)
             h_fb.push_back(FbBlock{(uint32_t)g, (uint32_t)(offsets[g] + s0), (uint32_t)std::min<uint64_t>(FB_CHUNK, n - s0)});
     }
@@ -324,7 +323,7 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     *out = nullptr;
     const int sp = op & 15, qz = op >> 4;
     if (R < 1 || R > MAX_R || d < 1 || d >= (1ll << 32) || k < 1 || k > d || s < 1 || s > 65535) return QS_INVALID_ARG;
-    if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1)) return QS_INVALID_ARG;
+    if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1 && qz != QS_NONE)) return QS_INVALID_ARG;
     qs_ctx* c = new qs_ctx();
     std::memset(&c->P, 0, sizeof(Plan));
     c->st = static_cast<cudaStream_t>(cuda_stream);
@@ -459,11 +458,10 @@ int64_t qs_wire_words(const qs_ctx* c) { return c ? c->wire_words : (int64_t)QS_
 
 int64_t qs_record_bits(const qs_ctx* c, const int64_t* n) {
     if (!c || !n) return QS_INVALID_ARG;
-    const bool has_lvl = c->P.qz != QS_SIGN_L1;
     int64_t bits = 0;
     for (int g = 0; g < c->P.nseg; ++g) {
         const int bi = std::max(1, ceil_log2((uint64_t)(c->off[g + 1] - c->off[g])));
-        bits += 64 + n[g] * (bi + 1 + (has_lvl ? c->P.bl : 0));
+        bits += 64 + n[g] * (int64_t)entry_bits((uint32_t)bi, (uint32_t)c->P.bl, c->P.qz);
     }
     return bits;
 }

@@ -220,6 +220,16 @@ __host__ __device__ __forceinline__ uint32_t words_for(uint32_t nfields, uint32_
     return (uint32_t)(((uint64_t)nfields * width + 31u) >> 5);
 }
 
+// words of the streams of a segment that sends n entries, and bits per entry
+__host__ __device__ __forceinline__ uint32_t streams_words(uint32_t n, uint32_t bi, uint32_t bl, int qz) {
+    if (qz == QS_NONE) return words_for(n, bi) + n;                     // indices, then 32-bit values
+    return words_for(n, bi) + words_for(n, 1) + (qz != QS_SIGN_L1 ? words_for(n, bl) : 0u);
+}
+__host__ __device__ __forceinline__ uint32_t entry_bits(uint32_t bi, uint32_t bl, int qz) {
+    if (qz == QS_NONE) return bi + 32u;
+    return bi + 1u + (qz != QS_SIGN_L1 ? bl : 0u);
+}
+
 // fp32 level of the QSGD quantizer and the value it stands for
 __device__ __forceinline__ int qsgd_level(float u, float N, int s, uint32_t w) {
     if (N == 0.0f) return 0;

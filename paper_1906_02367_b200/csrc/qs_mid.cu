@@ -623,6 +623,7 @@ template <bool RANDK>
 __device__ void stage_norm_accum(const Plan& P, const Tab& tab, unsigned long long (*acc)[2], uint32_t* sh_u) {
     const int lane = threadIdx.x & 31;
     const uint32_t total = tab.total_chunks;
+    if (P.qz == QS_NONE) return;                   // the plain sparsifier sends the values: no norm
     const bool l1 = P.qz == QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
@@ -754,7 +755,7 @@ template <bool RANDK>
 __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_chunks;
-    const bool sign_op = P.qz == QS_SIGN_L1;
+    const bool sign_op = P.qz == QS_SIGN_L1, plain = P.qz == QS_NONE;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
         const float N = c.un.norm, cs = P.cscale[c.seg];
@@ -779,11 +780,11 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t*
             if (is_kept<RANDK>(c.un, key[i], idx[i])) {
                 const bool neg = val[i] < 0.0f;
                 int level = 1;
-                if (!sign_op) level = qsgd_level(val[i], N, P.s, philox_word(P, c.r, idx[i], 0u));
+                if (!sign_op && !plain) level = qsgd_level(val[i], N, P.s, philox_word(P, c.r, idx[i], 0u));
                 q = Q_SEL | (neg ? Q_NEG : 0u) | (uint32_t)level;
                 cnt += 1u;
                 if (level) {
-                    mem[idx[i]] = val[i] - coord_value(P, N, level, neg, cs, k);
+                    mem[idx[i]] = val[i] - (plain ? val[i] : coord_value(P, N, level, neg, cs, k));
                     cnt += 1u << 16;
                     if (fused) atomicOr(&P.touch[idx[i]], 1u << c.r);     // the master's "who sent this index"
                 }
@@ -826,7 +827,6 @@ __device__ void stage_chunk_scan(const Plan& P, const Tab& tab, const Active& ac
         if (kept != P.kseg[u % P.nseg]) set_status(P, QS_STATE);
     }
     __syncthreads();
-    const bool has_lvl = P.qz != QS_SIGN_L1;
     for (int w = 0; w < act.n; ++w) {
         const int r = act.r[w];
         uint32_t carry = 2u * P.nseg;
@@ -837,8 +837,8 @@ __device__ void stage_chunk_scan(const Plan& P, const Tab& tab, const Active& ac
             if (g < (uint32_t)P.nseg) {
                 n = P.units[(size_t)r * P.nseg + g].n;
                 bi = P.bidx[g];
-                words = words_for(n, bi) + words_for(n, 1) + (has_lvl ? words_for(n, P.bl) : 0u);
-                bits += 64 + (long long)n * (bi + 1 + (has_lvl ? P.bl : 0));
+                words = streams_words(n, bi, (uint32_t)P.bl, P.qz);
+                bits += 64 + (long long)n * entry_bits(bi, (uint32_t)P.bl, P.qz);
             }
             uint32_t total;
             const uint32_t ex = block_excl_scan(words, sh, &total);
@@ -891,7 +891,7 @@ __device__ void stage_pack_dir(const Plan& P, const Active& act, uint32_t* wire,
 // streams of every segment, and the ordered kept list kept for inspection
 __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
     const uint32_t total = tab.total_chunks;
-    const bool has_lvl = P.qz != QS_SIGN_L1;
+    const bool plain = P.qz == QS_NONE, has_lvl = P.qz != QS_SIGN_L1 && !plain;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
         uint32_t run_k, run_s, unit_n, pay;
@@ -915,7 +915,7 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* 
                 uint32_t* row = wire + (size_t)c.r * stride;
                 row[0] = unit_n;
                 row[1] = __float_as_uint(c.un.norm);
-                const long long bits = 64 + (long long)unit_n * (bi + 1 + (has_lvl ? P.bl : 0));
+                const long long bits = 64 + (long long)unit_n * entry_bits(bi, (uint32_t)P.bl, P.qz);
                 P.bits[c.r] = bits;
                 if (bits_out) bits_out[c.r] = bits;
             }
@@ -949,8 +949,12 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* 
                 if (sent && run_s + (ex >> 16) < unit_n) {
                     const uint64_t js = run_s + (ex >> 16);
                     or_bits(w_idx, js * bi, bi, e[i] - lo);
-                    if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
-                    if (has_lvl) or_bits(w_lvl, js * P.bl, P.bl, (q[i] & 0xffffu) - 1u);
+                    if (plain) {
+                        w_sgn[js] = __float_as_uint(P.cand_val[c.base + c.first + i * BT + threadIdx.x]);   // value stream
+                    } else {
+                        if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
+                        if (has_lvl) or_bits(w_lvl, js * P.bl, P.bl, (q[i] & 0xffffu) - 1u);
+                    }
                     sent_mask |= 1u << i;
                 }
             }
@@ -972,8 +976,9 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* 
 #pragma unroll
             for (int i = 0; i < PER; ++i) {
                 if (!senders[i]) continue;
-                const float g = coord_value(P, c.un.norm, (int)(q[i] & 0xffffu), (q[i] & Q_NEG) != 0, P.cscale[c.seg],
-                                            P.kseg[c.seg]);
+                const float g = plain ? P.cand_val[c.base + c.first + i * BT + threadIdx.x]
+                                      : coord_value(P, c.un.norm, (int)(q[i] & 0xffffu), (q[i] & Q_NEG) != 0,
+                                                    P.cscale[c.seg], P.kseg[c.seg]);
                 if (senders[i] == (1u << c.r)) {
                     float acc = 0.0f;
                     acc = acc + g;
@@ -991,7 +996,6 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* 
 // ------------------------------------------------------------------ master
 // entry and stream offsets of each segment, read from the directory
 __device__ void stage_dec_prep(const Plan& P, const Active& act, const uint32_t* wire, long long stride, uint32_t* sh) {
-    const bool has_lvl = P.qz != QS_SIGN_L1;
     for (int w = blockIdx.x; w < act.n; w += gridDim.x) {
         const int r = act.r[w];
         const uint32_t* row = wire + (size_t)r * stride;
@@ -1002,7 +1006,7 @@ __device__ void stage_dec_prep(const Plan& P, const Active& act, const uint32_t*
             if (g < (uint32_t)P.nseg) {
                 n = row[2 * g];
                 if (n > P.kseg[g]) { n = 0; set_status(P, QS_INVALID_ARG); }     // not a record of this plan
-                words = words_for(n, P.bidx[g]) + words_for(n, 1) + (has_lvl ? words_for(n, P.bl) : 0u);
+                words = streams_words(n, P.bidx[g], (uint32_t)P.bl, P.qz);
             }
             uint32_t te, tw;
             const uint32_t ee = block_excl_scan(n, sh, &te);
@@ -1064,6 +1068,7 @@ __device__ __forceinline__ float entry_value(const Plan& P, const uint32_t* row,
     const uint32_t* w_sgn = en.w_idx + words_for(en.n, bi);
     const uint32_t* w_lvl = w_sgn + words_for(en.n, 1);
     const bool neg = (w_sgn[en.j >> 5] >> (en.j & 31u)) & 1u;
+    if (P.qz == QS_NONE) return __uint_as_float(w_sgn[en.j]);       // the value stream sits where the signs would
     const int level = P.qz == QS_SIGN_L1 ? 1 : (int)get_bits(w_lvl, (uint64_t)en.j * P.bl, P.bl) + 1;
     return coord_value(P, __uint_as_float(row[2 * en.seg + 1]), level, neg, P.cscale[en.seg], P.kseg[en.seg]);
 }

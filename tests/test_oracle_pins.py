@@ -557,3 +557,45 @@ def test_single_worker_entry_equals_the_batch_entry():
         one = O.compress_worker(plan, 5, r, x, xw[r].copy(), mr)
         assert one["rc"] == 0 and np.array_equal(one["wire"], out["wire"][r])
         assert np.array_equal(mr, m2[r]) and one["bits"] == out["bits"][r]
+
+
+# ----------------------------------------------------------------------------- sparsifier alone
+def test_plain_sparsifier_is_topk_itself():
+    # quantizer NONE: C(u) = Top_k(u) (Section 2.2), memory 0 on the kept set, gamma = k/d holds surely
+    R, d, k = 3, 900, 37
+    x, xw, mem = I.gaussian_round(R, d, seed=33)
+    plan = O.Plan(R, d, k=k, quantizer=O.NONE)
+    out, u, mem2 = run_details(plan, 2, x, xw, mem)
+    bi = clog2(d)
+    assert plan.wire_words() == 2 + -(-k * bi // 32) + k
+    acc = np.zeros(d, np.float64)
+    for r in range(R):
+        sel = brute_topk(u[r], k)
+        assert list(out["sel"][r]) == sel and out["n"][r, 0] == k
+        words = out["wire"][r]
+        assert int(words[0]) == k and int(words[1]) == 0
+        idx = [read_bits(words[2:], j * bi, bi) for j in range(k)]
+        vals = words[2 + -(-k * bi // 32): 2 + -(-k * bi // 32) + k].view(np.float32)
+        assert idx == sel and np.array_equal(vals.view(np.uint32), u[r, sel].view(np.uint32))
+        assert out["bits"][r] == 64 + k * (bi + 32)
+        want = u[r].copy()
+        want[sel] = 0.0
+        assert np.array_equal(mem2[r].view(np.uint32), want.view(np.uint32))
+        lhs = float((mem2[r].astype(np.float64) ** 2).sum())
+        assert lhs <= (1 - k / d) * float((u[r].astype(np.float64) ** 2).sum())
+        acc[sel] += u[r, sel].astype(np.float64)
+    x2 = x.copy()
+    assert O.unpack_accumulate(plan, x2, out["wire"]) == 0
+    assert np.allclose(x2, x - acc / R, rtol=1e-6, atol=1e-7)
+
+
+def test_plain_randk_contracts_in_expectation():
+    # E||u - Rand_k(u)||^2 = (1 - k/d) ||u||^2 (Section 2.2 with the proof of Lemma 8)
+    d, k, T = 60, 15, 3000
+    x, xw, mem = I.gaussian_round(1, d, seed=35)
+    plan = O.Plan(1, d, k=k, sparsifier=O.RANDK, quantizer=O.NONE, seed=3)
+    ratio = 0.0
+    for t in range(T):
+        out, u, mem2 = run_details(plan, t, x, xw, mem)
+        ratio += float((mem2[0].astype(np.float64) ** 2).sum() / (u[0].astype(np.float64) ** 2).sum()) / T
+    assert abs(ratio - (1 - k / d)) < 0.01
