@@ -29,21 +29,23 @@ constexpr int STAGES = QS_TMA_STAGES;      // (xw, mem) tile pairs in the ring
 #endif
 constexpr int XSLOTS = QS_TMA_XSLOTS;      // x tiles in their ring
 
+template <bool ANCH>
 struct TmaSmem {
-    float stage[STAGES][2][TILE];          // [0] xw tile, [1] mem tile (overwritten with u)
-    float xs[XSLOTS][TILE];
+    float stage[STAGES][ANCH ? 3 : 2][TILE];   // [0] xw tile, [1] mem tile (overwritten with u), [2] anchor tile
+    float xs[ANCH ? 1 : XSLOTS][ANCH ? 4 : TILE];   // x tiles (not read when every worker has its own anchor)
     uint64_t full[STAGES];
     uint64_t xfull[XSLOTS];
     uint32_t cnt[2][8 * GPW];              // candidates per group of the current tile (double-buffered)
     int abort_flag;
 };
 
-// Synchronous algorithm only (every worker's reference point is x); rows 16-byte aligned.
-template <bool RANDK>
+// Rows 16-byte aligned.  ANCH: Algorithm 2, worker r's reference point is anchors_r (a third tile per
+// item) instead of x.
+template <bool RANDK, bool ANCH>
 __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Active act, const int prefetch) {
     extern __shared__ __align__(128) unsigned char sh_raw[];
-    TmaSmem& S = *reinterpret_cast<TmaSmem*>(sh_raw);
-    uint32_t* tab = reinterpret_cast<uint32_t*>(sh_raw + sizeof(TmaSmem));
+    TmaSmem<ANCH>& S = *reinterpret_cast<TmaSmem<ANCH>*>(sh_raw);
+    uint32_t* tab = reinterpret_cast<uint32_t*>(sh_raw + sizeof(TmaSmem<ANCH>));
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ntiles = (P.d + TILE - 1) / TILE;
     const int nact = act.n;
@@ -72,14 +74,15 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
         const uint32_t bytes = (P.d - e0 < TILE ? P.d - e0 : TILE) * 4u;
         const int s = (int)(j % STAGES);
         const size_t row = (size_t)act.r[w] * P.d + e0;
-        if (w == 0) {
+        if (!ANCH && w == 0) {
             const int xsl = (int)(it % XSLOTS);
             mbar_expect(&S.xfull[xsl], bytes);
             bulk_load(S.xs[xsl], P.x + e0, bytes, &S.xfull[xsl]);
         }
-        mbar_expect(&S.full[s], 2u * bytes);
+        mbar_expect(&S.full[s], (ANCH ? 3u : 2u) * bytes);
         bulk_load(S.stage[s][0], P.xw + row, bytes, &S.full[s]);
         bulk_load(S.stage[s][1], P.mem + row, bytes, &S.full[s]);
+        if (ANCH) bulk_load(S.stage[s][ANCH ? 2 : 0], P.anchors + row, bytes, &S.full[s]);
     };
 
     if (threadIdx.x == 0)
@@ -99,7 +102,7 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
             issue(j + prefetch);
         }
         bool ok = mbar_wait(&S.full[s], (uint32_t)((j / STAGES) & 1));
-        if (w == 0) ok = ok && mbar_wait(&S.xfull[xsl], (uint32_t)((it / XSLOTS) & 1));
+        if (!ANCH && w == 0) ok = ok && mbar_wait(&S.xfull[xsl], (uint32_t)((it / XSLOTS) & 1));
         if (!ok) S.abort_flag = 1;           // seen by everyone at the barrier below
 
         const uint32_t* gs = tab + (size_t)r * P.nseg;
@@ -118,7 +121,8 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
                     sg[k][jj] = sq;
                 }
             }
-            const float4 xq = *reinterpret_cast<const float4*>(&S.xs[xsl][q]);
+            const float4 xq = ANCH ? *reinterpret_cast<const float4*>(&S.stage[s][ANCH ? 2 : 0][q])
+                                   : *reinterpret_cast<const float4*>(&S.xs[ANCH ? 0 : xsl][ANCH ? 0 : q]);
             const float4 wq = *reinterpret_cast<const float4*>(&S.stage[s][0][q]);
             const float4 mq = *reinterpret_cast<const float4*>(&S.stage[s][1][q]);
             uu[k][0] = mq.x + (xq.x - wq.x);
@@ -165,26 +169,36 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
     if (bad) set_status(P, QS_NONFINITE);
 }
 
-size_t pass_a_tma_smem(const Plan& P) { return sizeof(TmaSmem) + ((size_t)P.R * P.nseg + P.nseg + 1) * 4; }
+size_t pass_a_tma_smem(const Plan& P) {
+    return (P.anchors ? sizeof(TmaSmem<true>) : sizeof(TmaSmem<false>)) + ((size_t)P.R * P.nseg + P.nseg + 1) * 4;
+}
 
-bool pass_a_tma_usable(const Plan& P, bool aligned) {
-    return aligned && !P.anchors && pass_a_tma_smem(P) <= 100 * 1024;
+bool pass_a_tma_usable(const Plan& P, bool aligned) { return aligned && pass_a_tma_smem(P) <= 100 * 1024; }
+
+template <bool RANDK, bool ANCH>
+static cudaError_t tma_launch(const Plan& P, const Active& act, int sms, size_t smem, int prefetch, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(pass_a_tma_kernel<RANDK, ANCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    // tiles are dealt to blocks by stride, so the grid holds only blocks that are resident together
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pass_a_tma_kernel<RANDK, ANCH>, 256, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorInvalidConfiguration;
+    if (per_sm > QS_TMA_PER_SM) per_sm = QS_TMA_PER_SM;
+    const uint32_t ntiles = (P.d + TILE - 1) / TILE;
+    const uint32_t cap = (uint32_t)sms * (uint32_t)per_sm;
+    const int grid = (int)(ntiles < cap ? ntiles : cap);
+    pass_a_tma_kernel<RANDK, ANCH><<<grid, 256, smem, st>>>(P, act, prefetch);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_pass_a_tma(const Plan& P, const Active& act, int sms, cudaStream_t st) {
     const size_t smem = pass_a_tma_smem(P);
-    const bool rk = P.sp == QS_RANDK;
-    cudaError_t e = rk ? cudaFuncSetAttribute(pass_a_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                       : cudaFuncSetAttribute(pass_a_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    const uint32_t ntiles = (P.d + TILE - 1) / TILE;
-    const uint32_t cap = (uint32_t)sms * (uint32_t)QS_TMA_PER_SM;
-    const int grid = (int)(ntiles < cap ? ntiles : cap);
     int prefetch = STAGES - 2;
-    if (prefetch > (XSLOTS - 1) * act.n) prefetch = (XSLOTS - 1) * act.n;   // an x slot is refilled only after its tile is done
-    if (rk) pass_a_tma_kernel<true><<<grid, 256, smem, st>>>(P, act, prefetch);
-    else pass_a_tma_kernel<false><<<grid, 256, smem, st>>>(P, act, prefetch);
-    return cudaGetLastError();
+    if (!P.anchors && prefetch > (XSLOTS - 1) * act.n) prefetch = (XSLOTS - 1) * act.n;   // an x slot is refilled only after its tile is done
+    const bool rk = P.sp == QS_RANDK;
+    if (P.anchors) return rk ? tma_launch<true, true>(P, act, sms, smem, prefetch, st) : tma_launch<false, true>(P, act, sms, smem, prefetch, st);
+    return rk ? tma_launch<true, false>(P, act, sms, smem, prefetch, st) : tma_launch<false, false>(P, act, sms, smem, prefetch, st);
 }
 
 }  // namespace qs
