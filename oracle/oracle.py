@@ -118,6 +118,12 @@ def local_step(plan, xw, grad, eta, mask=None):
                          _p(m, C.c_uint8))
 
 
+def local_step_momentum(plan, xw, vel, grad, eta, mu, mask=None):
+    m = _mask(mask)
+    lib().qso_local_step_momentum(C.c_int(plan.R), C.c_int64(plan.d), _f32(xw), _f32(vel), _f32(grad),
+                                  C.c_float(eta), C.c_float(mu), _p(m, C.c_uint8))
+
+
 def compress_feedback(plan, rnd, x, xw, mem, anchors=None, mask=None, mode=SORT, nthreads=1,
                       details=False):
     """Worker half.  Returns dict(wire, bits[, sel, level, sign, norm, n])."""

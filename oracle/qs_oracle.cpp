@@ -43,6 +43,9 @@
 //             g = u on the kept set, so the memory becomes 0 there; the record carries 32-bit
 //             values instead of signs and levels, and all k entries.
 //   [pieces]  Corollary 1: each segment has its own k, norm, beta.
+//   [momentum] Section 5.1 applies momentum 0.9 on the local iterations and prints no
+//             formula: the heavy-ball form v <- mu v + grad, xhat <- xhat - eta v is taken,
+//             every product and sum rounded to fp32 on its own.
 //   [master]  acc = 0; acc += g_r in worker order; x = x - acc/R; indices no
 //             worker sent are left untouched.
 //   [wire]    per worker: a directory of nseg (n, norm bits) word pairs, then
@@ -471,6 +474,25 @@ void qso_local_step(int R, int64_t d, float* xw, const float* grad, float eta,
         for (int64_t i = 0; i < d; ++i) {
             float step = eta * grad[(int64_t)r * d + i];
             xw[(int64_t)r * d + i] = xw[(int64_t)r * d + i] - step;
+        }
+    }
+}
+
+// Local step with momentum (Section 5.1: momentum 0.9 applied on the local
+// iterations; the paper prints no formula, the heavy-ball form is taken):
+//   v_r <- mu * v_r + grad_r ;  xhat_r <- xhat_r - eta * v_r
+// every product and sum rounded to fp32 on its own.  mu = 0 is the plain step.
+void qso_local_step_momentum(int R, int64_t d, float* xw, float* vel, const float* grad,
+                             float eta, float mu, const uint8_t* mask) {
+    for (int r = 0; r < R; ++r) {
+        if (mask && !mask[r]) continue;
+        for (int64_t i = 0; i < d; ++i) {
+            const int64_t p = (int64_t)r * d + i;
+            float carried = mu * vel[p];
+            float v = carried + grad[p];
+            vel[p] = v;
+            float step = eta * v;
+            xw[p] = xw[p] - step;
         }
     }
 }

@@ -599,3 +599,53 @@ def test_plain_randk_contracts_in_expectation():
         out, u, mem2 = run_details(plan, t, x, xw, mem)
         ratio += float((mem2[0].astype(np.float64) ** 2).sum() / (u[0].astype(np.float64) ** 2).sum()) / T
     assert abs(ratio - (1 - k / d)) < 0.01
+
+
+# ---------------------------------------------------------------- momentum on the local iterations (Section 5.1)
+def test_momentum_step_with_mu_zero_is_the_plain_step():
+    R, d = 3, 97
+    g = np.random.default_rng(11)
+    plan = O.Plan(R, d, k=5, s=4)
+    xw = g.standard_normal((R, d)).astype(np.float32)
+    grad = g.standard_normal((R, d)).astype(np.float32)
+    a, b = xw.copy(), xw.copy()
+    vel = g.standard_normal((R, d)).astype(np.float32)      # ignored when mu = 0
+    O.local_step(plan, a, grad, 0.1)
+    O.local_step_momentum(plan, b, vel, grad, 0.1, 0.0)
+    assert np.array_equal(a, b)
+    assert np.array_equal(vel, grad)                        # v <- 0 * v + grad
+
+
+def test_momentum_constant_gradient_closed_form():
+    """Constant gradient c: v_n = c (1 - mu^n) / (1 - mu) and
+    x_n = x_0 - eta c (n - mu (1 - mu^n) / (1 - mu)) / (1 - mu)."""
+    R, d, n, eta, mu = 2, 64, 40, 0.01, 0.9
+    g = np.random.default_rng(12)
+    plan = O.Plan(R, d, k=4, s=4)
+    c = g.standard_normal((R, d)).astype(np.float32)
+    x0 = g.standard_normal((R, d)).astype(np.float32)
+    xw, vel = x0.copy(), np.zeros((R, d), np.float32)
+    for _ in range(n):
+        O.local_step_momentum(plan, xw, vel, c, eta, mu)
+    mu64, eta64, c64 = float(np.float32(mu)), float(np.float32(eta)), c.astype(np.float64)
+    v_n = c64 * (1 - mu64 ** n) / (1 - mu64)
+    x_n = x0.astype(np.float64) - eta64 * c64 * (n - mu64 * (1 - mu64 ** n) / (1 - mu64)) / (1 - mu64)
+    assert np.allclose(vel, v_n, rtol=1e-5, atol=1e-6)
+    assert np.allclose(xw, x_n, rtol=1e-5, atol=1e-5)
+    # a wrong sign or a velocity that is not carried would be far outside these tolerances
+    assert np.abs(xw - x0).max() > 10 * eta64 * np.abs(c64).max()
+
+
+def test_momentum_step_respects_the_mask():
+    R, d = 4, 33
+    g = np.random.default_rng(13)
+    plan = O.Plan(R, d, k=3, s=4)
+    xw = g.standard_normal((R, d)).astype(np.float32)
+    vel = g.standard_normal((R, d)).astype(np.float32)
+    grad = g.standard_normal((R, d)).astype(np.float32)
+    xw0, vel0 = xw.copy(), vel.copy()
+    O.local_step_momentum(plan, xw, vel, grad, 0.1, 0.9, mask=[1, 0, 0, 1])
+    assert np.array_equal(xw[1:3], xw0[1:3]) and np.array_equal(vel[1:3], vel0[1:3])
+    v = (np.float32(0.9) * vel0[0]).astype(np.float32) + grad[0]
+    assert np.array_equal(vel[0], v.astype(np.float32))
+    assert np.array_equal(xw[0], (xw0[0] - (np.float32(0.1) * v).astype(np.float32)).astype(np.float32))
