@@ -444,13 +444,79 @@ def run_async(args):
     ctx.destroy()
 
 
+def run_step(args):
+    """The round with the preceding local step taken inside it (qs_sync_round_step) against the two
+    calls it replaces, plain and with momentum, on the headline workload.  Not the headline line.
+    Bytes the fused form has to move: the round's 16 R d + 8 d plus the gradient read (4 R d), plus
+    the velocity read and written (8 R d) with momentum."""
+    import torch
+    from paper_1906_02367_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    sizes, off, d, seg_off, kseg = workload("flat", args.shrink)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(99)
+    per_elem = torch.from_numpy(np.repeat(I.tensor_scales(len(sizes), seed=0), np.diff(off))).to(dev)
+    x = torch.from_numpy(I.model_init(d, seed=0)).to(dev)
+    xw = x.expand(R, d).contiguous()
+    mem = torch.zeros((R, d), dtype=torch.float32, device=dev)
+    vel = torch.zeros((R, d), dtype=torch.float32, device=dev)
+    grad = torch.empty((R, d), dtype=torch.float32, device=dev)
+    e2 = torch.empty_like(grad)
+    ctx = B.Context(R, d, int(kseg[0]), 1, B.QS_TOPK, B.QS_SIGN_L1, seed=0)
+    ctx.bind(x, xw, mem)
+    wire = ctx.new_wire()
+    bits = torch.zeros(R, dtype=torch.int64, device=dev)
+    peak, peak_src = peak_hbm()
+
+    def new_grad():                    # Laplace(0, b_t) per tensor; eta = 1 makes the step the headline drift
+        grad.exponential_(generator=gen)
+        e2.exponential_(generator=gen)
+        grad.sub_(e2).mul_(per_elem)
+
+    def timed(fn):
+        times = []
+        for i in range(args.warmup + args.steps):
+            new_grad()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                times.append(a.elapsed_time(b))
+        assert ctx.sync_status() == 0, ctx.last_error()
+        return float(np.mean(times))
+
+    out = {}
+    for name, v, mu, extra in (("plain", None, 0.0, 4), ("momentum", vel, 0.5, 12)):
+        def separate():
+            if v is None:
+                ctx.local_step(grad, 1.0)
+            else:
+                ctx.local_step_momentum(grad, v, 1.0, mu)
+            ctx.sync_round(wire, bits_out=bits)
+        ms_sep = timed(separate)
+        vel.zero_()
+        ms_fused = timed(lambda: ctx.sync_round_step(wire, grad, 1.0, vel=v, mu=mu, bits_out=bits))
+        vel.zero_()
+        bmin = (16 + extra) * R * d + 8 * d + 2 * (int(bits.sum().item() + 7) // 8)
+        gbs = bmin / (ms_fused * 1e-3) / 1e9
+        out[name] = {"ms_two_calls": ms_sep, "ms_fused": ms_fused, "min_bytes_fused": bmin, "GBps_fused": gbs,
+                     "pct_of_nominal_8TBps": 100 * gbs / NOMINAL_HBM_GBS, "pct_of_measured_copy": 100 * gbs / peak}
+    print(json.dumps({"metric": "sync_round_with_local_step", "unit": "ms", "steps": args.steps, "warmup": args.warmup,
+                      "config": {"workload": f"ResNet-50-shaped round with its local step: R=8, d={d}, Top_k 0.1% flat, sign/l1"},
+                      "peak_source": peak_src, "variants": out}))
+    ctx.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor", "async"])
+    ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor", "async", "step"])
     ap.add_argument("--shrink", type=int, default=1, help="divide every tensor size (profiling on a small case)")
     ap.add_argument("--sweep5", action="store_true", help="run the d = 2^28 ratio x s sweep instead of the headline workload")
     ap.add_argument("--no-e2e", action="store_true")
@@ -463,6 +529,8 @@ def main():
         run_reference(args)
     elif args.variant == "async":
         run_async(args)
+    elif args.variant == "step":
+        run_step(args)
     else:
         run_ours(args)
 

@@ -125,6 +125,17 @@ int qs_bind(qs_ctx* ctx, float* x, float* xw, float* mem, float* anchors);
 int qs_local_step(qs_ctx* ctx, const float* grad, float eta, const uint8_t* worker_mask);
 
 /*
+ * qs_local_step_momentum — the local step with momentum on the local iterations, as the
+ * experiments of Section 5.1 run it (momentum 0.9; the paper prints no formula, the
+ * heavy-ball form is taken), for the masked workers:
+ *   vel_r <- mu * vel_r + grad_r ;  xw_r <- xw_r - eta * vel_r
+ * every product and sum rounded to fp32 on its own.  grad, vel: device, R x d; vel is
+ * caller-owned and updated in place.  mu = 0 gives qs_local_step (and vel_r = grad_r).
+ */
+int qs_local_step_momentum(qs_ctx* ctx, const float* grad, float* vel, float eta, float mu,
+                           const uint8_t* worker_mask);
+
+/*
  * qs_compress_feedback — worker half of a synchronisation (Alg. 1 lines 9-10; Alg. 2
  * lines 9-10) for the masked workers: forms u, finds the kept set of each segment,
  * computes the norm of the kept k-vector (the quantizer acts on it as a length-k
@@ -178,6 +189,20 @@ int qs_broadcast(qs_ctx* ctx, const uint8_t* worker_mask);
  */
 int qs_sync_round(qs_ctx* ctx, uint64_t round, const uint8_t* worker_mask, uint32_t* wire,
                   int64_t stride_words, int64_t* bits_out);
+
+/*
+ * qs_sync_round_step — the local step that precedes a synchronisation (Alg. 1 line 5; Alg. 2
+ * line 5) taken inside the round: the same final bytes in x, xw, mem, anchors, vel, wire
+ * and bits_out as qs_local_step (vel == NULL) or qs_local_step_momentum (vel != NULL) for
+ * the masked workers followed by qs_sync_round with the same mask.  The half-step model
+ * xw_r - eta * (...) is formed in the dense pass and never written: the broadcast that
+ * ends the round overwrites xw_r anyway, which saves one read and one write of xw_r.
+ * grad (and vel): device, R x d; rows of workers outside the mask are neither read nor
+ * written.  Rows that are not 16-byte aligned take the two calls named above instead.
+ */
+int qs_sync_round_step(qs_ctx* ctx, const float* grad, float* vel, float eta, float mu,
+                       uint64_t round, const uint8_t* worker_mask, uint32_t* wire,
+                       int64_t stride_words, int64_t* bits_out);
 
 /*
  * qs_export_selection — copies the result of the last compression, after it has been packed

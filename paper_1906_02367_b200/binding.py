@@ -21,7 +21,8 @@ QS_QSGD, QS_QSGD_SCALED, QS_SIGN_L1, QS_NONE = 0, 1, 2, 3
 QS_ROUND_AUTO = 2**64 - 1
 
 EXPORTS = [
-    "qs_init", "qs_set_segments", "qs_bind", "qs_local_step", "qs_compress_feedback", "qs_pack",
+    "qs_init", "qs_set_segments", "qs_bind", "qs_local_step", "qs_local_step_momentum", "qs_sync_round_step",
+    "qs_compress_feedback", "qs_pack",
     "qs_unpack_accumulate", "qs_broadcast", "qs_sync_round", "qs_export_selection", "qs_wire_words",
     "qs_record_bits", "qs_total_k", "qs_sync_status", "qs_last_error", "qs_get_round", "qs_set_round",
     "qs_get_stats", "qs_enable_phase_timing", "qs_get_phase_timing", "qs_get_stage_trace", "qs_unpack_accumulate_static",
@@ -48,6 +49,8 @@ def lib():
         L.qs_set_segments.argtypes = [vp, C.c_int, vp, vp]
         L.qs_bind.argtypes = [vp, vp, vp, vp, vp]
         L.qs_local_step.argtypes = [vp, vp, C.c_float, vp]
+        L.qs_local_step_momentum.argtypes = [vp, vp, vp, C.c_float, C.c_float, vp]
+        L.qs_sync_round_step.argtypes = [vp, vp, vp, C.c_float, C.c_float, u64, vp, vp, i64, vp]
         L.qs_compress_feedback.argtypes = [vp, u64, vp]
         L.qs_pack.argtypes = [vp, vp, i64, vp]
         L.qs_unpack_accumulate.argtypes = [vp, vp, i64, vp]
@@ -141,6 +144,20 @@ class Context:
         assert grad.is_cuda and grad.dtype == torch.float32 and grad.is_contiguous()
         m, mp = _mask(mask, self.R)
         self._check(lib().qs_local_step(self._h, _ptr(grad), float(eta), mp))
+
+    def local_step_momentum(self, grad, vel, eta, mu, mask=None):
+        for t in (grad, vel):
+            assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+        m, mp = _mask(mask, self.R)
+        self._check(lib().qs_local_step_momentum(self._h, _ptr(grad), _ptr(vel), float(eta), float(mu), mp))
+
+    def sync_round_step(self, wire, grad, eta, vel=None, mu=0.0, rnd=QS_ROUND_AUTO, mask=None, bits_out=None):
+        """The local step (with momentum when vel is given) taken inside the round."""
+        for t in (grad, vel):
+            assert t is None or (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous())
+        m, mp = _mask(mask, self.R)
+        self._check(lib().qs_sync_round_step(self._h, _ptr(grad), _ptr(vel), float(eta), float(mu), int(rnd), mp,
+                                             _ptr(wire), int(wire.shape[1]), _ptr(bits_out)))
 
     def compress_feedback(self, rnd=QS_ROUND_AUTO, mask=None):
         m, mp = _mask(mask, self.R)

@@ -282,16 +282,30 @@ int run_mid(qs_ctx* c, const Active& act, int do_compress, int do_pack, int do_d
     return after_launch(c, 1, "persistent kernel");
 }
 
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
 // dense pass, then the persistent kernel for the stages asked for
 int round_body(qs_ctx* c, uint64_t round, const Active& act, bool fused, uint32_t* wire, int64_t stride,
-               int64_t* bits_out) {
+               int64_t* bits_out, const StepArgs* step = nullptr) {
     Plan& P = c->P;
     P.round_lo = (uint32_t)round;
     P.round_hi = (uint32_t)(round >> 32);
     int rc;
     if (fused) mark(c, 0);
-    if (c->use_tma && pass_a_tma_usable(P, c->aligned)) {
-        const cudaError_t e = launch_pass_a_tma(P, act, c->sms, c->st);
+    StepArgs sa = {nullptr, nullptr, 0.0f, 0.0f};
+    int kind = 0;                                // local step taken inside the dense pass: 0 none, 1 plain, 2 momentum
+    if (step) {
+        sa = *step;
+        const bool rows16 = c->aligned && aligned16(sa.grad) && aligned16(sa.vel);
+        if (c->use_tma && rows16 && pass_a_tma_usable(P, true, sa.vel ? 2 : 1)) {
+            kind = sa.vel ? 2 : 1;
+        } else {                                 // the step as a launch of its own, then the plain dense pass
+            launch_local_step(P, act, sa, rows16, c->sms, c->st);
+            if ((rc = after_launch(c, 1, "local_step")) != QS_OK) return rc;
+        }
+    }
+    if (c->use_tma && pass_a_tma_usable(P, c->aligned, kind)) {
+        const cudaError_t e = launch_pass_a_tma(P, act, sa, kind, c->sms, c->st);
         if (e != cudaSuccess) return cuda_fail(c, e, "pass_a (bulk copy)");
     } else {
         launch_pass_a(P, act, 0, c->aligned, c->sms, c->st);
@@ -311,8 +325,6 @@ int round_body(qs_ctx* c, uint64_t round, const Active& act, bool fused, uint32_
     c->rounds += 1;
     return QS_OK;
 }
-
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
 
@@ -376,7 +388,18 @@ int qs_local_step(qs_ctx* c, const float* grad, float eta, const uint8_t* worker
     if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
-    launch_local_step(c->P, act, grad, eta, c->aligned && aligned16(grad), c->sms, c->st);
+    const StepArgs sa = {grad, nullptr, eta, 0.0f};
+    launch_local_step(c->P, act, sa, c->aligned && aligned16(grad), c->sms, c->st);
+    return after_launch(c, 1, "local_step");
+}
+
+int qs_local_step_momentum(qs_ctx* c, const float* grad, float* vel, float eta, float mu, const uint8_t* worker_mask) {
+    if (!c || !grad || !vel) return fail(c, QS_INVALID_ARG, "grad and vel are required");
+    if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
+    Active act;
+    if (!make_active(c, worker_mask, &act)) return QS_OK;
+    const StepArgs sa = {grad, vel, eta, mu};
+    launch_local_step(c->P, act, sa, c->aligned && aligned16(grad) && aligned16(vel), c->sms, c->st);
     return after_launch(c, 1, "local_step");
 }
 
@@ -424,6 +447,18 @@ int qs_sync_round(qs_ctx* c, uint64_t round, const uint8_t* worker_mask, uint32_
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
     return round_body(c, take_round(c, round), act, true, wire, stride_words, bits_out);
+}
+
+int qs_sync_round_step(qs_ctx* c, const float* grad, float* vel, float eta, float mu, uint64_t round,
+                       const uint8_t* worker_mask, uint32_t* wire, int64_t stride_words, int64_t* bits_out) {
+    if (!c || !wire || !grad) return fail(c, QS_INVALID_ARG, "grad and wire are required");
+    if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
+    if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
+    if (round != QS_ROUND_AUTO && round >= (1ull << 56)) return fail(c, QS_INVALID_ARG, "round must be below 2^56");
+    Active act;
+    if (!make_active(c, worker_mask, &act)) return QS_OK;
+    const StepArgs sa = {grad, vel, eta, mu};
+    return round_body(c, take_round(c, round), act, true, wire, stride_words, bits_out, &sa);
 }
 
 int qs_enable_phase_timing(qs_ctx* c, int on) {

@@ -25,6 +25,13 @@ constexpr int TRACE_SLOTS = 32;       // time stamps of the persistent kernel's 
 constexpr uint32_t Q_NEG = 1u << 16;
 constexpr uint32_t Q_SEL = 1u << 17;
 
+// the local step that precedes a synchronisation: grad R x d, vel R x d or nullptr
+struct StepArgs {
+    const float* grad;
+    float* vel;
+    float eta, mu;
+};
+
 struct Active {          // workers taking part in a call, ascending
     int n;
     uint32_t bits;

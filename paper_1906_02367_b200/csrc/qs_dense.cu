@@ -139,21 +139,29 @@ __global__ void __launch_bounds__(256) broadcast_kernel(const Plan P, const Acti
     }
 }
 
-template <bool ALIGNED>
-__global__ void __launch_bounds__(256) local_step_kernel(const Plan P, const Active act,
-                                                         const float* __restrict__ grad, const float eta) {
+template <bool ALIGNED, bool MOMENTUM>
+__global__ void __launch_bounds__(256) local_step_kernel(const Plan P, const Active act, const StepArgs sa) {
     const int lane = threadIdx.x & 31;
     const int r = act.r[blockIdx.y];
     const size_t row = (size_t)r * P.d;
     for (uint32_t g = blockIdx.x * 8u + (threadIdx.x >> 5); g < P.ngroups; g += gridDim.x * 8u) {
         const uint32_t e0 = g * (uint32_t)GROUP + (uint32_t)lane * 4u;
         if (e0 >= P.d) continue;
-        float w[4], gr[4];
+        float w[4], gr[4], v[4];
         load_quad<ALIGNED>(P.xw + row, e0, P.d, w);
-        load_quad<ALIGNED>(grad + row, e0, P.d, gr);
+        load_quad<ALIGNED>(sa.grad + row, e0, P.d, gr);
+        if (MOMENTUM) {
+            load_quad<ALIGNED>(sa.vel + row, e0, P.d, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float carried = sa.mu * v[j];
+                gr[j] = carried + gr[j];
+            }
+            store_quad<ALIGNED>(sa.vel + row, e0, P.d, gr);
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const float step = eta * gr[j];
+            const float step = sa.eta * gr[j];
             w[j] = w[j] - step;
         }
         store_quad<ALIGNED>(P.xw + row, e0, P.d, w);
@@ -195,11 +203,15 @@ void launch_broadcast(const Plan& P, const Active& act, bool aligned, int sms, c
     else broadcast_kernel<false><<<grid, 256, 0, st>>>(P, act);
 }
 
-void launch_local_step(const Plan& P, const Active& act, const float* grad, float eta, bool aligned,
-                       int sms, cudaStream_t st) {
+void launch_local_step(const Plan& P, const Active& act, const StepArgs& sa, bool aligned, int sms, cudaStream_t st) {
     const dim3 grid(dense_grid(P, sms, 2), act.n);
-    if (aligned) local_step_kernel<true><<<grid, 256, 0, st>>>(P, act, grad, eta);
-    else local_step_kernel<false><<<grid, 256, 0, st>>>(P, act, grad, eta);
+    if (sa.vel) {
+        if (aligned) local_step_kernel<true, true><<<grid, 256, 0, st>>>(P, act, sa);
+        else local_step_kernel<false, true><<<grid, 256, 0, st>>>(P, act, sa);
+    } else {
+        if (aligned) local_step_kernel<true, false><<<grid, 256, 0, st>>>(P, act, sa);
+        else local_step_kernel<false, false><<<grid, 256, 0, st>>>(P, act, sa);
+    }
 }
 
 }  // namespace qs

@@ -7,11 +7,12 @@ namespace qs {
 // qs_dense.cu
 void launch_pass_a(const Plan& P, const Active& act, int mode, bool aligned, int sms, cudaStream_t st);
 void launch_broadcast(const Plan& P, const Active& act, bool aligned, int sms, cudaStream_t st);
-void launch_local_step(const Plan& P, const Active& act, const float* grad, float eta, bool aligned,
-                       int sms, cudaStream_t st);
-// qs_dense_tma.cu: the dense pass fed by bulk copies (aligned rows, synchronous algorithm)
-bool pass_a_tma_usable(const Plan& P, bool aligned);
-cudaError_t launch_pass_a_tma(const Plan& P, const Active& act, int sms, cudaStream_t st);
+// the local step: sa.vel == nullptr plain, otherwise with momentum
+void launch_local_step(const Plan& P, const Active& act, const StepArgs& sa, bool aligned, int sms, cudaStream_t st);
+// qs_dense_tma.cu: the dense pass fed by bulk copies (aligned rows); step 0 none, 1 the plain local
+// step taken on the way (sa.grad, sa.eta), 2 the step with momentum (sa.vel, sa.mu too)
+bool pass_a_tma_usable(const Plan& P, bool aligned, int step);
+cudaError_t launch_pass_a_tma(const Plan& P, const Active& act, const StepArgs& sa, int step, int sms, cudaStream_t st);
 // qs_mid.cu: the persistent kernel that runs every stage after the dense pass
 int mid_blocks_per_sm(bool randk);
 cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode, int patch,

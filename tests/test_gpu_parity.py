@@ -282,6 +282,57 @@ def test_local_step_matches():
     p.close()
 
 
+def test_local_step_with_momentum_matches():
+    R, d = 3, 10007
+    x, xw, mem = I.gaussian_round(R, d, seed=20)
+    p = Pair(R, d, k=10, x=x, xw=xw, mem=mem)
+    vel = np.zeros((R, d), np.float32)
+    gvel = torch.zeros((R, d), device="cuda")
+    for t, mask in enumerate((None, np.array([1, 0, 1], np.uint8), None)):
+        grad = I.gaussian_drift(R, d, 3, t, std=1.0)
+        O.local_step_momentum(p.plan, p.xw, vel, grad, 0.05, 0.9, mask)
+        p.ctx.local_step_momentum(torch.from_numpy(grad).cuda(), gvel, 0.05, 0.9, mask)
+        p.check_state("momentum step")
+        assert bits_equal(gvel.cpu().numpy(), vel)
+    p.close()
+
+
+@pytest.mark.parametrize("d", [6 * 2048 + 1024, 30001])            # bulk-copy path; rows not 16-byte aligned
+@pytest.mark.parametrize("momentum", [False, True])
+@pytest.mark.parametrize("asynchronous", [False, True])
+def test_round_with_the_local_step_taken_inside(d, momentum, asynchronous):
+    """qs_sync_round_step leaves the bytes of the local step followed by the round (oracle: its two calls)."""
+    R, k, eta, mu = 4, 60, 0.05, 0.9
+    x, xw, mem = I.gaussian_round(R, d, seed=29)
+    anchors = xw.copy() if asynchronous else None
+    sizes = [d // 3, d - d // 3]
+    off = np.array([0, sizes[0], d], np.int64)
+    p = Pair(R, d, s=16, seed=5, offsets=off, kseg=np.array([k // 2, k], np.int64), x=x, xw=xw, mem=mem, anchors=anchors)
+    vel = np.zeros((R, d), np.float32)
+    gvel = torch.zeros((R, d), device="cuda") if momentum else None
+    masks = [None, np.array([1, 0, 1, 1], np.uint8), np.array([0, 1, 0, 0], np.uint8)] if asynchronous else [None] * 3
+    for rnd, mask in enumerate(masks):
+        grad = I.gaussian_drift(R, d, 7, rnd, std=0.3)
+        if momentum:
+            O.local_step_momentum(p.plan, p.xw, vel, grad, eta, mu, mask)
+        else:
+            O.local_step(p.plan, p.xw, grad, eta, mask)
+        out = O.sync_round(p.plan, rnd, p.x, p.xw, p.mem, anchors=p.anchors, mask=mask)
+        assert out["rc"] == 0
+        p.ctx.sync_round_step(p.wire, torch.from_numpy(grad).cuda(), eta, vel=gvel, mu=mu, rnd=rnd, mask=mask,
+                              bits_out=p.gbits)
+        assert p.ctx.sync_status() == 0, p.ctx.last_error()
+        # a worker outside the mask keeps its model: the oracle did not step it either
+        p.check_state(f"round {rnd} with its local step")
+        if momentum:
+            assert bits_equal(gvel.cpu().numpy(), vel)
+        w = p.wire.cpu().numpy().view(np.uint32)
+        for r in range(R):
+            if mask is None or mask[r]:
+                assert np.array_equal(w[r], out["wire"][r]), f"record, worker {r}"
+    p.close()
+
+
 def test_round_is_deterministic():
     R, d, k = 4, 70000, 700
     x, xw, mem = I.gaussian_round(R, d, seed=23)
