@@ -11,7 +11,7 @@ import numpy as np
 from . import build as _build
 
 TOPK, RANDK = 0, 1
-QSGD, QSGD_SCALED, SIGN_L1, NONE = 0, 1, 2, 3
+QSGD, QSGD_SCALED, SIGN_L1, NONE, SIGN_L2 = 0, 1, 2, 3, 4
 SORT, NTH = 0, 1
 
 _lib = None

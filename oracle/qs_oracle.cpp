@@ -42,6 +42,9 @@
 //             operator with gamma = k/d, Section 2.2; the Top_k-SGD scheme of the comparisons):
 //             g = u on the kept set, so the memory becomes 0 there; the record carries 32-bit
 //             values instead of signs and levels, and all k entries.
+//   [sign-l2] quantizer 4 is Lemma 3's operator with m = 2: g = N2/k with N2 the l2 norm of
+//             the kept vector ([norm]); record as for quantizer 2.  m >= 3 is not provided (its
+//             sum of m-th powers has no exact fp64 terms, and gamma_m only shrinks with m).
 //   [pieces]  Corollary 1: each segment has its own k, norm, beta.
 //   [momentum] Section 5.1 applies momentum 0.9 on the local iterations and prints no
 //             formula: the heavy-ball form v <- mu v + grad, xhat <- xhat - eta v is taken,
@@ -80,7 +83,8 @@
 namespace {
 
 enum { SP_TOPK = 0, SP_RANDK = 1 };
-enum { QZ_QSGD = 0, QZ_QSGD_SCALED = 1, QZ_SIGN_L1 = 2, QZ_NONE = 3 };
+enum { QZ_QSGD = 0, QZ_QSGD_SCALED = 1, QZ_SIGN_L1 = 2, QZ_NONE = 3, QZ_SIGN_L2 = 4 };
+inline bool is_sign(int quantizer) { return quantizer == QZ_SIGN_L1 || quantizer == QZ_SIGN_L2; }
 enum { ERR_OK = 0, ERR_ARG = -1, ERR_CAPACITY = -4, ERR_NONFINITE = -5 };
 
 // ---------------------------------------------------------------- Philox
@@ -288,11 +292,11 @@ uint32_t get_bits(const uint32_t* w, int64_t bitpos, int width) {
 // words of the streams of a segment that sends n entries, and bits per entry
 int64_t payload_words(int64_t n, int bi, int bl, int quantizer) {
     if (quantizer == QZ_NONE) return words_for(n, bi) + n;                 // indices, then 32-bit values
-    return words_for(n, bi) + words_for(n, 1) + (quantizer != QZ_SIGN_L1 ? words_for(n, bl) : 0);
+    return words_for(n, bi) + words_for(n, 1) + (!is_sign(quantizer) ? words_for(n, bl) : 0);
 }
 int entry_bits(int bi, int bl, int quantizer) {
     if (quantizer == QZ_NONE) return bi + 32;
-    return bi + 1 + (quantizer != QZ_SIGN_L1 ? bl : 0);
+    return bi + 1 + (!is_sign(quantizer) ? bl : 0);
 }
 
 struct Plan {
@@ -334,7 +338,8 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
         else select_randk(P.seed, round, (uint32_t)r, lo, n_el, k, mode, idx.data());
         std::vector<float> kept(k);
         for (int64_t j = 0; j < k; ++j) kept[j] = u[lo + idx[j]];
-        const float N = plain ? 0.0f : has_levels ? norm_l2_exact(kept.data(), k) : norm_l1_exact(kept.data(), k);
+        const float N = plain ? 0.0f
+                      : (has_levels || P.quantizer == QZ_SIGN_L2) ? norm_l2_exact(kept.data(), k) : norm_l1_exact(kept.data(), k);
         const float c = (float)(1.0 / (1.0 + beta_qsgd(k, P.s)));
         std::vector<int64_t> s_idx; std::vector<int> s_lvl, s_neg; std::vector<float> s_val;
         for (int64_t j = 0; j < k; ++j) {

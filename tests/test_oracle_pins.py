@@ -196,7 +196,7 @@ def values_from_details(plan, out, r):
         k = int(plan.kseg[sg])
         N = out["norm"][r, sg]
         lv = out["level"][r, pos:pos + k].astype(np.float32)
-        if plan.quantizer == O.SIGN_L1:
+        if plan.quantizer in (O.SIGN_L1, O.SIGN_L2):
             mag = np.full(k, N / np.float32(k), np.float32)
         else:
             mag = (N * lv) / np.float32(plan.s)
@@ -283,7 +283,7 @@ def test_scaled_operator_is_the_unscaled_one_times_c():
 def decode_dense(plan, out, r):
     dense = np.zeros(plan.d, np.float64)
     g = values_from_details(plan, out, r).astype(np.float64)
-    if plan.quantizer != O.SIGN_L1:
+    if plan.quantizer not in (O.SIGN_L1, O.SIGN_L2):
         g[out["level"][r] == 0] = 0.0
     dense[out["sel"][r]] = g
     return dense
@@ -649,3 +649,56 @@ def test_momentum_step_respects_the_mask():
     v = (np.float32(0.9) * vel0[0]).astype(np.float32) + grad[0]
     assert np.array_equal(vel[0], v.astype(np.float32))
     assert np.array_equal(xw[0], (xw0[0] - (np.float32(0.1) * v).astype(np.float32)).astype(np.float32))
+
+
+# ---------------------------------------------------------------- Lemma 3 with m = 2 (sign scaled by the l2 norm)
+def test_sign_l2_closed_form_contraction_and_record():
+    R, d = 2, 300
+    x, xw, mem = I.gaussian_round(R, d, seed=14)
+    for k in (1, 17, d):
+        plan = O.Plan(R, d, k=k, quantizer=O.SIGN_L2)
+        out, u, mem2 = run_details(plan, 0, x, xw, mem)
+        assert plan.wire_words() == O.Plan(R, d, k=k, quantizer=O.SIGN_L1).wire_words()
+        for r in range(R):
+            kept = u[r][out["sel"][r]]
+            N2 = out["norm"][r, 0]
+            assert N2 == exact_l2(kept)                               # the norm in the record is the l2 norm
+            u64 = u[r].astype(np.float64)
+            N1 = float(np.abs(kept.astype(np.float64)).sum())
+            lhs = float((mem2[r].astype(np.float64) ** 2).sum())
+            # sum over the kept set of (u_i - a sgn_i)^2 with a = N2/k, plus the untouched rest
+            rhs = float((u64 ** 2).sum()) - 2.0 * float(N2) / k * N1 + float(N2) ** 2 / k
+            assert lhs == pytest.approx(rhs, rel=1e-5)
+            # compression operator with gamma_2 = k^(2/2 - 1) / d = 1/d, surely for Top_k
+            assert lhs <= (1.0 - 1.0 / d) * float((u64 ** 2).sum()) * (1 + 1e-6)
+            # the record decodes to +-N2/k on the kept set
+            dense = decode_dense(plan, out, r)
+            want = np.zeros(d)
+            want[out["sel"][r]] = np.where(kept < 0, -1.0, 1.0) * float(np.float32(N2) / np.float32(k))
+            assert np.array_equal(dense, want)
+            if k == 1:                                                # one kept entry: C(u) = u there, memory 0
+                assert mem2[r][out["sel"][r][0]] == 0.0
+    # the same kept set as the l1-scaled operator (the sparsifier does not see the quantizer)
+    a, _, _ = run_details(O.Plan(R, d, k=17, quantizer=O.SIGN_L1), 0, x, xw, mem)
+    b, _, _ = run_details(O.Plan(R, d, k=17, quantizer=O.SIGN_L2), 0, x, xw, mem)
+    assert np.array_equal(a["sel"], b["sel"]) and np.array_equal(a["sign"], b["sign"])
+
+
+def test_sign_l2_master_decodes_the_record():
+    R, d, k = 3, 500, 20
+    x, xw, mem = I.gaussian_round(R, d, seed=15)
+    plan = O.Plan(R, d, k=k, quantizer=O.SIGN_L2)
+    out, u, _ = run_details(plan, 0, x, xw, mem)
+    acc = np.zeros(d, np.float32)
+    for r in range(R):
+        g = np.zeros(d, np.float32)
+        g[out["sel"][r]] = values_from_details(plan, out, r)
+        acc = (acc + g).astype(np.float32)
+    want = x.copy()
+    touched = np.zeros(d, bool)
+    for r in range(R):
+        touched[out["sel"][r]] = True
+    want[touched] = (x[touched] - acc[touched] / np.float32(R)).astype(np.float32)
+    x2 = x.copy()
+    assert O.unpack_accumulate(plan, x2, out["wire"]) == 0
+    assert np.array_equal(x2, want)
