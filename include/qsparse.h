@@ -74,6 +74,9 @@ enum {
  * Top_k-SGD scheme the paper compares with).  g = u on the kept set; the record carries the
  * kept values as 32-bit words in place of the sign and level streams, all k of them. */
 #define QS_NONE 3
+/* Sign scaled by the l2 norm over k (Lemma 3 with m = 2; gamma_2 = 1/d): g = +-N2/k with N2 the
+ * exactly summed l2 norm of the kept vector; record as for QS_SIGN_L1.  m >= 3 is not provided. */
+#define QS_SIGN_L2 4
 /* op argument of qs_init */
 #define QS_OP(sparsifier, quantizer) ((sparsifier) | ((quantizer) << 4))
 

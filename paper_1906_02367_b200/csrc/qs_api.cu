@@ -335,7 +335,7 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     *out = nullptr;
     const int sp = op & 15, qz = op >> 4;
     if (R < 1 || R > MAX_R || d < 1 || d >= (1ll << 32) || k < 1 || k > d || s < 1 || s > 65535) return QS_INVALID_ARG;
-    if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1 && qz != QS_NONE)) return QS_INVALID_ARG;
+    if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1 && qz != QS_NONE && qz != QS_SIGN_L2)) return QS_INVALID_ARG;
     qs_ctx* c = new qs_ctx();
     std::memset(&c->P, 0, sizeof(Plan));
     c->st = static_cast<cudaStream_t>(cuda_stream);

@@ -223,6 +223,8 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* sh, ui
 
 __device__ __forceinline__ void set_status(const Plan& P, int code) { atomicCAS(P.status, 0, code); }
 
+__host__ __device__ __forceinline__ bool qz_is_sign(int qz) { return qz == QS_SIGN_L1 || qz == QS_SIGN_L2; }
+
 __host__ __device__ __forceinline__ uint32_t words_for(uint32_t nfields, uint32_t width) {
     return (uint32_t)(((uint64_t)nfields * width + 31u) >> 5);
 }
@@ -230,11 +232,11 @@ __host__ __device__ __forceinline__ uint32_t words_for(uint32_t nfields, uint32_
 // words of the streams of a segment that sends n entries, and bits per entry
 __host__ __device__ __forceinline__ uint32_t streams_words(uint32_t n, uint32_t bi, uint32_t bl, int qz) {
     if (qz == QS_NONE) return words_for(n, bi) + n;                     // indices, then 32-bit values
-    return words_for(n, bi) + words_for(n, 1) + (qz != QS_SIGN_L1 ? words_for(n, bl) : 0u);
+    return words_for(n, bi) + words_for(n, 1) + (!qz_is_sign(qz) ? words_for(n, bl) : 0u);
 }
 __host__ __device__ __forceinline__ uint32_t entry_bits(uint32_t bi, uint32_t bl, int qz) {
     if (qz == QS_NONE) return bi + 32u;
-    return bi + 1u + (qz != QS_SIGN_L1 ? bl : 0u);
+    return bi + 1u + (!qz_is_sign(qz) ? bl : 0u);
 }
 
 // fp32 level of the QSGD quantizer and the value it stands for
@@ -252,7 +254,7 @@ __device__ __forceinline__ int qsgd_level(float u, float N, int s, uint32_t w) {
 __device__ __forceinline__ float coord_value(const Plan& P, float N, int level, bool neg, float c,
                                              uint32_t k) {
     float g;
-    if (P.qz == QS_SIGN_L1) {
+    if (qz_is_sign(P.qz)) {                      // Lemma 3: the l1 (m = 1) or l2 (m = 2) norm over k
         g = N / (float)k;
     } else {
         g = (N * (float)level) / (float)P.s;

@@ -755,7 +755,7 @@ template <bool RANDK>
 __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_chunks;
-    const bool sign_op = P.qz == QS_SIGN_L1, plain = P.qz == QS_NONE;
+    const bool sign_op = qz_is_sign(P.qz), plain = P.qz == QS_NONE;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
         const float N = c.un.norm, cs = P.cscale[c.seg];
@@ -891,7 +891,7 @@ __device__ void stage_pack_dir(const Plan& P, const Active& act, uint32_t* wire,
 // streams of every segment, and the ordered kept list kept for inspection
 __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
     const uint32_t total = tab.total_chunks;
-    const bool plain = P.qz == QS_NONE, has_lvl = P.qz != QS_SIGN_L1 && !plain;
+    const bool plain = P.qz == QS_NONE, has_lvl = !qz_is_sign(P.qz) && !plain;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
         uint32_t run_k, run_s, unit_n, pay;
@@ -1069,7 +1069,7 @@ __device__ __forceinline__ float entry_value(const Plan& P, const uint32_t* row,
     const uint32_t* w_lvl = w_sgn + words_for(en.n, 1);
     const bool neg = (w_sgn[en.j >> 5] >> (en.j & 31u)) & 1u;
     if (P.qz == QS_NONE) return __uint_as_float(w_sgn[en.j]);       // the value stream sits where the signs would
-    const int level = P.qz == QS_SIGN_L1 ? 1 : (int)get_bits(w_lvl, (uint64_t)en.j * P.bl, P.bl) + 1;
+    const int level = qz_is_sign(P.qz) ? 1 : (int)get_bits(w_lvl, (uint64_t)en.j * P.bl, P.bl) + 1;
     return coord_value(P, __uint_as_float(row[2 * en.seg + 1]), level, neg, P.cscale[en.seg], P.kseg[en.seg]);
 }
 

@@ -59,7 +59,7 @@ __device__ __forceinline__ float record_value(const StaticArgs& a, const uint32_
     const bool neg = (w_sgn[j >> 5] >> (j & 31u)) & 1u;
     const float N = __uint_as_float(row[1]);
     float g;
-    if (a.quantizer == QS_SIGN_L1) {
+    if (qs::qz_is_sign(a.quantizer)) {
         g = N / (float)a.k;
     } else {
         const int level = (int)field(w_lvl, (uint64_t)j * a.bl, a.bl) + 1;
@@ -151,14 +151,14 @@ int qs_unpack_accumulate_static(int R, int64_t d, int64_t k, int s, int quantize
                                 int64_t stride_words, const uint8_t* worker_mask, void* cuda_stream) {
     if (d > STATIC_MAX_D) return QS_TOO_LARGE;
     if (R < 1 || R > qs::MAX_R || d < 1 || k < 1 || k > d || s < 1 || s > 65535 || !x || !wire) return QS_INVALID_ARG;
-    if (quantizer != QS_QSGD && quantizer != QS_QSGD_SCALED && quantizer != QS_SIGN_L1) return QS_INVALID_ARG;
+    if (quantizer != QS_QSGD && quantizer != QS_QSGD_SCALED && quantizer != QS_SIGN_L1 && quantizer != QS_SIGN_L2) return QS_INVALID_ARG;
     StaticArgs a;
     a.R = R; a.s = s; a.quantizer = quantizer;
     a.d = (uint32_t)d; a.k = (uint32_t)k;
     a.bl = ceil_log2_host((unsigned long long)s) < 1 ? 1 : ceil_log2_host((unsigned long long)s);
     a.bi = ceil_log2_host((unsigned long long)d) < 1 ? 1 : ceil_log2_host((unsigned long long)d);
     const long long need = 2 + (long long)qs::words_for(a.k, a.bi) + qs::words_for(a.k, 1) +
-                           (quantizer != QS_SIGN_L1 ? (long long)qs::words_for(a.k, a.bl) : 0);
+                           (!qs::qz_is_sign(quantizer) ? (long long)qs::words_for(a.k, a.bl) : 0);
     if (stride_words < need) return QS_CAPACITY;
     const double b1 = (double)k / ((double)s * (double)s), b2 = std::sqrt((double)k) / (double)s;
     a.cscale = (float)(1.0 / (1.0 + (b1 < b2 ? b1 : b2)));

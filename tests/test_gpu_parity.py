@@ -128,7 +128,7 @@ def test_config1_single_round():
 @pytest.mark.parametrize("d,k", [(1, 1), (2, 1), (2, 2), (31, 4), (32, 32), (33, 7), (127, 9), (128, 1), (129, 129),
                                  (1000, 10), (4099, 41), (7850, 40)])
 @pytest.mark.parametrize("sp,qz", [(O.TOPK, O.QSGD), (O.TOPK, O.SIGN_L1), (O.RANDK, O.QSGD_SCALED), (O.RANDK, O.SIGN_L1),
-                                   (O.TOPK, O.NONE), (O.RANDK, O.NONE)])
+                                   (O.TOPK, O.NONE), (O.RANDK, O.NONE), (O.TOPK, O.SIGN_L2)])
 def test_small_and_ragged_sizes(d, k, sp, qz):
     R = 3
     x, xw, mem = I.gaussian_round(R, d, seed=d)
@@ -186,7 +186,7 @@ def test_per_tensor_and_flat_over_rounds():
                 dict(offsets=off, kseg=I.k_per_tensor_ratio(sizes)),
                 dict(offsets=off, kseg=I.k_per_tensor_capped(sizes, 10))]
     for kw in variants:
-        for qz in (O.SIGN_L1, O.QSGD, O.NONE):
+        for qz in (O.SIGN_L1, O.QSGD, O.NONE, O.SIGN_L2):
             p = Pair(R, d, s=16, quantizer=qz, seed=3, x=x, xw=np.broadcast_to(x, (R, d)).copy(), mem=zeros, **kw)
             for rnd in range(6):
                 p.drift(I.laplace_drift(R, off, scales, 0, rnd))
@@ -251,7 +251,7 @@ def test_colliding_workers():
     x, xw, mem = I.gaussian_round(R, d, seed=13)
     xw[:] = xw[0]
     mem[:] = mem[0]
-    for qz in (O.QSGD, O.SIGN_L1, O.NONE):
+    for qz in (O.QSGD, O.SIGN_L1, O.NONE, O.SIGN_L2):
         p = Pair(R, d, k=k, s=16, quantizer=qz, seed=4, x=x, xw=xw, mem=mem)
         p.round_fused(0)
         p.close()

@@ -21,7 +21,7 @@ def _bits(t):
     return t.cpu().numpy().view(np.uint32)
 
 
-@pytest.mark.parametrize("quantizer,s", [(0, 16), (1, 4), (2, 1)])
+@pytest.mark.parametrize("quantizer,s", [(0, 16), (1, 4), (2, 1), (4, 1)])
 def test_static_update_matches_the_regular_one_twice(quantizer, s):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
