@@ -510,13 +510,82 @@ def run_step(args):
     ctx.destroy()
 
 
+def run_sharded(args):
+    """The headline job (R = 8 workers) spread over the ranks: each rank holds R / N workers and a
+    replica of x, the packed records are all-gathered (NCCL), every rank decodes all of them.  Total
+    work is fixed, so this line reports strong scaling; the default line stays N independent replicas."""
+    import torch
+    import torch.distributed as dist
+    from paper_1906_02367_b200 import binding as B, sharded
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    sizes, off, d, seg_off, kseg = workload("flat", args.shrink)
+    base, count = sharded.partition(R, world)[rank]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(777 + rank)
+    per_elem = torch.from_numpy(np.repeat(I.tensor_scales(len(sizes), seed=0), np.diff(off))).to(dev)
+    x = torch.from_numpy(I.model_init(d, seed=0)).to(dev)
+    xw = x.expand(count, d).contiguous()
+    mem = torch.zeros((count, d), dtype=torch.float32, device=dev)
+    e1 = torch.empty((count, d), dtype=torch.float32, device=dev)
+    e2 = torch.empty_like(e1)
+    ctx = B.Context(count, d, int(kseg[0]), 1, B.QS_TOPK, B.QS_SIGN_L1, seed=0)
+    ctx.bind(x, xw, mem)
+    wire = ctx.new_wire()
+    job = sharded.ShardedRound(R, ctx, wire, rank=rank, world=world)
+
+    def drift():
+        e1.exponential_(generator=gen)
+        e2.exponential_(generator=gen)
+        e1.sub_(e2).mul_(per_elem)
+        xw.add_(e1)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        drift()
+        job.round(t)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    for i in range(args.steps):
+        drift()
+        if world > 1:
+            dist.barrier()                # the ranks enter the round together, as after a local step
+        starts[i].record()
+        job.round(args.warmup + i)
+        ends[i].record()
+    barrier()
+    assert ctx.sync_status() == 0, ctx.last_error()
+    total_ms = max_over_ranks(float(sum(a.elapsed_time(b) for a, b in zip(starts, ends))), dev)
+    bmin = 16 * R * d + 8 * d * world                  # every rank updates its own replica of x
+    if rank == 0:
+        print(json.dumps({
+            "metric": "sharded_round_effective_bandwidth", "value": bmin * args.steps / (total_ms * 1e-3) / 1e9, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "strong", "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"ResNet-50-shaped round, R=8 workers over {world} GPU(s), d={d}, Top_k 0.1% flat, sign/l1; "
+                                   "separate calls with one all-gather of the records", "workers_per_gpu": count}}))
+    ctx.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor", "async", "step"])
+    ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor", "async", "step", "sharded"])
     ap.add_argument("--shrink", type=int, default=1, help="divide every tensor size (profiling on a small case)")
     ap.add_argument("--sweep5", action="store_true", help="run the d = 2^28 ratio x s sweep instead of the headline workload")
     ap.add_argument("--no-e2e", action="store_true")
@@ -531,6 +600,8 @@ def main():
         run_async(args)
     elif args.variant == "step":
         run_step(args)
+    elif args.variant == "sharded":
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -121,6 +121,23 @@ int qs_set_segments(qs_ctx* ctx, int nseg, const int64_t* offsets, const int64_t
 int qs_bind(qs_ctx* ctx, float* x, float* xw, float* mem, float* anchors);
 
 /*
+ * qs_set_sharding — the masterless form of the method (Section 1: each worker exchanges its
+ * updates with all other workers and the aggregation is done without a master), for a job of
+ * R_total workers spread over several contexts, one per GPU: this context holds the workers
+ * worker_base .. worker_base + R - 1.  After the call
+ *   - the random draws (QSGD levels, Rand_k) use the global worker id, so a worker's record does
+ *     not depend on where it runs;
+ *   - qs_unpack_accumulate expects the records of the whole job: wire rows and worker_mask are
+ *     indexed by global worker id (R_total rows), and the update divides by R_total;
+ *   - qs_compress_feedback, qs_pack, qs_broadcast, qs_local_step keep local indices (R rows);
+ *   - qs_sync_round and qs_sync_round_step return QS_STATE unless R_total == R: the records of
+ *     the other shards have to be gathered between qs_pack and qs_unpack_accumulate.
+ * Every shard decodes the same R_total records in the same order, so the replicas of x stay
+ * bit-identical.  Requires worker_base >= 0 and worker_base + R <= R_total <= 32.
+ */
+int qs_set_sharding(qs_ctx* ctx, int worker_base, int R_total);
+
+/*
  * qs_local_step — the local SGD step of Algorithm 1 (line 5) for the masked workers:
  *   xw_r <- xw_r - eta * grad_r, a multiply and a subtract, each rounded to fp32.
  *   grad: device, R x d.

@@ -21,7 +21,7 @@ QS_QSGD, QS_QSGD_SCALED, QS_SIGN_L1, QS_NONE, QS_SIGN_L2 = 0, 1, 2, 3, 4
 QS_ROUND_AUTO = 2**64 - 1
 
 EXPORTS = [
-    "qs_init", "qs_set_segments", "qs_bind", "qs_local_step", "qs_local_step_momentum", "qs_sync_round_step",
+    "qs_init", "qs_set_segments", "qs_set_sharding", "qs_bind", "qs_local_step", "qs_local_step_momentum", "qs_sync_round_step",
     "qs_compress_feedback", "qs_pack",
     "qs_unpack_accumulate", "qs_broadcast", "qs_sync_round", "qs_export_selection", "qs_wire_words",
     "qs_record_bits", "qs_total_k", "qs_sync_status", "qs_last_error", "qs_get_round", "qs_set_round",
@@ -48,6 +48,7 @@ def lib():
         L.qs_init.argtypes = [C.POINTER(vp), C.c_int, i64, i64, C.c_int, C.c_int, u64, vp]
         L.qs_set_segments.argtypes = [vp, C.c_int, vp, vp]
         L.qs_bind.argtypes = [vp, vp, vp, vp, vp]
+        L.qs_set_sharding.argtypes = [vp, C.c_int, C.c_int]
         L.qs_local_step.argtypes = [vp, vp, C.c_float, vp]
         L.qs_local_step_momentum.argtypes = [vp, vp, vp, C.c_float, C.c_float, vp]
         L.qs_sync_round_step.argtypes = [vp, vp, vp, C.c_float, C.c_float, u64, vp, vp, i64, vp]
@@ -120,6 +121,7 @@ class Context:
             raise QsError(rc, "qs_init failed")
         self._keep = []
         self.nseg = 1
+        self.R_total = self.R
 
     def _check(self, rc):
         if rc < 0:
@@ -132,6 +134,10 @@ class Context:
         self._check(lib().qs_set_segments(self._h, len(ks), off.ctypes.data_as(C.c_void_p),
                                           ks.ctypes.data_as(C.c_void_p)))
         self.nseg = len(ks)
+
+    def set_sharding(self, worker_base, R_total):
+        self._check(lib().qs_set_sharding(self._h, int(worker_base), int(R_total)))
+        self.R_total = int(R_total)
 
     def bind(self, x, xw, mem, anchors=None):
         for t in (x, xw, mem) + ((anchors,) if anchors is not None else ()):
@@ -168,7 +174,7 @@ class Context:
         self._check(lib().qs_pack(self._h, _ptr(wire), int(wire.shape[1]), _ptr(bits_out)))
 
     def unpack_accumulate(self, wire, mask=None):
-        m, mp = _mask(mask, self.R)
+        m, mp = _mask(mask, self.R_total)        # the records of the whole job
         self._check(lib().qs_unpack_accumulate(self._h, _ptr(wire), int(wire.shape[1]), mp))
 
     def broadcast(self, mask=None):

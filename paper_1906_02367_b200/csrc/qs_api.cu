@@ -136,6 +136,18 @@ int make_active(const qs_ctx* c, const uint8_t* mask, Active* a) {
     return a->n;
 }
 
+// the records to decode: workers of the whole (possibly sharded) job
+int make_active_job(const qs_ctx* c, const uint8_t* mask, Active* a) {
+    a->n = 0;
+    a->bits = 0;
+    for (int r = 0; r < c->P.rdiv; ++r)
+        if (!mask || mask[r]) {
+            a->r[a->n++] = r;
+            a->bits |= 1u << r;
+        }
+    return a->n;
+}
+
 int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t* kseg) {
     Plan& P = c->P;
     const int64_t d = (int64_t)P.d;
@@ -237,8 +249,8 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(sel_q, (size_t)R * P.K, true);
     AL(pay_off, P.U, true);
     AL(bits, R, true);
-    AL(dec_ent, (size_t)R * (nseg + 1), true);
-    AL(dec_pay, P.U, true);
+    AL(dec_ent, (size_t)32 * (nseg + 1), true);
+    AL(dec_pay, (size_t)32 * nseg, true);
     AL(touch, (size_t)d, true);
     AL(coll, (size_t)R * P.K, false);
     AL(ncoll, 1, true);
@@ -361,6 +373,7 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     c->mid_grid = c->sms * (per_sm < want ? per_sm : want);
     Plan& P = c->P;
     P.R = R; P.d = (uint32_t)d; P.s = s; P.sp = sp; P.qz = qz;
+    P.wbase = 0; P.rdiv = R;
     P.seed_lo = (uint32_t)seed; P.seed_hi = (uint32_t)(seed >> 32);
     const int64_t offsets[2] = {0, d};
     const int rc = install_segments(c, 1, offsets, &k);
@@ -379,6 +392,16 @@ int qs_bind(qs_ctx* c, float* x, float* xw, float* mem, float* anchors) {
     c->P.x = x; c->P.xw = xw; c->P.mem = mem; c->P.anchors = anchors;
     c->aligned = (c->P.d % 4 == 0) && aligned16(x) && aligned16(xw) && aligned16(mem) && aligned16(anchors);
     c->bound = true;
+    c->compressed = false;
+    return QS_OK;
+}
+
+int qs_set_sharding(qs_ctx* c, int worker_base, int R_total) {
+    if (!c) return QS_INVALID_ARG;
+    if (worker_base < 0 || R_total > MAX_R || worker_base + c->P.R > R_total)
+        return fail(c, QS_INVALID_ARG, "need 0 <= worker_base and worker_base + R <= R_total <= 32");
+    c->P.wbase = worker_base;
+    c->P.rdiv = R_total;
     c->compressed = false;
     return QS_OK;
 }
@@ -425,7 +448,7 @@ int qs_unpack_accumulate(qs_ctx* c, const uint32_t* wire, int64_t stride_words, 
     if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
     if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
     Active act;
-    if (!make_active(c, worker_mask, &act)) return QS_OK;
+    if (!make_active_job(c, worker_mask, &act)) return QS_OK;
     return run_mid(c, act, 0, 0, 1, 0, const_cast<uint32_t*>(wire), stride_words, nullptr);
 }
 
@@ -444,6 +467,7 @@ int qs_sync_round(qs_ctx* c, uint64_t round, const uint8_t* worker_mask, uint32_
     if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
     if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
     if (round != QS_ROUND_AUTO && round >= (1ull << 56)) return fail(c, QS_INVALID_ARG, "round must be below 2^56");
+    if (c->P.rdiv != c->P.R) return fail(c, QS_STATE, "a sharded context runs the separate calls: the records of the other shards are needed");
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
     return round_body(c, take_round(c, round), act, true, wire, stride_words, bits_out);
@@ -455,6 +479,7 @@ int qs_sync_round_step(qs_ctx* c, const float* grad, float* vel, float eta, floa
     if (!c->bound) return fail(c, QS_STATE, "no buffers bound");
     if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
     if (round != QS_ROUND_AUTO && round >= (1ull << 56)) return fail(c, QS_INVALID_ARG, "round must be below 2^56");
+    if (c->P.rdiv != c->P.R) return fail(c, QS_STATE, "a sharded context runs the separate calls: the records of the other shards are needed");
     Active act;
     if (!make_active(c, worker_mask, &act)) return QS_OK;
     const StepArgs sa = {grad, vel, eta, mu};

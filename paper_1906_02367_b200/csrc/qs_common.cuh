@@ -56,6 +56,7 @@ struct FbBlock {         // fallback histogram work item: one stretch of one seg
 
 struct Plan {
     int R, nseg, s, sp, qz, bl;
+    int wbase, rdiv;           // sharded job: global id of local worker 0, workers in the whole job (divisor of the update)
     uint32_t d, ngroups, ntile, nblk, nsup, K, U, nfb, maxchunks;
     uint32_t seed_lo, seed_hi, round_lo, round_hi;
     uint64_t cap;
@@ -94,8 +95,8 @@ struct Plan {
     uint32_t* sel_q;           // R x K
     uint32_t* pay_off;         // R x nseg: word offset of the segment's streams
     long long* bits;           // R
-    uint32_t* dec_ent;         // R x (nseg + 1)
-    uint32_t* dec_pay;         // R x nseg
+    uint32_t* dec_ent;         // 32 x (nseg + 1): any worker of a sharded job
+    uint32_t* dec_pay;         // 32 x nseg
     uint32_t* touch;           // d, zero between rounds
     uint2* coll;               // R x K: (coordinate, unit) of indices several workers sent, fused round
     uint32_t* ncoll;           // 1, zero between rounds
@@ -121,7 +122,7 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
 // the four words for coordinates 4q .. 4q+3 of one worker
 __device__ __forceinline__ uint4 philox_quad(const Plan& P, uint32_t worker, uint32_t q,
                                              uint32_t stream) {
-    return philox4x32_10(make_uint4(q, worker, P.round_lo, (P.round_hi << 8) | stream),
+    return philox4x32_10(make_uint4(q, worker + (uint32_t)P.wbase, P.round_lo, (P.round_hi << 8) | stream),
                          make_uint2(P.seed_lo, P.seed_hi));
 }
 

@@ -982,7 +982,7 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* 
                 if (senders[i] == (1u << c.r)) {
                     float acc = 0.0f;
                     acc = acc + g;
-                    P.x[e[i]] = xv[i] - acc / (float)P.R;
+                    P.x[e[i]] = xv[i] - acc / (float)P.rdiv;
                     P.touch[e[i]] = 0u;
                 } else {
                     gval[(size_t)c.r * P.cap + e[i]] = g;
@@ -1117,7 +1117,7 @@ __device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t
             e2.coord = en.coord;
             acc = acc + entry_value(P, wire + (size_t)r2 * stride, e2);
         }
-        const float xn = P.x[en.coord] - acc / (float)P.R;
+        const float xn = P.x[en.coord] - acc / (float)P.rdiv;
         P.x[en.coord] = xn;
         if (patch) {
             for (int w = 0; w < act.n; ++w) {
@@ -1143,7 +1143,7 @@ __device__ void stage_coll_apply(const Plan& P) {
             rest &= rest - 1u;
             acc = acc + gval[(size_t)r2 * P.cap + coord];
         }
-        P.x[coord] = P.x[coord] - acc / (float)P.R;
+        P.x[coord] = P.x[coord] - acc / (float)P.rdiv;
         P.touch[coord] = 0u;
     }
 }

@@ -1,0 +1,70 @@
+"""The synchronisation round over several GPUs, one process per GPU (torch.distributed).
+
+The masterless form the paper mentions in Section 1: every worker's record goes to all the others
+and each aggregates for itself.  Worker r lives on rank r // (R / G); a rank compresses and packs its
+own workers (qs_compress_feedback, qs_pack on a context that qs_set_sharding told its place in the
+job), the packed records are exchanged with ONE all-gather (the only data-path collective: a few
+tens of KB per worker), then every rank decodes the same R records in worker order
+(qs_unpack_accumulate), so the replicas of x stay bit-identical, and broadcasts to its own workers
+locally.  The gathered records land in this rank's memory before any kernel reads them.
+
+Only host logic lives here: the partition, the masks, the collective.  The arithmetic is in the
+library; `engine` is the object that runs it (a binding.Context by default).
+"""
+import numpy as np
+import torch
+import torch.distributed as dist
+
+
+def partition(R, world):
+    """(first worker, number of workers) of every rank: equal contiguous blocks."""
+    if world < 1 or R % world != 0:
+        raise ValueError("the number of workers must be a multiple of the number of ranks")
+    per = R // world
+    return [(g * per, per) for g in range(world)]
+
+
+def local_mask(mask, base, count):
+    """The part of a job-wide worker mask (None = everyone) that concerns this rank's workers."""
+    if mask is None:
+        return None
+    m = np.ascontiguousarray(mask, dtype=np.uint8)
+    return m[base:base + count].copy()
+
+
+def gather_records(wire_local, R, group=None):
+    """All ranks' packed records, rows ordered by global worker id (ranks hold contiguous blocks, so
+    rank order is worker order).  wire_local: (R / G, stride) int32; returns (R, stride)."""
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    if world == 1:
+        return wire_local
+    out = torch.empty((R, wire_local.shape[1]), dtype=wire_local.dtype, device=wire_local.device)
+    dist.all_gather_into_tensor(out, wire_local.contiguous(), group=group)
+    return out
+
+
+class ShardedRound:
+    """One rank's share of a job of R workers.  x is this rank's replica of the global model; xw, mem
+    (and anchors) hold this rank's workers only."""
+
+    def __init__(self, R, engine, wire_local, rank=None, world=None, group=None):
+        self.group = group
+        self.world = world if world is not None else (dist.get_world_size(group) if dist.is_initialized() else 1)
+        self.rank = rank if rank is not None else (dist.get_rank(group) if dist.is_initialized() else 0)
+        self.R = int(R)
+        self.base, self.count = partition(self.R, self.world)[self.rank]
+        self.engine = engine
+        self.wire_local = wire_local
+        engine.set_sharding(self.base, self.R)
+
+    def round(self, rnd, mask=None, bits_out=None):
+        """Algorithm 1 (mask None) or Algorithm 2 (mask over the R workers of the job) for round rnd."""
+        mine = local_mask(mask, self.base, self.count)
+        if mine is None or mine.any():
+            self.engine.compress_feedback(rnd, mine)
+            self.engine.pack(self.wire_local, bits_out)
+        records = gather_records(self.wire_local, self.R, self.group)
+        self.engine.unpack_accumulate(records, mask)
+        if mine is None or mine.any():
+            self.engine.broadcast(mine)
+        return records

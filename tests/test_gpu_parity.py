@@ -333,6 +333,58 @@ def test_round_with_the_local_step_taken_inside(d, momentum, asynchronous):
     p.close()
 
 
+@pytest.mark.parametrize("sp,qz", [(O.TOPK, O.QSGD), (O.RANDK, O.QSGD_SCALED), (O.TOPK, O.SIGN_L1)])
+def test_sharded_contexts_reproduce_the_whole_job(sp, qz):
+    """Two contexts, each holding half of the workers (qs_set_sharding), run one after the other on
+    this GPU; their records are concatenated in worker order as the all-gather would leave them."""
+    from paper_1906_02367_b200 import sharded
+    R, d, G = 4, 50000, 2
+    off = np.array([0, 20000, d], np.int64)
+    kseg = np.array([150, 300], np.int64)
+    x, xw, mem = I.gaussian_round(R, d, seed=61)
+    xw[2] = xw[1]; mem[2] = mem[1]                                  # workers on different shards collide
+    plan = O.Plan(R, d, s=8, sparsifier=sp, quantizer=qz, seed=9, offsets=off, kseg=kseg)
+    dev = torch.device("cuda:0")
+    shards = []
+    for base, count in sharded.partition(R, G):
+        gx = torch.from_numpy(x.copy()).to(dev)
+        gxw = torch.from_numpy(xw[base:base + count].copy()).to(dev)
+        gmem = torch.from_numpy(mem[base:base + count].copy()).to(dev)
+        ctx = B.Context(count, d, int(kseg[0]), 8, sp, qz, seed=9)
+        ctx.set_segments(off, kseg)
+        ctx.bind(gx, gxw, gmem)
+        ctx.set_sharding(base, R)
+        shards.append((base, count, ctx, gx, gxw, gmem, ctx.new_wire()))
+    masks = [None, np.array([1, 0, 1, 1], np.uint8), np.array([0, 0, 0, 1], np.uint8)]
+    for rnd, mask in enumerate(masks):
+        delta = I.gaussian_drift(R, d, 4, rnd, std=1e-2)
+        xw += delta
+        out = O.sync_round(plan, rnd, x, xw, mem, mask=mask)
+        assert out["rc"] == 0
+        for base, count, ctx, gx, gxw, gmem, wire in shards:
+            gxw += torch.from_numpy(delta[base:base + count]).to(dev)
+            mine = sharded.local_mask(mask, base, count)
+            if mine is None or mine.any():
+                ctx.compress_feedback(rnd, mine)
+                ctx.pack(wire)
+        records = torch.cat([sh[6] for sh in shards], dim=0)        # what the all-gather delivers
+        w = records.cpu().numpy().view(np.uint32)
+        for r in range(R):
+            if mask is None or mask[r]:
+                assert np.array_equal(w[r], out["wire"][r]), f"record of worker {r}"
+        for base, count, ctx, gx, gxw, gmem, wire in shards:
+            ctx.unpack_accumulate(records, mask)
+            ctx.broadcast(sharded.local_mask(mask, base, count))
+            assert ctx.sync_status() == 0, ctx.last_error()
+            assert bits_equal(gx.cpu().numpy(), x), f"replica of x, shard at {base}"
+            assert bits_equal(gxw.cpu().numpy(), xw[base:base + count])
+            assert bits_equal(gmem.cpu().numpy(), mem[base:base + count])
+    with pytest.raises(B.QsError):                                  # the fused call needs every record locally
+        shards[0][2].sync_round(shards[0][6])
+    for sh in shards:
+        sh[2].destroy()
+
+
 def test_round_is_deterministic():
     R, d, k = 4, 70000, 700
     x, xw, mem = I.gaussian_round(R, d, seed=23)

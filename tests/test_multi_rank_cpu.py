@@ -39,3 +39,106 @@ def test_single_process_needs_no_group():
     import bench
     assert bench.max_over_ranks(3.5, torch.device("cpu")) == 3.5
     assert bench.workload("per_tensor")[2] == 25557032 and len(bench.workload("per_tensor")[4]) == 161
+
+
+# ---------------------------------------------------------------- sharded round (records all-gathered), 2 ranks
+class _OracleEngine:
+    """Stands in for the CUDA context on a machine without a GPU: same calls, the oracle's arithmetic."""
+
+    def __init__(self, O, plan_job, x, xw, mem, anchors=None):
+        self.O, self.plan, self.x, self.xw, self.mem, self.anchors = O, plan_job, x, xw, mem, anchors
+        self.base, self.records = 0, None
+
+    def set_sharding(self, base, R_total):
+        assert R_total == self.plan.R
+        self.base = base
+
+    def compress_feedback(self, rnd, mask):
+        self.records = {}
+        for r in range(self.xw.shape[0]):
+            if mask is None or mask[r]:
+                ref = self.x if self.anchors is None else self.anchors[r]
+                out = self.O.compress_worker(self.plan, rnd, self.base + r, ref, self.xw[r], self.mem[r], mode=self.O.SORT)
+                assert out["rc"] == 0
+                self.records[r] = out["wire"]
+
+    def pack(self, wire_local, bits_out=None):
+        for r, w in self.records.items():
+            wire_local[r] = torch.from_numpy(w.view("int32"))
+
+    def unpack_accumulate(self, records, mask):
+        assert self.O.unpack_accumulate(self.plan, self.x, records.numpy().view("uint32"), mask) == 0
+
+    def broadcast(self, mask):
+        import numpy as np
+        for r in range(self.xw.shape[0]):
+            if mask is None or mask[r]:
+                self.xw[r] = self.x
+                if self.anchors is not None:
+                    self.anchors[r] = self.x
+
+
+def _sharded_main(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import oracle as O
+    from paper_1906_02367_b200 import inputs as I, sharded
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    R, d, k = 4, 3000, 40
+    plan = O.Plan(R, d, k=k, s=16, sparsifier=O.TOPK, quantizer=O.QSGD, seed=3)
+    x, xw, mem = I.gaussian_round(R, d, seed=50)
+    anchors = xw.copy()
+    base, count = sharded.partition(R, world)[rank]
+    eng = _OracleEngine(O, plan, x.copy(), xw[base:base + count].copy(), mem[base:base + count].copy(),
+                        anchors[base:base + count].copy())
+    wire_local = torch.zeros((count, plan.wire_words()), dtype=torch.int32)
+    job = sharded.ShardedRound(R, eng, wire_local)
+    masks = [None, np.array([1, 0, 0, 1], np.uint8), np.array([0, 0, 1, 1], np.uint8)]   # the last leaves rank 0 idle
+    for rnd, mask in enumerate(masks):
+        eng.xw += I.gaussian_drift(R, d, 8, rnd, std=1e-2)[base:base + count]
+        job.round(rnd, mask)
+    out[rank] = (eng.x.tobytes(), eng.xw.tobytes(), eng.mem.tobytes(), eng.anchors.tobytes())
+    dist.destroy_process_group()
+
+
+def test_sharded_round_equals_the_single_process_round():
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    from oracle import oracle as O
+    from paper_1906_02367_b200 import inputs as I
+    world, port = 2, 31500 + os.getpid() % 2000
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_sharded_main, args=(world, port, out), nprocs=world, join=True)
+        got = {r: out[r] for r in range(world)}
+    R, d, k = 4, 3000, 40
+    plan = O.Plan(R, d, k=k, s=16, sparsifier=O.TOPK, quantizer=O.QSGD, seed=3)
+    x, xw, mem = I.gaussian_round(R, d, seed=50)
+    anchors = xw.copy()
+    masks = [None, np.array([1, 0, 0, 1], np.uint8), np.array([0, 0, 1, 1], np.uint8)]
+    for rnd, mask in enumerate(masks):
+        xw += I.gaussian_drift(R, d, 8, rnd, std=1e-2)
+        assert O.sync_round(plan, rnd, x, xw, mem, anchors=anchors, mask=mask)["rc"] == 0
+    per = R // world
+    for r in range(world):
+        gx, gxw, gmem, ganch = got[r]
+        assert gx == x.tobytes(), f"replica of x on rank {r}"
+        assert gxw == xw[r * per:(r + 1) * per].tobytes()
+        assert gmem == mem[r * per:(r + 1) * per].tobytes()
+        assert ganch == anchors[r * per:(r + 1) * per].tobytes()
+
+
+def test_partition_and_masks():
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import pytest
+    from paper_1906_02367_b200 import sharded
+    assert sharded.partition(8, 4) == [(0, 2), (2, 2), (4, 2), (6, 2)]
+    assert sharded.partition(8, 1) == [(0, 8)]
+    with pytest.raises(ValueError):
+        sharded.partition(8, 3)
+    assert sharded.local_mask(None, 2, 2) is None
+    assert sharded.local_mask([1, 0, 0, 1, 1, 1], 2, 2).tolist() == [0, 1]
+    w = torch.arange(6, dtype=torch.int32).reshape(2, 3)
+    assert sharded.gather_records(w, 2) is w                   # no process group: one rank holds everything
