@@ -13,7 +13,10 @@ constexpr int GPW = 2;               // groups per warp in a tile
 constexpr int STILE = 8 * GPW * GROUP;   // coordinates per tile: 8 warps x GPW groups = 2048
 constexpr int BLK_TILES = 16;        // tiles per candidate block (32768 coordinates)
 constexpr int SUP_BLOCKS = 64;       // blocks per super-block of the two-level candidate counts
-constexpr int CHUNK = 2048;          // candidates per selection chunk (256 threads x 8)
+#ifndef QS_CHUNK
+#define QS_CHUNK 1024
+#endif
+constexpr int CHUNK = QS_CHUNK;     // candidates per selection chunk (a multiple of the 256 threads)
 constexpr int UT_MAX = 2048;         // units whose table fits in the persistent kernel's shared memory
 constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (top 11 key bits)
 constexpr int FB_SHIFT = 21;
