@@ -228,7 +228,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.guess = const_cast<uint32_t*>(g_up);
 #define AL(field, count, zero) if ((rc = dev_alloc(c, &P.field, (size_t)(count), zero)) != QS_OK) return rc
     AL(stage, (size_t)R * P.cap, false);
-    AL(tile_cnt, (size_t)R * P.ntile, true);
+    AL(tile_cnt, (size_t)R * P.nblk * BLK_TILES, true);
     AL(blk_count, (size_t)R * P.nblk, true);
     AL(sup_count, (size_t)R * P.nsup, true);
     AL(seg_start, (size_t)R * (nseg + 1), true);

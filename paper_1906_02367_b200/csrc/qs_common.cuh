@@ -77,7 +77,7 @@ struct Plan {
     // scratch
     uint32_t* guess;           // R x nseg, sort-key space
     uint2* stage;              // R x cap (index, value bits): candidates as the dense pass left them, tile t at t * STILE
-    uint32_t* tile_cnt;        // R x ntile
+    uint32_t* tile_cnt;        // R x (nblk x BLK_TILES): rows padded to whole blocks, the padding stays zero
     uint32_t* blk_count;       // R x nblk, zero between rounds
     uint32_t* sup_count;       // R x nsup, zero between rounds
     uint32_t* seg_start;       // R x (nseg + 1): first candidate of each segment in the ordered list
@@ -160,7 +160,7 @@ __device__ __forceinline__ void tile_write(const Plan& P, int r, uint32_t tile, 
     if (warp == 7) {
         const uint32_t total = warp_sum(lane < 8 * GPW ? sh_cnt[lane] : 0u);
         if (lane == 0) {
-            P.tile_cnt[(size_t)r * P.ntile + tile] = total;
+            P.tile_cnt[(size_t)r * P.nblk * BLK_TILES + tile] = total;
             if (total) {
                 const uint32_t blk = tile / BLK_TILES;
                 atomicAdd(&P.blk_count[(size_t)r * P.nblk + blk], total);

@@ -123,7 +123,7 @@ __device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask
         for (uint32_t i = sup * SUP_BLOCKS + lane; i < blk; i += 32) part += P.blk_count[(size_t)r * P.nblk + i];
         const uint32_t base = warp_sum(part);
         const uint32_t t0 = blk * BLK_TILES;
-        const uint32_t tc = (lane < BLK_TILES && t0 + lane < P.ntile) ? P.tile_cnt[(size_t)r * P.ntile + t0 + lane] : 0u;
+        const uint32_t tc = lane < BLK_TILES ? P.tile_cnt[(size_t)r * P.nblk * BLK_TILES + t0 + lane] : 0u;
         const uint32_t incl = warp_incl_scan(tc, lane);          // lanes >= BLK_TILES repeat the total
         const uint32_t n = __shfl_sync(0xffffffffu, incl, 31);
         const size_t row = (size_t)r * P.cap;
@@ -192,6 +192,182 @@ __device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask
             ss[sgm] = base + a;
         }
         if (blk == P.nblk - 1 && lane == 0) ss[P.nseg] = base + n;
+    }
+    if (local_bins) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < act.n * 256; i += BT)
+            if (sh_bins[i]) atomicAdd(&P.hist[(size_t)act.r[i >> 8] * 256 + (i & 255)], sh_bins[i]);
+        __syncthreads();
+    }
+}
+
+constexpr uint32_t ORDER_ITEMS_MAX = 8192;    // words of shared memory the order stage may use for its sums
+
+// Exclusive sums in place over a[0..n) in shared memory, started at `base`; a[n] receives the end.
+__device__ void smem_excl_scan(uint32_t* a, uint32_t n, uint32_t base, uint32_t* sh_scan) {
+    const uint32_t per = (n + BT - 1) / BT;
+    const uint32_t i0 = threadIdx.x * per < n ? threadIdx.x * per : n;
+    const uint32_t i1 = i0 + per < n ? i0 + per : n;
+    uint32_t sum = 0;
+    for (uint32_t i = i0; i < i1; ++i) sum += a[i];
+    uint32_t total;
+    uint32_t run = base + block_excl_scan(sum, sh_scan, &total);
+    for (uint32_t i = i0; i < i1; ++i) {
+        const uint32_t c = a[i];
+        a[i] = run;
+        run += c;
+    }
+    if (threadIdx.x == 0) a[n] = base + total;
+    __syncthreads();
+}
+
+// largest i in [0, n) with a[i] <= g (a ascending, a[0] <= g)
+__device__ __forceinline__ uint32_t last_not_above(const uint32_t* a, uint32_t n, uint32_t g) {
+    uint32_t lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const uint32_t m = (lo + hi) >> 1;
+        if (a[m] <= g) lo = m; else hi = m;
+    }
+    return lo;
+}
+
+// The same stage with the work dealt evenly, for act.n x nsup <= ORDER_SUPS_MAX.  Candidates pile up
+// where the coordinates are large (a few tensors), so a split by region leaves most warps idle.
+// Here every block sums the (worker, super-block) counts in shared memory, takes an equal share of
+// the worker-major candidate sequence, wherever it lies, sums the block counts of the super-blocks
+// its share touches (a window at a time), and copies: entry -> block by binary search, -> tile by
+// the block's sixteen tile counts, -> its place in the tile's run.  No block reads more counts
+// than its share needs: a table every block reads in full is a hot spot in the L2.
+constexpr uint32_t ORDER_SUPS_MAX = 2048;
+constexpr uint32_t ORDER_WIN = (ORDER_ITEMS_MAX - ORDER_SUPS_MAX - 8) / SUP_BLOCKS;   // super-blocks per window
+
+template <bool RANDK>
+__device__ void stage_order_even(const Plan& P, const Active& act, uint32_t only_mask, uint32_t* sh_bins,
+                                 uint32_t* sh_tab, uint32_t* sh_scan) {
+    const int lane = threadIdx.x & 31;
+    const bool local_bins = P.nseg == 1 && act.n <= 8;
+    if (local_bins)
+        for (int i = threadIdx.x; i < FB_BINS; i += BT) sh_bins[i] = 0;
+    uint32_t* psup = sh_tab;                             // ns + 1 sums over (worker, super-block)
+    uint32_t* pre = sh_tab + ORDER_SUPS_MAX + 4;         // sums over the blocks of the current window
+    const uint32_t ns = P.nsup * (uint32_t)act.n;
+    for (uint32_t i = threadIdx.x; i < ns; i += BT) {
+        const uint32_t wslot = i / P.nsup;
+        const int r = act.r[wslot];
+        psup[i] = (only_mask && !((only_mask >> r) & 1u)) ? 0u : P.sup_count[(size_t)r * P.nsup + (i - wslot * P.nsup)];
+    }
+    __syncthreads();
+    smem_excl_scan(psup, ns, 0u, sh_scan);
+    const uint32_t total = psup[ns];
+    const uint32_t g_lo = (uint32_t)(((uint64_t)total * blockIdx.x) / gridDim.x);
+    const uint32_t g_hi = (uint32_t)(((uint64_t)total * (blockIdx.x + 1u)) / gridDim.x);
+    if (g_lo < g_hi) {                                   // the same for every thread of the block
+        const uint32_t s_a = last_not_above(psup, ns, g_lo), s_b = last_not_above(psup, ns, g_hi - 1u);
+        for (uint32_t sw = s_a; sw <= s_b; sw += ORDER_WIN) {
+            const uint32_t se = sw + ORDER_WIN < s_b + 1u ? sw + ORDER_WIN : s_b + 1u;
+            const uint32_t nbw = (se - sw) * SUP_BLOCKS;
+            for (uint32_t i = threadIdx.x; i < nbw; i += BT) {
+                const uint32_t sg = sw + i / SUP_BLOCKS;
+                const uint32_t wslot = sg / P.nsup;
+                const uint32_t blk = (sg - wslot * P.nsup) * SUP_BLOCKS + i % SUP_BLOCKS;
+                const int r = act.r[wslot];
+                const bool out = blk >= P.nblk || (only_mask && !((only_mask >> r) & 1u));
+                pre[i] = out ? 0u : P.blk_count[(size_t)r * P.nblk + blk];
+            }
+            __syncthreads();
+            smem_excl_scan(pre, nbw, psup[sw], sh_scan);
+            if (pre[nbw] != psup[se]) set_status(P, QS_STATE);   // the two levels of counts disagree
+            const uint32_t lo = g_lo > psup[sw] ? g_lo : psup[sw];
+            const uint32_t hi = g_hi < psup[se] ? g_hi : psup[se];
+            constexpr int OB = 4;                 // entries per thread whose reads are issued together
+            for (uint32_t g0 = lo; g0 < hi; g0 += BT * OB) {
+                uint2 ent[OB];
+                uint32_t wsl[OB], pos[OB];
+#pragma unroll
+                for (int q = 0; q < OB; ++q) {
+                    const uint32_t g = g0 + q * BT + threadIdx.x;
+                    ent[q] = make_uint2(0u, 0u);
+                    wsl[q] = 0; pos[q] = 0;
+                    if (g < hi) {
+                        const uint32_t a = last_not_above(pre, nbw, g);      // the block that holds entry g
+                        const uint32_t sg = sw + a / SUP_BLOCKS;
+                        const uint32_t wslot = sg / P.nsup;
+                        const uint32_t blk = (sg - wslot * P.nsup) * SUP_BLOCKS + a % SUP_BLOCKS;
+                        const int r = act.r[wslot];
+                        uint32_t off = g - pre[a];
+                        const uint32_t t0 = blk * BLK_TILES;
+                        // the block's sixteen tile counts: 64 aligned bytes
+                        const uint4* tq = reinterpret_cast<const uint4*>(P.tile_cnt + (size_t)r * P.nblk * BLK_TILES + t0);
+                        const uint4 q0 = tq[0], q1 = tq[1], q2 = tq[2], q3 = tq[3];
+                        const uint32_t tc[BLK_TILES] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w,
+                                                        q2.x, q2.y, q2.z, q2.w, q3.x, q3.y, q3.z, q3.w};
+                        uint32_t t = 0;
+                        bool found = false;
+#pragma unroll
+                        for (int i = 0; i < BLK_TILES; ++i) {
+                            if (!found) {
+                                if (off < tc[i]) { t = i; found = true; }
+                                else off -= tc[i];
+                            }
+                        }
+                        wsl[q] = wslot;
+                        pos[q] = g - psup[wslot * P.nsup];
+                        if (found) ent[q] = P.stage[(size_t)r * P.cap + (size_t)(t0 + t) * STILE + off];
+                        else set_status(P, QS_STATE);    // the counts of the dense pass disagree with each other
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < OB; ++q) {
+                    const uint32_t g = g0 + q * BT + threadIdx.x;
+                    const bool valid = g < hi;
+                    const uint32_t idx = ent[q].x;
+                    const int r = act.r[wsl[q]];
+                    uint32_t sk = 0, seg = 0;
+                    if (valid) {
+                        const float val = __uint_as_float(ent[q].y);
+                        sk = RANDK ? ~philox_word(P, (uint32_t)r, idx, 1u) : topk_key(val);
+                        const size_t o = (size_t)r * P.cap + pos[q];
+                        P.cand_idx[o] = idx;
+                        P.cand_val[o] = val;
+                        if (RANDK) P.cand_key[o] = sk;
+                        seg = segment_of(P, idx);
+                    }
+                    // level 0 of the radix select: count the top key byte per unit
+                    const uint32_t tag = (wsl[q] << 24) | (seg << 8) | (sk >> 24);
+                    const uint32_t live = __ballot_sync(0xffffffffu, valid);
+                    if (valid) {
+                        const uint32_t peers = __match_any_sync(live, tag);
+                        if (lane == __ffs(peers) - 1) {
+                            if (local_bins) atomicAdd(&sh_bins[wsl[q] * 256 + (sk >> 24)], __popc(peers));
+                            else atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
+                        }
+                    }
+                }
+            }
+            __syncthreads();                      // the window's sums are replaced next
+        }
+    }
+    // where each segment's candidates begin in the worker's ordered list
+    const uint32_t nb = (uint32_t)act.n * (uint32_t)(P.nseg + 1);
+    for (uint32_t it = blockIdx.x * BT + threadIdx.x; it < nb; it += gridDim.x * BT) {
+        const uint32_t wslot = it / (uint32_t)(P.nseg + 1), sgm = it - wslot * (uint32_t)(P.nseg + 1);
+        const int r = act.r[wslot];
+        if (only_mask && !((only_mask >> r) & 1u)) continue;
+        uint32_t* ss = P.seg_start + (size_t)r * (P.nseg + 1);
+        const uint32_t wbase = psup[wslot * P.nsup];
+        if (sgm == (uint32_t)P.nseg) { ss[sgm] = psup[(wslot + 1) * P.nsup] - wbase; continue; }
+        const uint32_t bound = P.seg_off[sgm];
+        const uint32_t tile = bound / (uint32_t)STILE, blk = tile / (uint32_t)BLK_TILES, sup = blk / (uint32_t)SUP_BLOCKS;
+        uint32_t at = psup[wslot * P.nsup + sup] - wbase;
+        for (uint32_t bq = sup * SUP_BLOCKS; bq < blk; ++bq) at += P.blk_count[(size_t)r * P.nblk + bq];
+        for (uint32_t t = blk * BLK_TILES; t < tile; ++t) at += P.tile_cnt[(size_t)r * P.nblk * BLK_TILES + t];
+        const uint2* run = P.stage + (size_t)r * P.cap + (size_t)tile * STILE;
+        uint32_t a = 0, b = P.tile_cnt[(size_t)r * P.nblk * BLK_TILES + tile];   // first entry of the tile with index >= bound
+        while (a < b) {
+            const uint32_t m = (a + b) >> 1;
+            if (run[m].x < bound) a = m + 1; else b = m;
+        }
+        ss[sgm] = at + a;
     }
     if (local_bins) {
         __syncthreads();
@@ -1225,7 +1401,11 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_cnt[2 * 8 * GPW];
     __shared__ uint32_t sh_flag;
     __shared__ int sh_abort;
-    __shared__ __align__(128) uint32_t t_start[UT_MAX], t_c[UT_MAX], t_cb[UT_MAX + 4];
+    // unit table (three arrays) / candidate-count sums of the order stage / tile buffers of the broadcast
+    __shared__ __align__(128) uint32_t sh_tab[ORDER_ITEMS_MAX + 8];
+    uint32_t* t_start = sh_tab;
+    uint32_t* t_c = sh_tab + UT_MAX;
+    uint32_t* t_cb = sh_tab + 2 * UT_MAX;         // UT_MAX + 1 entries
     __shared__ __align__(8) uint64_t sh_mbar[3];
     __shared__ __align__(16) unsigned char sh_big[FB_BINS * 4];   // fallback bins / radix bins / exponent sums
     const Plan& P = a.P;
@@ -1251,7 +1431,9 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     Tab tab;
     const bool fused = a.do_compress && a.do_pack && a.do_decode;   // whole round: the master update rides along
     if (a.do_compress) {
-        stage_order<RANDK>(P, act, 0u, bins);
+        const bool even = P.nsup * (uint32_t)act.n <= ORDER_SUPS_MAX;
+        if (even) stage_order_even<RANDK>(P, act, 0u, bins, sh_tab, sh_scan);
+        else stage_order<RANDK>(P, act, 0u, bins);
         QS_BARRIER();
         const uint32_t missed = build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
         if (missed) {                              // the same value in every block
@@ -1261,7 +1443,8 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
             QS_BARRIER();
             stage_reflag<RANDK>(P, act, missed, sh_cnt);
             QS_BARRIER();
-            stage_order<RANDK>(P, act, missed, bins);
+            if (even) stage_order_even<RANDK>(P, act, missed, bins, sh_tab, sh_scan);
+            else stage_order<RANDK>(P, act, missed, bins);
             QS_BARRIER();
             if (build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab)) set_status(P, QS_STATE);   // the exact pass cannot miss
             if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd((unsigned long long*)&P.stats[0], (unsigned long long)__popc(missed));
