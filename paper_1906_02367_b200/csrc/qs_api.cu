@@ -252,6 +252,8 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(dec_ent, (size_t)32 * (nseg + 1), true);
     AL(dec_pay, (size_t)32 * nseg, true);
     AL(touch, (size_t)d, true);
+    AL(bm1, 2 * (((size_t)d + 31) >> 5), true);
+    P.bm2 = P.bm1 + (((size_t)d + 31) >> 5);
     AL(coll, (size_t)R * P.K, false);
     AL(ncoll, 1, true);
     AL(status, 1, true);

@@ -101,6 +101,8 @@ struct Plan {
     uint32_t* dec_ent;         // 32 x (nseg + 1): any worker of a sharded job
     uint32_t* dec_pay;         // 32 x nseg
     uint32_t* touch;           // d, zero between rounds
+    uint32_t* bm1;             // ceil(d / 32): coordinates some worker sent (fused round)
+    uint32_t* bm2;             // ceil(d / 32): coordinates several workers sent; directly behind bm1
     uint2* coll;               // R x K: (coordinate, unit) of indices several workers sent, fused round
     uint32_t* ncoll;           // 1, zero between rounds
     int* status;

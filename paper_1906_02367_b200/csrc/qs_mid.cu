@@ -785,6 +785,17 @@ __device__ void stage_tie_find(const Plan& P, const Tab& tab, uint32_t* sh, uint
 }
 
 // ------------------------------------------------------------------ quantize
+// Fused round, the master's "was this index sent, and by more than one worker": one bit per
+// coordinate in each of two bitmaps that the kernel clears when it starts, small enough to stay
+// in the L2 between the stage that sets them and the stage that reads them.
+__device__ __forceinline__ void mark_sender(const Plan& P, uint32_t idx) {
+    const uint32_t bit = 1u << (idx & 31u);
+    if (atomicOr(&P.bm1[idx >> 5], bit) & bit) atomicOr(&P.bm2[idx >> 5], bit);
+}
+
+// quantizers that send every kept entry with level 1: nothing about the record depends on the norm
+__device__ __forceinline__ bool qz_early(int qz) { return qz_is_sign(qz) || qz == QS_NONE; }
+
 template <bool RANDK>
 __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t idx) {
     return sk > un.tau || (sk == un.tau && idx <= un.tie_max);
@@ -796,10 +807,14 @@ __device__ void unit_norm(const Plan& P, uint32_t u);
 // products are summed as two 24-bit halves (QSGD), or the 24-bit mantissas themselves (Sign).
 // A 64-bit sum cannot overflow below 2^32 terms.
 template <bool RANDK>
-__device__ void stage_norm_accum(const Plan& P, const Tab& tab, unsigned long long (*acc)[2], uint32_t* sh_u) {
-    const int lane = threadIdx.x & 31;
+__device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, unsigned long long (*acc)[2], uint32_t* sh_u,
+                                 uint32_t* sh_w) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_chunks;
-    if (P.qz == QS_NONE) return;                   // the plain sparsifier sends the values: no norm
+    const bool plain = P.qz == QS_NONE;            // the plain sparsifier sends the values: no norm
+    // merge: a whole round with a quantizer that sends every kept entry at level 1; the counts and
+    // the sender bits are known here, and the pack stage does the rest of the quantize stage's work
+    const bool early = merge;
     const bool l1 = P.qz == QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
@@ -815,13 +830,18 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, unsigned long lo
         }
         acc[threadIdx.x][0] = 0ull;
         acc[threadIdx.x][1] = 0ull;
+        uint32_t nkept = 0;                          // lane 0 of each warp counts
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
             const bool kept = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
             const uint32_t live = __ballot_sync(0xffffffffu, kept);
-            if (kept) {
+            if (early) {
+                if (lane == 0) nkept += __popc(live);
+                if (kept) mark_sender(P, idx[i]);
+            }
+            if (kept && !plain) {
                 const uint32_t b = __float_as_uint(val[i]);
                 const uint32_t e = (b >> 23) & 255u;
                 const uint32_t m = e ? ((b & 0x7fffffu) | 0x800000u) : (b & 0x7fffffu);
@@ -838,7 +858,14 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, unsigned long lo
                 }
             }
         }
+        if (early && lane == 0) sh_w[wid] = nkept;
         __syncthreads();
+        if (early && threadIdx.x == 0) {
+            uint32_t t = 0;
+            for (int w = 0; w < BT / 32; ++w) t += sh_w[w];
+            P.chunk_cnt[chunk] = t | (t << 16);      // kept | sent << 16
+        }
+        if (plain) continue;
         const unsigned long long a0 = acc[threadIdx.x][0], a1 = acc[threadIdx.x][1];
         if (a0 | a1) {
             unsigned long long* g = P.eacc + ((size_t)c.u * 256 + threadIdx.x) * 2;
@@ -962,7 +989,7 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t*
                 if (level) {
                     mem[idx[i]] = val[i] - (plain ? val[i] : coord_value(P, N, level, neg, cs, k));
                     cnt += 1u << 16;
-                    if (fused) atomicOr(&P.touch[idx[i]], 1u << c.r);     // the master's "who sent this index"
+                    if (fused) mark_sender(P, idx[i]);
                 }
             }
             P.cand_q[c.base + off] = q;
@@ -1064,30 +1091,69 @@ __device__ void stage_pack_dir(const Plan& P, const Active& act, uint32_t* wire,
     }
 }
 
-// streams of every segment, and the ordered kept list kept for inspection
-__device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
+// four sums over the block at once; every thread gets all four.  sh: 4 x (BT / 32) words
+__device__ __forceinline__ void block_sum4(uint32_t v[4], uint32_t* sh) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    __syncthreads();                              // sh may still be read from a previous call
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t w = __reduce_add_sync(0xffffffffu, v[j]);
+        if (lane == 0) sh[j * (BT / 32) + wid] = w;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint32_t t = 0;
+#pragma unroll
+        for (int w = 0; w < BT / 32; ++w) t += sh[j * (BT / 32) + w];
+        v[j] = t;
+    }
+}
+
+// streams of every segment, and the ordered kept list kept for inspection.  A thread takes PER
+// consecutive candidates, so one scan over the block places them all.
+template <bool RANDK>
+__device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
     const uint32_t total = tab.total_chunks;
     const bool plain = P.qz == QS_NONE, has_lvl = !qz_is_sign(P.qz) && !plain;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
         const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+        // this thread's candidates first: their reads overlap the sums below
+        uint32_t q[PER], e[PER];
+        float val[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const uint32_t off = c.first + threadIdx.x * PER + i;
+            const bool in = off < c.c;
+            e[i] = in ? P.cand_idx[c.base + off] : 0u;
+            q[i] = (in && !merge) ? P.cand_q[c.base + off] : 0u;
+            val[i] = (in && (merge || plain)) ? P.cand_val[c.base + off] : 0.0f;
+            if (merge && in) {
+                // the quantize stage's part for level-1 quantizers: sign, and the memory update
+                const uint32_t key = RANDK ? P.cand_key[c.base + off] : topk_key(val[i]);
+                if (is_kept<RANDK>(c.un, key, e[i])) {
+                    const bool neg = val[i] < 0.0f;
+                    q[i] = Q_SEL | (neg ? Q_NEG : 0u) | 1u;
+                    P.mem[(size_t)c.r * P.d + e[i]] = val[i] - (plain ? val[i] : coord_value(P, c.un.norm, 1, neg, P.cscale[c.seg], P.kseg[c.seg]));
+                }
+            }
+        }
         uint32_t run_k, run_s, unit_n, pay;
         const uint32_t bi = P.bidx[c.seg], lo = P.seg_off[c.seg];
         if (tab.fast) {
             // positions from the chunk counts of the unit directly (no scan stage ran)
             const uint32_t c1 = tab.cb[c.u + 1];
-            uint32_t bk = 0, bs = 0, ak = 0, as = 0;
+            uint32_t sums[4] = {0u, 0u, 0u, 0u};          // kept before, sent before, kept in all, sent in all
             for (uint32_t i = c.cb + threadIdx.x; i < c1; i += BT) {
                 const uint32_t v = P.chunk_cnt[i];
-                ak += v & 0xffffu; as += v >> 16;
-                if (i < chunk) { bk += v & 0xffffu; bs += v >> 16; }
+                sums[2] += v & 0xffffu; sums[3] += v >> 16;
+                if (i < chunk) { sums[0] += v & 0xffffu; sums[1] += v >> 16; }
             }
-            uint32_t t0, t1, t2, t3;
-            block_excl_scan(bk, sh, &t0); block_excl_scan(bs, sh, &t1);
-            block_excl_scan(ak, sh, &t2); block_excl_scan(as, sh, &t3);
-            run_k = t0; run_s = t1; unit_n = t3; pay = 2u;
+            block_sum4(sums, sh);
+            run_k = sums[0]; run_s = sums[1]; unit_n = sums[3]; pay = 2u;
             if (chunk == c.cb && threadIdx.x == 0) {          // the unit's first chunk writes its directory entry
                 P.units[c.u].n = unit_n;
-                if (t2 != P.kseg[c.seg]) set_status(P, QS_STATE);
+                if (sums[2] != P.kseg[c.seg]) set_status(P, QS_STATE);
                 uint32_t* row = wire + (size_t)c.r * stride;
                 row[0] = unit_n;
                 row[1] = __float_as_uint(c.un.norm);
@@ -1106,27 +1172,26 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* 
         uint32_t* w_lvl = w_sgn + words_for(unit_n, 1);
         uint32_t* o_idx = P.sel_idx + (size_t)c.r * P.K + P.kprefix[c.seg];
         uint32_t* o_q = P.sel_q + (size_t)c.r * P.K + P.kprefix[c.seg];
-        uint32_t q[PER], e[PER], sent_mask = 0;
-#pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            const uint32_t off = c.first + i * BT + threadIdx.x;
-            q[i] = off < c.c ? P.cand_q[c.base + off] : 0u;
-            e[i] = off < c.c ? P.cand_idx[c.base + off] : 0u;
-        }
+        uint32_t mine = 0, sent_mask = 0;             // kept | sent << 16 among this thread's candidates
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
-            uint32_t tot;
-            const uint32_t ex = block_excl_scan(kept | (sent << 16), sh, &tot);
-            if (kept && run_k + (ex & 0xffffu) < P.kseg[c.seg]) {      // (the bound holds by construction)
-                const uint32_t jk = run_k + (ex & 0xffffu);
+            mine += kept | (sent << 16);
+        }
+        uint32_t tot;
+        const uint32_t ex = block_excl_scan(mine, sh, &tot);
+        uint32_t jk = run_k + (ex & 0xffffu), js0 = run_s + (ex >> 16);
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
+            if (kept && jk < P.kseg[c.seg]) {                          // (the bound holds by construction)
                 o_idx[jk] = e[i];
                 o_q[jk] = q[i];
-                if (sent && run_s + (ex >> 16) < unit_n) {
-                    const uint64_t js = run_s + (ex >> 16);
+                if (sent && js0 < unit_n) {
+                    const uint64_t js = js0;
                     or_bits(w_idx, js * bi, bi, e[i] - lo);
                     if (plain) {
-                        w_sgn[js] = __float_as_uint(P.cand_val[c.base + c.first + i * BT + threadIdx.x]);   // value stream
+                        w_sgn[js] = __float_as_uint(val[i]);                   // value stream
                     } else {
                         if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
                         if (has_lvl) or_bits(w_lvl, js * P.bl, P.bl, (q[i] & 0xffffu) - 1u);
@@ -1134,35 +1199,36 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, uint32_t* 
                     sent_mask |= 1u << i;
                 }
             }
-            run_k += tot & 0xffffu;
-            run_s += tot >> 16;
+            jk += kept;
+            js0 += sent;
         }
         if (fused) {
             // Master update riding along: an index only this worker sent gets acc = 0 + g,
             // x <- x - acc / R right here; an index with several senders has each sender leave its
-            // value at (worker, coordinate) and the lowest sender list it for the next stage.
+            // value at (worker, coordinate) and set its bit in the index's word of sender bits;
+            // whoever finds that word empty lists the index for the next stage.
             // All reads of one kind are issued together: this part is bound by memory latency.
-            uint32_t senders[PER];
+            uint32_t multi = 0;
             float xv[PER];
 #pragma unroll
-            for (int i = 0; i < PER; ++i) senders[i] = ((sent_mask >> i) & 1u) ? P.touch[e[i]] : 0u;
+            for (int i = 0; i < PER; ++i)
+                if (((sent_mask >> i) & 1u) && ((P.bm2[e[i] >> 5] >> (e[i] & 31u)) & 1u)) multi |= 1u << i;
 #pragma unroll
-            for (int i = 0; i < PER; ++i) xv[i] = (senders[i] == (1u << c.r)) ? P.x[e[i]] : 0.0f;
+            for (int i = 0; i < PER; ++i) xv[i] = ((sent_mask & ~multi) >> i) & 1u ? P.x[e[i]] : 0.0f;
             float* gval = reinterpret_cast<float*>(P.stage);
 #pragma unroll
             for (int i = 0; i < PER; ++i) {
-                if (!senders[i]) continue;
-                const float g = plain ? P.cand_val[c.base + c.first + i * BT + threadIdx.x]
+                if (!((sent_mask >> i) & 1u)) continue;
+                const float g = plain ? val[i]
                                       : coord_value(P, c.un.norm, (int)(q[i] & 0xffffu), (q[i] & Q_NEG) != 0,
                                                     P.cscale[c.seg], P.kseg[c.seg]);
-                if (senders[i] == (1u << c.r)) {
+                if (!((multi >> i) & 1u)) {
                     float acc = 0.0f;
                     acc = acc + g;
                     P.x[e[i]] = xv[i] - acc / (float)P.rdiv;
-                    P.touch[e[i]] = 0u;
                 } else {
                     gval[(size_t)c.r * P.cap + e[i]] = g;
-                    if ((uint32_t)(__ffs(senders[i]) - 1) == c.r) P.coll[atomicAdd(P.ncoll, 1u)] = make_uint2(e[i], c.u);
+                    if (atomicOr(&P.touch[e[i]], 1u << c.r) == 0u) P.coll[atomicAdd(P.ncoll, 1u)] = make_uint2(e[i], c.u);
                 }
             }
         }
@@ -1430,6 +1496,11 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     }
     Tab tab;
     const bool fused = a.do_compress && a.do_pack && a.do_decode;   // whole round: the master update rides along
+    if (fused) {
+        const uint32_t nw = 2u * ((P.d + 31u) >> 5);          // the two bitmaps are one allocation
+        for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < nw; i += gridDim.x * BT) P.bm1[i] = 0u;
+    }
+    const bool merge = fused && qz_early(P.qz);                     // level-1 quantizers: no quantize stage of its own
     if (a.do_compress) {
         const bool even = P.nsup * (uint32_t)act.n <= ORDER_SUPS_MAX;
         if (even) stage_order_even<RANDK>(P, act, 0u, bins, sh_tab, sh_scan);
@@ -1469,10 +1540,12 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
             stage_tie_find<RANDK>(P, tab, sh_scan, &sh_small[2], sh_w);
             QS_BARRIER();
         }
-        stage_norm_accum<RANDK>(P, tab, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0]);
+        stage_norm_accum<RANDK>(P, tab, merge, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0], sh_w);
         QS_BARRIER();
-        stage_quant<RANDK>(P, tab, fused, &sh_small[0], sh_w);
-        QS_BARRIER();
+        if (!merge) {
+            stage_quant<RANDK>(P, tab, fused, &sh_small[0], sh_w);
+            QS_BARRIER();
+        }
         if (!tab.fast) {
             stage_chunk_scan(P, tab, act, sh_scan);
             QS_BARRIER();
@@ -1483,7 +1556,7 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
     }
     if (a.do_pack) {
         if (!tab.fast) stage_pack_dir(P, act, a.wire, a.stride, a.bits_out);
-        stage_pack(P, tab, fused, a.wire, a.stride, a.bits_out, &sh_small[0], sh_scan);
+        stage_pack<RANDK>(P, tab, fused, merge, a.wire, a.stride, a.bits_out, &sh_small[0], sh_scan);
         if (a.do_decode) QS_BARRIER();
     }
     if (fused) {
