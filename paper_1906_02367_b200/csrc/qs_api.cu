@@ -257,7 +257,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(coll, (size_t)R * P.K, false);
     AL(ncoll, 1, true);
     AL(status, 1, true);
-    AL(bar, 2, true);
+    AL(bar, 4, true);
     AL(trace, TRACE_SLOTS, true);
     AL(stats, 2, true);
 #undef AL
@@ -276,7 +276,7 @@ int rezero(qs_ctx* c) {
     QS_CUDA_TRY(c, cudaMemsetAsync(P.ncoll, 0, sizeof(uint32_t), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.units, 0, sizeof(Unit) * P.U, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.status, 0, sizeof(int), c->st));
-    QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 2 * sizeof(uint32_t), c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 4 * sizeof(uint32_t), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.blk_count, 0, sizeof(uint32_t) * P.R * P.nblk, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.sup_count, 0, sizeof(uint32_t) * P.R * P.nsup, c->st));
     return QS_OK;

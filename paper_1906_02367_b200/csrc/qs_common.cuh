@@ -106,7 +106,7 @@ struct Plan {
     uint2* coll;               // R x K: (coordinate, unit) of indices several workers sent, fused round
     uint32_t* ncoll;           // 1, zero between rounds
     int* status;
-    uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel
+    uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel, [2], [3] tile tickets
     unsigned long long* trace; // TRACE_SLOTS global-timer stamps of the last persistent launch, or null
     long long* stats;          // device counters: [0] fallback worker-rounds, [1] candidates
 };

@@ -1425,34 +1425,49 @@ __device__ void stage_broadcast_bulk(const Plan& P, const Active& act, float* bu
     for (int b = 0; b < 3; ++b) mbar_init(&mbar[b], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();                              // the buffers were ordinary shared memory until now
+    // Tiles are handed out by a ticket counter: blocks that sit closer to the memory they touch
+    // take more of them, and all blocks finish together.  The next ticket is drawn one tile ahead
+    // so that its round trip is off the path.
     const uint32_t ntiles = P.ntile;
-    const uint32_t mine = blockIdx.x < ntiles ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-    auto load = [&](uint32_t i) {
-        const uint32_t e0 = (blockIdx.x + i * gridDim.x) * (uint32_t)STILE;
+    uint32_t ticket = atomicAdd(P.bar + 2, 1u);
+    uint32_t t0 = 0, t1 = 0, t2 = 0, issued = 0;
+    bool more = true;
+    auto load = [&]() {                              // next tile into buffer issued % 3
+        if (!more) return;
+        const uint32_t t = ticket;
+        if (t >= ntiles) { more = false; return; }
+        ticket = atomicAdd(P.bar + 2, 1u);
+        const uint32_t b = issued % 3;
+        if (b == 0) t0 = t; else if (b == 1) t1 = t; else t2 = t;
+        const uint32_t e0 = t * (uint32_t)STILE;
         const uint32_t bytes = (P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE) * 4u;
-        mbar_expect(&mbar[i % 3], bytes);
-        bulk_load(buf[i % 3], P.x + e0, bytes, &mbar[i % 3]);
+        mbar_expect(&mbar[b], bytes);
+        bulk_load(buf[b], P.x + e0, bytes, &mbar[b]);
+        ++issued;
     };
-    for (uint32_t i = 0; i < 2 && i < mine; ++i) load(i);
+    load();
+    load();
     uint32_t done = 0;
-    for (uint32_t i = 0; i < mine; ++i) {
-        if (!mbar_wait(&mbar[i % 3], (i / 3) & 1u)) { *sh_abort = 1; break; }
+    for (uint32_t i = 0; i < issued; ++i) {
+        const uint32_t b = i % 3;
+        if (!mbar_wait(&mbar[b], (i / 3) & 1u)) { *sh_abort = 1; break; }
         done = i + 1;
-        const uint32_t e0 = (blockIdx.x + i * gridDim.x) * (uint32_t)STILE;
+        const uint32_t t = b == 0 ? t0 : b == 1 ? t1 : t2;
+        const uint32_t e0 = t * (uint32_t)STILE;
         const uint32_t bytes = (P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE) * 4u;
         for (int w = 0; w < act.n; ++w) {
-            bulk_store(P.xw + (size_t)act.r[w] * P.d + e0, buf[i % 3], bytes);
-            if (P.anchors) bulk_store(P.anchors + (size_t)act.r[w] * P.d + e0, buf[i % 3], bytes);
+            bulk_store(P.xw + (size_t)act.r[w] * P.d + e0, buf[b], bytes);
+            if (P.anchors) bulk_store(P.anchors + (size_t)act.r[w] * P.d + e0, buf[b], bytes);
         }
         bulk_commit();
-        if (i + 2 < mine) {
+        if (more) {
             bulk_wait_read<1>();                     // the buffer of tile i - 1 has been read by its stores
-            load(i + 2);
+            load();
         }
     }
     if (*sh_abort) {
         // loads already issued get a bounded chance to land before the block leaves
-        for (uint32_t i = done; i < mine && i < done + 2; ++i) mbar_wait(&mbar[i % 3], (i / 3) & 1u);
+        for (uint32_t i = done; i < issued; ++i) mbar_wait(&mbar[i % 3], (i / 3) & 1u);
         set_status(P, QS_TIMEOUT);
     }
     bulk_wait_all();
@@ -1592,6 +1607,8 @@ __global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
         if (atomicAdd(P.bar + 1, 1u) == gridDim.x - 1) {
             P.bar[0] = 0;
             P.bar[1] = 0;
+            P.bar[2] = 0;                            // tile tickets of the broadcast
+            P.bar[3] = 0;                            // tile tickets of the next dense pass
             *P.ncoll = 0;
         }
     }
