@@ -43,6 +43,7 @@ struct TmaCtl {
     uint64_t full[MAX_STAGES];
     uint64_t xfull[XSLOTS];
     uint32_t cnt[2][8 * GPW];              // candidates per group of the current tile (double-buffered)
+    uint32_t tiles[4];                     // tile of each of the last tile iterations (>= ntiles: no tile is left)
     int abort_flag;
 };
 
@@ -81,19 +82,33 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
     }
     __syncthreads();
 
-    // items of this block: tile iteration `it` (tile = blockIdx.x + it * gridDim.x) x active worker
-    const uint32_t my_tiles = blockIdx.x < ntiles ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-    const uint32_t nitems = my_tiles * (uint32_t)nact;          // below 2^26: at most 2^21 tiles, 32 workers
+    // Items of this block: tile iteration `it` x active worker.  Tiles are handed out by a ticket
+    // counter (the next ticket is drawn one tile ahead, off the path), so that every block works
+    // until the pass is over whatever its share of the memory system was; a ticket beyond the
+    // last tile is passed on to the consumers as the end mark.
     auto slot = [&](int s, int t) { return ring + ((size_t)s * NT + t) * TILE; };
 
     // running position of the producer (the item whose loads start next) and of the consumers: tile
     // iteration, worker, ring slot, and for the consumers the slot's phase; no divisions in the loop
-    uint32_t p_it = 0, p_j = 0;
+    uint32_t p_it = 0, p_j = 0, p_tile = 0, ticket = 0;
     int p_w = 0, p_s = 0;
+    bool more = true;
+    if (threadIdx.x == 0) ticket = atomicAdd(P.bar + 3, 1u);
     auto issue = [&]() {                     // thread 0: start the loads of the producer's item
         const uint32_t it = p_it;
         const int w = p_w;
-        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        if (w == 0) {                        // a new tile
+            p_tile = ticket;
+            S.tiles[it & 3u] = p_tile;
+            if (p_tile >= ntiles) {          // the end mark travels on the item's barrier, with no bytes
+                more = false;
+                mbar_expect(&S.full[p_s], 0u);
+                ++p_j;
+                return;
+            }
+            ticket = atomicAdd(P.bar + 3, 1u);
+        }
+        const uint32_t tile = p_tile;
         const uint32_t e0 = tile * TILE;
         const uint32_t bytes = (P.d - e0 < TILE ? P.d - e0 : TILE) * 4u;
         const int s = p_s;
@@ -115,27 +130,27 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
     };
 
     if (threadIdx.x == 0)
-        while (p_j < (uint32_t)prefetch && p_j < nitems) issue();
+        while (p_j < (uint32_t)prefetch && more) issue();
     // stores (one group per item) that may still be reading their slot when the slot `prefetch`
     // items ahead is refilled: that slot was last used nst - prefetch items before the current one
     const int pending_ok = nst - prefetch - 1;
 
     bool bad = false;
     int sg[GP][4] = {};                      // segments of this lane's quads, refreshed once per tile
-    uint32_t j = 0, it = 0, ph = 0;
+    uint32_t j = 0, it = 0, ph = 0, tile = 0;
     int w = 0, s = 0;
-    for (; j < nitems; ++j) {
+    for (;; ++j) {
         const int r = act.r[w];
-        const uint32_t tile = blockIdx.x + it * gridDim.x;
         const int xsl = (int)(it % XSLOTS);
-        if (threadIdx.x == 0 && p_j < nitems) {
+        if (threadIdx.x == 0 && more) {
             if (pending_ok >= 2) bulk_wait_read<2>();
             else if (pending_ok == 1) bulk_wait_read<1>();
             else bulk_wait_read<0>();
             issue();
         }
         bool ok = mbar_wait(&S.full[s], ph);
-        if (!ANCH && w == 0) ok = ok && mbar_wait(&S.xfull[xsl], (uint32_t)((it / XSLOTS) & 1));
+        if (w == 0 && ok) tile = S.tiles[it & 3u];       // written by the producer before it armed the barrier
+        if (!ANCH && w == 0 && tile < ntiles) ok = ok && mbar_wait(&S.xfull[xsl], (uint32_t)((it / XSLOTS) & 1));   // no x tile comes with the end mark
         if (!ok) S.abort_flag = 1;           // seen by everyone at the barrier below
 
         const uint32_t* gs = tab + (size_t)r * P.nseg;
@@ -203,6 +218,7 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
         fence_async_smem();                  // the tiles written above must be visible to the bulk stores
         __syncthreads();
         if (S.abort_flag) break;
+        if (tile >= ntiles) break;           // the end mark: nothing was loaded for this item (every thread read the same mark)
         if (threadIdx.x == 0) {
             const uint32_t t0 = tile * TILE;
             const uint32_t bytes = (P.d - t0 < TILE ? P.d - t0 : TILE) * 4u;
