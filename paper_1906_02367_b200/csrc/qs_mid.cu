@@ -1138,6 +1138,24 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge
                 }
             }
         }
+        // Master update riding along (whole round): which of this thread's entries are sent is known
+        // from q alone, so the reads it needs (was the index sent by several workers; x) start now
+        // and are in flight while the positions are worked out.
+        uint32_t sent_mask = 0, multi = 0;
+        float xv[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            if ((q[i] & Q_SEL) && (q[i] & 0xffffu)) sent_mask |= 1u << i;
+            xv[i] = 0.0f;
+        }
+        if (fused) {
+#pragma unroll
+            for (int i = 0; i < PER; ++i)
+                if (((sent_mask >> i) & 1u) && ((P.bm2[e[i] >> 5] >> (e[i] & 31u)) & 1u)) multi |= 1u << i;
+#pragma unroll
+            for (int i = 0; i < PER; ++i)
+                if (((sent_mask & ~multi) >> i) & 1u) xv[i] = P.x[e[i]];
+        }
         uint32_t run_k, run_s, unit_n, pay;
         const uint32_t bi = P.bidx[c.seg], lo = P.seg_off[c.seg];
         if (tab.fast) {
@@ -1172,7 +1190,7 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge
         uint32_t* w_lvl = w_sgn + words_for(unit_n, 1);
         uint32_t* o_idx = P.sel_idx + (size_t)c.r * P.K + P.kprefix[c.seg];
         uint32_t* o_q = P.sel_q + (size_t)c.r * P.K + P.kprefix[c.seg];
-        uint32_t mine = 0, sent_mask = 0;             // kept | sent << 16 among this thread's candidates
+        uint32_t mine = 0;                            // kept | sent << 16 among this thread's candidates
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
@@ -1196,25 +1214,16 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge
                         if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
                         if (has_lvl) or_bits(w_lvl, js * P.bl, P.bl, (q[i] & 0xffffu) - 1u);
                     }
-                    sent_mask |= 1u << i;
                 }
             }
             jk += kept;
             js0 += sent;
         }
         if (fused) {
-            // Master update riding along: an index only this worker sent gets acc = 0 + g,
-            // x <- x - acc / R right here; an index with several senders has each sender leave its
-            // value at (worker, coordinate) and set its bit in the index's word of sender bits;
-            // whoever finds that word empty lists the index for the next stage.
-            // All reads of one kind are issued together: this part is bound by memory latency.
-            uint32_t multi = 0;
-            float xv[PER];
-#pragma unroll
-            for (int i = 0; i < PER; ++i)
-                if (((sent_mask >> i) & 1u) && ((P.bm2[e[i] >> 5] >> (e[i] & 31u)) & 1u)) multi |= 1u << i;
-#pragma unroll
-            for (int i = 0; i < PER; ++i) xv[i] = ((sent_mask & ~multi) >> i) & 1u ? P.x[e[i]] : 0.0f;
+            // an index only this worker sent gets acc = 0 + g, x <- x - acc / R right here; an index
+            // with several senders has each sender leave its value at (worker, coordinate) and set
+            // its bit in the index's word of sender bits; whoever finds that word empty lists the
+            // index for the next stage.
             float* gval = reinterpret_cast<float*>(P.stage);
 #pragma unroll
             for (int i = 0; i < PER; ++i) {
@@ -1475,7 +1484,7 @@ __device__ void stage_broadcast_bulk(const Plan& P, const Active& act, float* bu
 
 // ------------------------------------------------------------------ the persistent kernel
 template <bool RANDK>
-__global__ void __launch_bounds__(BT) mid_kernel(const MidArgs a) {
+__global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_scan[33];
     __shared__ uint32_t sh_small[8];              // unit id, prefix, select scratch
     __shared__ uint32_t sh_w[BT / 32];
