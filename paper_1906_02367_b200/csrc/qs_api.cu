@@ -1,4 +1,5 @@
 // C boundary of the sync-round library: context, tables, scratch and the order of launches.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -175,7 +176,9 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.bl = std::max(1, ceil_log2((uint64_t)P.s));
     P.maxchunks = (uint32_t)R * (uint32_t)((d + CHUNK - 1) / CHUNK + nseg);
 
-    std::vector<uint32_t> h_off(nseg + 1), h_k(nseg), h_kp(nseg + 1, 0), h_target(nseg), h_grp, h_guess;
+    std::vector<uint32_t> h_off(nseg + 1), h_k(nseg), h_kp(nseg + 1, 0), h_target(nseg), h_grp, h_guess, h_order(nseg);
+    std::vector<uint32_t> h_pay((size_t)R * nseg, 0u);
+    std::vector<long long> h_bits(R, 0ll);
     std::vector<float> h_c(nseg);
     std::vector<uint8_t> h_bi(nseg);
     std::vector<FbBlock> h_fb;
@@ -189,11 +192,19 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
         const double a = (double)k / ((double)P.s * (double)P.s), b = std::sqrt((double)k) / (double)P.s;
         h_c[g] = (float)(1.0 / (1.0 + (a < b ? a : b)));
         h_bi[g] = (uint8_t)std::max(1, ceil_log2(n));
+        // quantizers that send every kept entry: the streams' places and the bit count never change
+        if (qz_is_sign(P.qz) || P.qz == QS_NONE)
+            for (int r = 0; r < R; ++r) {
+                h_pay[(size_t)r * nseg + g] = (uint32_t)words;
+                h_bits[r] += 64 + (long long)k * entry_bits(h_bi[g], (uint32_t)P.bl, P.qz);
+            }
         words += streams_words((uint32_t)k, h_bi[g], (uint32_t)P.bl, P.qz);
+        h_order[g] = (uint32_t)g;
         for (uint64_t s0 = 0; s0 < n; s0 += FB_CHUNK)
             h_fb.push_back(FbBlock{(uint32_t)g, (uint32_t)(offsets[g] + s0), (uint32_t)std::min<uint64_t>(FB_CHUNK, n - s0)});
     }
     h_off[nseg] = (uint32_t)d;
+    std::stable_sort(h_order.begin(), h_order.end(), [&](uint32_t a, uint32_t b) { return h_target[a] > h_target[b]; });
     P.K = h_kp[nseg];
     P.nfb = (uint32_t)h_fb.size();
     c->wire_words = words;
@@ -221,7 +232,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     int rc;
 #define UP(field, vec) if ((rc = dev_upload(c, &P.field, vec)) != QS_OK) return rc
     UP(seg_off, h_off); UP(kseg, h_k); UP(kprefix, h_kp); UP(grp_seg, h_grp); UP(target, h_target);
-    UP(cscale, h_c); UP(bidx, h_bi); UP(fb_tab, h_fb);
+    UP(cscale, h_c); UP(bidx, h_bi); UP(fb_tab, h_fb); UP(seg_order, h_order);
 #undef UP
     const uint32_t* g_up = nullptr;
     if ((rc = dev_upload(c, &g_up, h_guess)) != QS_OK) return rc;
@@ -247,8 +258,10 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(fb_hist, (size_t)P.U * FB_BINS, true);
     AL(sel_idx, (size_t)R * P.K, true);
     AL(sel_q, (size_t)R * P.K, true);
-    AL(pay_off, P.U, true);
-    AL(bits, R, true);
+    AL(pay_off, P.U, false);
+    AL(bits, R, false);
+    QS_CUDA_TRY(c, cudaMemcpyAsync(P.pay_off, h_pay.data(), h_pay.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, c->st));
+    QS_CUDA_TRY(c, cudaMemcpyAsync(P.bits, h_bits.data(), h_bits.size() * sizeof(long long), cudaMemcpyHostToDevice, c->st));
     AL(dec_ent, (size_t)32 * (nseg + 1), true);
     AL(dec_pay, (size_t)32 * nseg, true);
     AL(touch, (size_t)d, true);
@@ -257,7 +270,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(coll, (size_t)R * P.K, false);
     AL(ncoll, 1, true);
     AL(status, 1, true);
-    AL(bar, 4, true);
+    AL(bar, 8, true);
     AL(trace, TRACE_SLOTS, true);
     AL(stats, 2, true);
 #undef AL
@@ -276,7 +289,7 @@ int rezero(qs_ctx* c) {
     QS_CUDA_TRY(c, cudaMemsetAsync(P.ncoll, 0, sizeof(uint32_t), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.units, 0, sizeof(Unit) * P.U, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.status, 0, sizeof(int), c->st));
-    QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 4 * sizeof(uint32_t), c->st));
+    QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 8 * sizeof(uint32_t), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.blk_count, 0, sizeof(uint32_t) * P.R * P.nblk, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.sup_count, 0, sizeof(uint32_t) * P.R * P.nsup, c->st));
     return QS_OK;
@@ -376,6 +389,8 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     Plan& P = c->P;
     P.R = R; P.d = (uint32_t)d; P.s = s; P.sp = sp; P.qz = qz;
     P.wbase = 0; P.rdiv = R;
+    P.unit_cap = UNIT_CAP;                         // QSPARSE_UNIT_CAP (0 .. 4096) overrides, for tests of both paths
+    if (const char* e = std::getenv("QSPARSE_UNIT_CAP")) P.unit_cap = (uint32_t)std::min(std::max(std::atoi(e), 0), UNIT_CAP);
     P.seed_lo = (uint32_t)seed; P.seed_hi = (uint32_t)(seed >> 32);
     const int64_t offsets[2] = {0, d};
     const int rc = install_segments(c, 1, offsets, &k);

@@ -18,6 +18,7 @@ constexpr int SUP_BLOCKS = 64;       // blocks per super-block of the two-level 
 #endif
 constexpr int CHUNK = QS_CHUNK;     // candidates per selection chunk (a multiple of the 256 threads)
 constexpr int UT_MAX = 2048;         // units whose table fits in the persistent kernel's shared memory
+constexpr int UNIT_CAP = 4096;       // candidates of a unit that one block may select from on its own (16 per thread)
 constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (top 11 key bits)
 constexpr int FB_SHIFT = 21;
 constexpr int FB_CHUNK = 65536;      // coordinates per fallback-histogram block
@@ -62,6 +63,7 @@ struct Plan {
     int wbase, rdiv;           // sharded job: global id of local worker 0, workers in the whole job (divisor of the update)
     uint32_t d, ngroups, ntile, nblk, nsup, K, U, nfb, maxchunks;
     uint32_t seed_lo, seed_hi, round_lo, round_hi;
+    uint32_t unit_cap;         // a round whose units all have at most this many candidates selects per block (0: never)
     uint64_t cap;
     // tables (device)
     const uint32_t* seg_off;   // nseg + 1
@@ -69,6 +71,7 @@ struct Plan {
     const uint32_t* kprefix;   // nseg + 1
     const uint32_t* grp_seg;   // ngroups: segment of the group's first coordinate
     const uint32_t* target;    // nseg: candidates aimed for
+    const uint32_t* seg_order; // nseg: segments by falling candidate target (largest units are dealt first)
     const float* cscale;       // nseg: fl32(1 / (1 + beta_{k,s}))
     const uint8_t* bidx;       // nseg: bits per index field
     const FbBlock* fb_tab;     // nfb
@@ -96,8 +99,8 @@ struct Plan {
     uint32_t* fb_hist;         // U x FB_BINS, zero between rounds
     uint32_t* sel_idx;         // R x K
     uint32_t* sel_q;           // R x K
-    uint32_t* pay_off;         // R x nseg: word offset of the segment's streams
-    long long* bits;           // R
+    uint32_t* pay_off;         // R x nseg: word offset of the segment's streams (fixed when every kept entry is sent)
+    long long* bits;           // R: bits of the worker's record (likewise)
     uint32_t* dec_ent;         // 32 x (nseg + 1): any worker of a sharded job
     uint32_t* dec_pay;         // 32 x nseg
     uint32_t* touch;           // d, zero between rounds
@@ -106,7 +109,7 @@ struct Plan {
     uint2* coll;               // R x K: (coordinate, unit) of indices several workers sent, fused round
     uint32_t* ncoll;           // 1, zero between rounds
     int* status;
-    uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel, [2], [3] tile tickets
+    uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel, [2], [3] tile tickets, [4] unit tickets
     unsigned long long* trace; // TRACE_SLOTS global-timer stamps of the last persistent launch, or null
     long long* stats;          // device counters: [0] fallback worker-rounds, [1] candidates
 };

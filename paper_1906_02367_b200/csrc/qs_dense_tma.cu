@@ -136,7 +136,10 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
     const int pending_ok = nst - prefetch - 1;
 
     bool bad = false;
-    int sg[GP][4] = {};                      // segments of this lane's quads, refreshed once per tile
+    int sq0[GP] = {};                        // segment of each group's first coordinate, refreshed once per tile
+    bool uni[GP];                            // the whole group lies in that segment (the rule, segments being long)
+#pragma unroll
+    for (int k = 0; k < GP; ++k) uni[k] = true;
     uint32_t j = 0, it = 0, ph = 0, tile = 0;
     int w = 0, s = 0;
     for (;; ++j) {
@@ -174,12 +177,16 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
             const uint32_t q = (warp * GP + k) * GROUP + lane * 4;
             const uint32_t e0 = tile * TILE + q;
             if (w == 0 && P.nseg > 1) {
-                int sq = g < P.ngroups ? (int)P.grp_seg[g] : 0;
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    while (sq + 1 < P.nseg && e0 + jj >= seg_off[sq + 1]) ++sq;
-                    sg[k][jj] = sq;
+                // segment of the group's first coordinate, from the offsets in shared memory (a load
+                // from global memory here would stall the tile behind the copies in flight)
+                int lo = 0, hi = P.nseg;
+                const uint32_t first = g * (uint32_t)GROUP;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (seg_off[mid] <= first) lo = mid; else hi = mid;
                 }
+                sq0[k] = lo;
+                uni[k] = lo + 1 >= P.nseg || seg_off[lo + 1] >= first + (uint32_t)GROUP;
             }
             const float4 xq = xq_[k], mq = mq_[k];
             float4 wq = wq_[k];
@@ -210,9 +217,18 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
                 const uint4 h = philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
                 sk[0] = ~h.x; sk[1] = ~h.y; sk[2] = ~h.z; sk[3] = ~h.w;
             }
+            if (uni[k]) {                    // one threshold for the whole group (the same branch in every lane)
+                const uint32_t thr = gs[sq0[k]];
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj)
-                bal[k][jj] = __ballot_sync(0xffffffffu, in && sk[jj] >= gs[sg[k][jj]]);
+                for (int jj = 0; jj < 4; ++jj) bal[k][jj] = __ballot_sync(0xffffffffu, in && sk[jj] >= thr);
+            } else {                         // a segment border inside the group: per coordinate
+                int sq = sq0[k];
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    while (sq + 1 < P.nseg && e0 + jj >= seg_off[sq + 1]) ++sq;
+                    bal[k][jj] = __ballot_sync(0xffffffffu, in && sk[jj] >= gs[sq]);
+                }
+            }
         }
         tile_counts(S.cnt[j & 1], warp, lane, bal);
         fence_async_smem();                  // the tiles written above must be visible to the bulk stores

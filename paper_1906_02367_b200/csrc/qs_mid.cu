@@ -78,14 +78,21 @@ __device__ __forceinline__ uint32_t sort_key(const Plan& P, size_t pos) {
     return RANDK ? P.cand_key[pos] : topk_key(P.cand_val[pos]);
 }
 
+// quantizers that send every kept entry with level 1: nothing about the record depends on the norm
+__device__ __forceinline__ bool qz_early(int qz) { return qz_is_sign(qz) || qz == QS_NONE; }
+
 // Unit table: where each (worker, segment) unit's candidates start, how many there are, and the
 // number of chunks before it.  Every block builds it for itself in shared memory.
 struct Tab {
     const uint32_t* start;
     const uint32_t* c;
     const uint32_t* cb;      // U + 1 entries
+    const uint32_t* lb;      // U + 1 entries: chunks of long units before each unit
     uint32_t total_chunks;
-    bool fast;               // one segment and few chunks per unit: pack finds its own positions
+    uint32_t total_long;     // chunks of the units that take the grid-wide select
+    uint32_t short_c;        // a unit with at most this many candidates is selected from by one block on its own
+    bool any_short;          // there is such a unit
+    bool fast;               // pack finds its own positions: few chunks per unit, and the streams' places are known
 };
 
 __device__ __forceinline__ uint32_t segment_of(const Plan& P, uint32_t e) {
@@ -245,9 +252,12 @@ template <bool RANDK>
 __device__ void stage_order_even(const Plan& P, const Active& act, uint32_t only_mask, uint32_t* sh_bins,
                                  uint32_t* sh_tab, uint32_t* sh_scan) {
     const int lane = threadIdx.x & 31;
-    const bool local_bins = P.nseg == 1 && act.n <= 8;
+    // one segment: the top-byte counts, which pile up on two or three bins per worker, are gathered
+    // per block in shared memory for the eight workers from the first one of the block's share on
+    const bool local_bins = P.nseg == 1;
     if (local_bins)
         for (int i = threadIdx.x; i < FB_BINS; i += BT) sh_bins[i] = 0;
+    uint32_t ws0 = 0;                                    // first worker slot with local bins
     uint32_t* psup = sh_tab;                             // ns + 1 sums over (worker, super-block)
     uint32_t* pre = sh_tab + ORDER_SUPS_MAX + 4;         // sums over the blocks of the current window
     const uint32_t ns = P.nsup * (uint32_t)act.n;
@@ -263,6 +273,7 @@ __device__ void stage_order_even(const Plan& P, const Active& act, uint32_t only
     const uint32_t g_hi = (uint32_t)(((uint64_t)total * (blockIdx.x + 1u)) / gridDim.x);
     if (g_lo < g_hi) {                                   // the same for every thread of the block
         const uint32_t s_a = last_not_above(psup, ns, g_lo), s_b = last_not_above(psup, ns, g_hi - 1u);
+        ws0 = s_a / P.nsup;
         for (uint32_t sw = s_a; sw <= s_b; sw += ORDER_WIN) {
             const uint32_t se = sw + ORDER_WIN < s_b + 1u ? sw + ORDER_WIN : s_b + 1u;
             const uint32_t nbw = (se - sw) * SUP_BLOCKS;
@@ -338,7 +349,7 @@ __device__ void stage_order_even(const Plan& P, const Active& act, uint32_t only
                     if (valid) {
                         const uint32_t peers = __match_any_sync(live, tag);
                         if (lane == __ffs(peers) - 1) {
-                            if (local_bins) atomicAdd(&sh_bins[wsl[q] * 256 + (sk >> 24)], __popc(peers));
+                            if (local_bins && wsl[q] - ws0 < 8u) atomicAdd(&sh_bins[(wsl[q] - ws0) * 256 + (sk >> 24)], __popc(peers));
                             else atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
                         }
                     }
@@ -371,8 +382,9 @@ __device__ void stage_order_even(const Plan& P, const Active& act, uint32_t only
     }
     if (local_bins) {
         __syncthreads();
-        for (int i = threadIdx.x; i < act.n * 256; i += BT)
-            if (sh_bins[i]) atomicAdd(&P.hist[(size_t)act.r[i >> 8] * 256 + (i & 255)], sh_bins[i]);
+        for (int i = threadIdx.x; i < 8 * 256; i += BT)
+            if (sh_bins[i] && ws0 + (uint32_t)(i >> 8) < (uint32_t)act.n)
+                atomicAdd(&P.hist[(size_t)act.r[ws0 + (uint32_t)(i >> 8)] * 256 + (i & 255)], sh_bins[i]);
         __syncthreads();
     }
 }
@@ -380,8 +392,8 @@ __device__ void stage_order_even(const Plan& P, const Active& act, uint32_t only
 // Builds the unit table; returns the workers (bit mask) that have a unit with fewer candidates
 // than k.  Every block computes the same thing from the same data.
 __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_start, uint32_t* t_c, uint32_t* t_cb,
-                                uint32_t* sh, uint32_t* sh_flag, Tab* tab) {
-    if (threadIdx.x == 0) *sh_flag = 0;
+                                uint32_t* t_lb, uint32_t* sh, uint32_t* sh_flag, Tab* tab) {
+    if (threadIdx.x == 0) { sh_flag[0] = 0; sh_flag[1] = 0; sh_flag[2] = 0; sh_flag[3] = 0; }   // workers that fell short; the longest list; units; any short unit
     __syncthreads();
     uint32_t carry = 0;
     for (uint32_t ub = 0; ub < P.U; ub += BT) {
@@ -394,6 +406,8 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
                 start = ss[seg];
                 c = ss[seg + 1] - start;
                 if (c < P.kseg[seg]) atomicOr(sh_flag, 1u << r);
+                atomicMax(sh_flag + 1, c);
+                if (c) atomicAdd(sh_flag + 2, 1u);
             }
         }
         uint32_t total;
@@ -403,11 +417,34 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
     }
     if (threadIdx.x == 0) t_cb[P.U] = carry;
     __syncthreads();
-    tab->start = t_start; tab->c = t_c; tab->cb = t_cb; tab->total_chunks = carry;
-    bool fast = P.nseg == 1;
-    for (uint32_t u = 0; fast && u < P.U; ++u) fast = t_cb[u + 1] - t_cb[u] <= 1024u;
-    tab->fast = fast;
-    return *sh_flag;
+    tab->start = t_start; tab->c = t_c; tab->cb = t_cb; tab->lb = t_lb; tab->total_chunks = carry;
+    const uint32_t longest = sh_flag[1];
+    // the streams' places: one segment, or a quantizer that sends every kept entry (fixed places)
+    tab->fast = (P.nseg == 1 || qz_early(P.qz)) && (longest + CHUNK - 1) / CHUNK <= 1024u;
+    // Which units one block selects from on its own (block barriers only), and which take the
+    // grid-wide radix levels: all of them in a block each when every list is short and there is a
+    // block per unit; otherwise only the lists of at most one candidate per thread.
+    uint32_t short_c = 0;
+    if (P.unit_cap) {
+        const bool all = longest <= P.unit_cap && sh_flag[2] <= gridDim.x;
+        short_c = all ? P.unit_cap : (P.unit_cap < (uint32_t)BT ? P.unit_cap : (uint32_t)BT);
+    }
+    tab->short_c = short_c;
+    carry = 0;
+    for (uint32_t ub = 0; ub < P.U; ub += BT) {
+        const uint32_t u = ub + threadIdx.x;
+        const uint32_t c = u < P.U ? t_c[u] : 0u;
+        if (c && c <= short_c) sh_flag[3] = 1u;            // some unit is short (same value from every writer)
+        uint32_t total;
+        const uint32_t ex = block_excl_scan(c > short_c ? (c + CHUNK - 1) / CHUNK : 0u, sh, &total);
+        if (u < P.U) t_lb[u] = carry + ex;
+        carry += total;
+    }
+    if (threadIdx.x == 0) t_lb[P.U] = carry;
+    __syncthreads();
+    tab->total_long = carry;
+    tab->any_short = sh_flag[3] != 0u;
+    return sh_flag[0];
 }
 
 // histogram of the top 11 key bits of one stretch of one segment, for missed workers
@@ -568,7 +605,7 @@ __device__ void derive_prefix(const Plan& P, uint32_t u, uint32_t k, int level, 
     *above_total = at;
 }
 
-struct ChunkCtx { uint32_t u, r, seg, first, c, cb; Unit un; size_t base; };
+struct ChunkCtx { uint32_t u, r, seg, first, c, cb, chunk; Unit un; size_t base; };   // chunk: its number among all chunks
 
 // which unit a chunk belongs to (one search per block, shared through sh_u)
 __device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, const Tab& tab, uint32_t chunk, uint32_t* sh_u) {
@@ -583,6 +620,32 @@ __device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, const Tab& tab,
     c.c = tab.c[c.u];
     c.cb = tab.cb[c.u];
     c.first = (chunk - c.cb) * CHUNK;
+    c.chunk = chunk;
+    c.base = (size_t)c.r * P.cap + tab.start[c.u];
+    return c;
+}
+
+// the same for chunk q of the long units only (the stages of the grid-wide select walk these)
+__device__ __forceinline__ ChunkCtx long_chunk_context(const Plan& P, const Tab& tab, uint32_t q, uint32_t* sh_u) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t lo = 0, hi = P.U;               // the last unit with lb <= q: short units before it share its lb
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (tab.lb[mid] <= q) lo = mid; else hi = mid;
+        }
+        *sh_u = lo;
+    }
+    __syncthreads();
+    ChunkCtx c;
+    c.u = *sh_u;
+    c.un = P.units[c.u];
+    c.r = c.u / P.nseg;
+    c.seg = c.u % P.nseg;
+    c.c = tab.c[c.u];
+    c.cb = tab.cb[c.u];
+    c.first = (q - tab.lb[c.u]) * CHUNK;
+    c.chunk = c.cb + (q - tab.lb[c.u]);
     c.base = (size_t)c.r * P.cap + tab.start[c.u];
     return c;
 }
@@ -591,10 +654,10 @@ __device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, const Tab& tab,
 template <bool RANDK>
 __device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* sh_hist, uint32_t* sh_u, uint32_t* sh_prefix) {
     const int lane = threadIdx.x & 31;
-    const uint32_t total = tab.total_chunks;
+    const uint32_t total = tab.total_long;
     const int shift = 24 - 8 * level;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+        const ChunkCtx c = long_chunk_context(P, tab, chunk, sh_u);
         uint32_t sk[PER];
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
@@ -626,13 +689,31 @@ __device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* s
     }
 }
 
+// Prediction for the next round (Top_k): move the candidate floor so that about `target`
+// coordinates pass it, assuming the tail keeps its shape (log-linear in the count).  One thread.
+__device__ void predict_floor(const Plan& P, uint32_t r, uint32_t seg, uint32_t tau, uint32_t uc, uint32_t k) {
+    uint32_t* gp = &P.guess[(size_t)r * P.nseg + seg];
+    const float tk = __uint_as_float(tau >> 1), tg = __uint_as_float(*gp >> 1);
+    const float target = (float)P.target[seg];
+    float tn = tg;
+    if (uc > k && tk > tg) {
+        float ratio = __logf(target / (float)k) / __logf((float)uc / (float)k);
+        ratio = fminf(fmaxf(ratio, 0.25f), 4.0f);
+        tn = tk - (tk - tg) * ratio;
+    } else if (uc <= k) {
+        tn = tk * 0.75f;
+    }
+    tn = fminf(fmaxf(tn, tk * 0.25f), tk);
+    *gp = __float_as_uint(tn) << 1;
+}
+
 // threshold key, tie cut and next prediction of each unit; clears its histograms
 template <bool RANDK>
 __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     for (uint32_t u = blockIdx.x; u < P.U; u += gridDim.x) {
         const uint32_t uc = tab.c[u];
-        if (uc == 0) continue;
+        if (uc <= tab.short_c) continue;           // no candidates (idle worker), or a block did the unit on its own
         const uint32_t seg = u % P.nseg, r = u / P.nseg, k = P.kseg[seg];
         __syncthreads();
         if (wid == 0) {
@@ -683,23 +764,7 @@ __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32
             out.emin = 255u;
             out.emax = 0u;
             out.norm = 0.0f;
-            if (!RANDK) {
-                // prediction for the next round: move the candidate floor so that about `target`
-                // coordinates pass it, assuming the tail keeps its shape (log-linear in the count)
-                uint32_t* gp = &P.guess[(size_t)r * P.nseg + seg];
-                const float tk = __uint_as_float(tau >> 1), tg = __uint_as_float(*gp >> 1);
-                const float target = (float)P.target[seg];
-                float tn = tg;
-                if (uc > k && tk > tg) {
-                    float ratio = __logf(target / (float)k) / __logf((float)uc / (float)k);
-                    ratio = fminf(fmaxf(ratio, 0.25f), 4.0f);
-                    tn = tk - (tk - tg) * ratio;
-                } else if (uc <= k) {
-                    tn = tk * 0.75f;
-                }
-                tn = fminf(fmaxf(tn, tk * 0.25f), tk);
-                *gp = __float_as_uint(tn) << 1;
-            }
+            if (!RANDK) predict_floor(P, r, seg, tau, uc, k);
         }
     }
 }
@@ -708,8 +773,8 @@ __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32
 template <bool RANDK>
 __device__ void stage_tie_count(const Plan& P, const Tab& tab, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (uint32_t chunk = blockIdx.x; chunk < tab.total_chunks; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+    for (uint32_t chunk = blockIdx.x; chunk < tab.total_long; chunk += gridDim.x) {
+        const ChunkCtx c = long_chunk_context(P, tab, chunk, sh_u);
         if (c.un.tie_t == 0) continue;
         uint32_t cnt = 0;
 #pragma unroll
@@ -723,7 +788,7 @@ __device__ void stage_tie_count(const Plan& P, const Tab& tab, uint32_t* sh_u, u
         if (threadIdx.x == 0) {
             uint32_t t = 0;
             for (int w = 0; w < BT / 32; ++w) t += sh_w[w];
-            P.chunk_cnt[chunk] = t;
+            P.chunk_cnt[c.chunk] = t;
         }
     }
 }
@@ -793,31 +858,107 @@ __device__ __forceinline__ void mark_sender(const Plan& P, uint32_t idx) {
     if (atomicOr(&P.bm1[idx >> 5], bit) & bit) atomicOr(&P.bm2[idx >> 5], bit);
 }
 
-// quantizers that send every kept entry with level 1: nothing about the record depends on the norm
-__device__ __forceinline__ bool qz_early(int qz) { return qz_is_sign(qz) || qz == QS_NONE; }
-
 template <bool RANDK>
 __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t idx) {
     return sk > un.tau || (sk == un.tau && idx <= un.tie_max);
 }
 
-__device__ void unit_norm(const Plan& P, uint32_t u);
+__device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count);
+
+// Exact per-exponent sums in 32-bit words (shared-memory atomics on 32 bits are single
+// instructions): a value below 2^29 is added as its low 16 bits and the rest; with at most
+// UNIT_CAP / 32 additions per word neither can overflow.  acc[e] = {lo16, rest} of the first sum,
+// {lo16, rest} of the second.
+__device__ __forceinline__ void sums_add(uint32_t (*acc)[4], uint32_t e, uint32_t lo, uint32_t hi, bool two) {
+    atomicAdd(&acc[e][0], lo & 0xffffu);
+    atomicAdd(&acc[e][1], lo >> 16);
+    if (two) {
+        atomicAdd(&acc[e][2], hi & 0xffffu);
+        atomicAdd(&acc[e][3], hi >> 16);
+    }
+}
+
+// The same for the lanes of `live`: lanes whose values share an exponent add one sum per warp.
+__device__ __forceinline__ void sums_add_warp(uint32_t (*acc)[4], uint32_t live, uint32_t e, uint32_t lo, uint32_t hi,
+                                              bool two, int lane) {
+    uint32_t rem = live;
+    bool mine = true;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int ld = __ffs(rem) - 1;
+        const uint32_t e0 = __shfl_sync(live, e, ld);
+        const bool in = mine && e == e0;
+        const uint32_t same = __ballot_sync(live, in);
+        // at most 32 values below 2^24: the 32-bit sums are exact
+        const uint32_t slo = __reduce_add_sync(live, in ? lo : 0u);
+        const uint32_t shi = __reduce_add_sync(live, in ? hi : 0u);
+        if (lane == ld) sums_add(acc, e0, slo, shi, two);
+        if (in) mine = false;
+        rem &= ~same;
+        if (!rem) break;
+    }
+    if (mine) sums_add(acc, e, lo, hi, two);
+}
+
+// Norm from per-exponent sums that span at most 12 exponents, each sum below 2^44: the exact sum
+// fits 64 (magnitudes) or 128 (squares) bits, and one conversion rounds it to fp64 (to nearest
+// even).  Other cases take norm_of_sums; both give the correctly rounded exact sum.  The sums are
+// read four exponents at a time, so their reads are in flight together.
+template <class Load>
+__device__ float norm_of_sums_near(uint32_t emin, uint32_t emax, bool l1, Load load) {
+    const int e_lo = emin ? (int)emin : 1;                 // subnormals share the exponent of e = 1
+    unsigned long long tot1 = 0ull;
+    unsigned __int128 tot2 = 0;
+    for (uint32_t eb = emin; eb <= emax; eb += 4) {
+        unsigned long long a0[4], a1[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            a0[j] = 0ull; a1[j] = 0ull;
+            if (eb + j <= emax) load(eb + j, &a0[j], &a1[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t e = eb + j;
+            const int sh = (e ? (int)e : 1) - e_lo;
+            if (l1) tot1 += a0[j] << sh;
+            else tot2 += ((unsigned __int128)a0[j] + ((unsigned __int128)a1[j] << 24)) << (2 * sh);
+        }
+    }
+    double sum;
+    if (l1) {
+        sum = ldexp(__ull2double_rn(tot1), e_lo - 1 - 149);
+    } else {
+        const unsigned long long hi = (unsigned long long)(tot2 >> 64), lo = (unsigned long long)tot2;
+        if (hi == 0ull) {
+            sum = ldexp(__ull2double_rn(lo), 2 * (e_lo - 1) - 298);
+        } else {
+            // the top 64 bits with everything below folded into the lowest one: the conversion then
+            // rounds as if it had seen all the bits
+            const int s = 64 - __clzll(hi);
+            unsigned long long top = (unsigned long long)(tot2 >> s);
+            if ((lo << (64 - s)) != 0ull) top |= 1ull;
+            sum = ldexp(__ull2double_rn(top), s + 2 * (e_lo - 1) - 298);
+        }
+    }
+    return l1 ? __double2float_rn(sum) : __double2float_rn(sqrt(sum));
+}
+
 
 // Per-exponent integer sums of the kept values: for exponent e the squares' 48-bit mantissa
 // products are summed as two 24-bit halves (QSGD), or the 24-bit mantissas themselves (Sign).
 // A 64-bit sum cannot overflow below 2^32 terms.
 template <bool RANDK>
-__device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, unsigned long long (*acc)[2], uint32_t* sh_u,
-                                 uint32_t* sh_w) {
+__device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint32_t (*acc)[4], uint32_t* sh_u,
+                                 uint32_t* sh_w, uint32_t* sh_e) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const uint32_t total = tab.total_chunks;
+    const uint32_t total = tab.total_long;
     const bool plain = P.qz == QS_NONE;            // the plain sparsifier sends the values: no norm
     // merge: a whole round with a quantizer that sends every kept entry at level 1; the counts and
     // the sender bits are known here, and the pack stage does the rest of the quantize stage's work
     const bool early = merge;
     const bool l1 = P.qz == QS_SIGN_L1;
     for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+        const ChunkCtx c = long_chunk_context(P, tab, chunk, sh_u);
         float val[PER];
         uint32_t idx[PER], key[PER];
 #pragma unroll
@@ -828,20 +969,24 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, unsi
             idx[i] = in ? P.cand_idx[c.base + off] : 0xffffffffu;
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
         }
-        acc[threadIdx.x][0] = 0ull;
-        acc[threadIdx.x][1] = 0ull;
+        *reinterpret_cast<uint4*>(acc[threadIdx.x]) = make_uint4(0u, 0u, 0u, 0u);
         uint32_t nkept = 0;                          // lane 0 of each warp counts
         __syncthreads();
+        // sender bits first, all of them: the answers (was the bit set already) are used further down
+        uint32_t seen[PER];
+        bool kept[PER];
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            const bool kept = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
-            const uint32_t live = __ballot_sync(0xffffffffu, kept);
-            if (early) {
-                if (lane == 0) nkept += __popc(live);
-                if (kept) mark_sender(P, idx[i]);
-            }
-            if (kept && !plain) {
+            kept[i] = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
+            seen[i] = 0u;
+            if (early && kept[i]) seen[i] = atomicOr(&P.bm1[idx[i] >> 5], 1u << (idx[i] & 31u)) & (1u << (idx[i] & 31u));
+        }
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const uint32_t live = __ballot_sync(0xffffffffu, kept[i]);
+            if (early && lane == 0) nkept += __popc(live);
+            if (kept[i] && !plain) {
                 const uint32_t b = __float_as_uint(val[i]);
                 const uint32_t e = (b >> 23) & 255u;
                 const uint32_t m = e ? ((b & 0x7fffffu) | 0x800000u) : (b & 0x7fffffu);
@@ -852,36 +997,50 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, unsi
                 // at most 32 values below 2^24: the 32-bit sums are exact
                 const uint32_t slo = __reduce_add_sync(peers, lo);
                 const uint32_t shi = __reduce_add_sync(peers, hi);
-                if (lane == __ffs(peers) - 1) {
-                    atomicAdd(&acc[e][0], (unsigned long long)slo);
-                    if (!l1) atomicAdd(&acc[e][1], (unsigned long long)shi);
-                }
+                if (lane == __ffs(peers) - 1) sums_add(acc, e, slo, shi, !l1);
             }
         }
+#pragma unroll
+        for (int i = 0; i < PER; ++i)
+            if (seen[i]) atomicOr(&P.bm2[idx[i] >> 5], seen[i]);
         if (early && lane == 0) sh_w[wid] = nkept;
         __syncthreads();
         if (early && threadIdx.x == 0) {
             uint32_t t = 0;
             for (int w = 0; w < BT / 32; ++w) t += sh_w[w];
-            P.chunk_cnt[chunk] = t | (t << 16);      // kept | sent << 16
+            P.chunk_cnt[c.chunk] = t | (t << 16);    // kept | sent << 16
         }
         if (plain) continue;
-        const unsigned long long a0 = acc[threadIdx.x][0], a1 = acc[threadIdx.x][1];
+        const uint4 a = *reinterpret_cast<const uint4*>(acc[threadIdx.x]);
+        const unsigned long long a0 = ((unsigned long long)a.y << 16) + a.x, a1 = ((unsigned long long)a.w << 16) + a.z;
         if (a0 | a1) {
             unsigned long long* g = P.eacc + ((size_t)c.u * 256 + threadIdx.x) * 2;
             if (a0) atomicAdd(g, a0);
             if (a1) atomicAdd(g + 1, a1);
-            atomicMin(&P.units[c.u].emin, threadIdx.x);
-            atomicMax(&P.units[c.u].emax, threadIdx.x);
         }
+        // The exponent range of the unit: one update per chunk, and only when the chunk widens the
+        // range it saw on entry.  Every block works on the same few units, and the words of a unit
+        // share a line of the L2 that serves one access at a time.
+        const uint32_t used = __ballot_sync(0xffffffffu, (a0 | a1) != 0ull);
+        if (lane == 0) sh_e[wid] = used;
         // the chunk that completes its unit turns the sums into the norm
         __threadfence();
         __syncthreads();
         if (threadIdx.x == 0) {
+            uint32_t lo_e = 256u, hi_e = 0u;
+            for (int w = 0; w < BT / 32; ++w)
+                if (sh_e[w]) {
+                    const uint32_t first = (uint32_t)w * 32u + (uint32_t)__ffs(sh_e[w]) - 1u, last = (uint32_t)w * 32u + 31u - (uint32_t)__clz(sh_e[w]);
+                    lo_e = lo_e < first ? lo_e : first;
+                    hi_e = hi_e > last ? hi_e : last;
+                }
+            if (lo_e < c.un.emin) atomicMin(&P.units[c.u].emin, lo_e);
+            if (hi_e > c.un.emax) atomicMax(&P.units[c.u].emax, hi_e);
+            __threadfence();
             const uint32_t nch = tab.cb[c.u + 1] - c.cb;
             if (atomicAdd(&P.units[c.u].done, 1u) == nch - 1) {
                 __threadfence();
-                unit_norm(P, c.u);
+                unit_norm(P, c.u, c.c);
                 P.units[c.u].done = 0;
             }
         }
@@ -905,51 +1064,278 @@ __device__ void big_add(uint32_t* dig, int ndig, unsigned long long v, int bitpo
     }
 }
 
-// one thread, once per unit, after every chunk has added its sums: exact sum -> fp64 (round to
-// nearest even) -> norm in fp32.  The sums were built with atomics in the L2: read them there.
-__device__ void unit_norm(const Plan& P, uint32_t u) {
-    {
-        Unit& un = P.units[u];
-        const uint32_t emin = __ldcg(&un.emin), emax = __ldcg(&un.emax);
-        if (emin > emax) return;
-        constexpr int ND = 24;                      // 768 bits
-        uint32_t dig[ND];
-        for (int j = 0; j < ND; ++j) dig[j] = 0;
-        const bool l1 = P.qz == QS_SIGN_L1;
-        // bit 0 stands for 2^-298 (squares) or 2^-149 (magnitudes)
-        for (uint32_t e = emin; e <= emax; ++e) {
-            unsigned long long* g = P.eacc + ((size_t)u * 256 + e) * 2;
-            const unsigned long long a0 = __ldcg(g), a1 = __ldcg(g + 1);
-            if (!(a0 | a1)) continue;
-            g[0] = 0ull; g[1] = 0ull;
-            const int ee = e ? (int)e : 1;          // subnormals share the exponent of e = 1
-            if (l1) {
-                big_add(dig, ND, a0, ee - 1);
-            } else {
-                big_add(dig, ND, a0, 2 * (ee - 1));
-                big_add(dig, ND, a1, 2 * (ee - 1) + 24);
+// Exact sum of the per-exponent integer sums (exponents emin .. emax, read through `load`) ->
+// fp64 (round to nearest even) -> norm in fp32.  One thread.
+template <class Load>
+__device__ float norm_of_sums(uint32_t emin, uint32_t emax, bool l1, Load load) {
+    constexpr int ND = 24;                      // 768 bits
+    uint32_t dig[ND];
+    for (int j = 0; j < ND; ++j) dig[j] = 0;
+    // bit 0 stands for 2^-298 (squares) or 2^-149 (magnitudes)
+    for (uint32_t e = emin; e <= emax; ++e) {
+        unsigned long long a0, a1;
+        load(e, &a0, &a1);
+        if (!(a0 | a1)) continue;
+        const int ee = e ? (int)e : 1;          // subnormals share the exponent of e = 1
+        if (l1) {
+            big_add(dig, ND, a0, ee - 1);
+        } else {
+            big_add(dig, ND, a0, 2 * (ee - 1));
+            big_add(dig, ND, a1, 2 * (ee - 1) + 24);
+        }
+    }
+    int tw = ND - 1;
+    while (tw >= 0 && dig[tw] == 0) --tw;
+    double sum = 0.0;
+    if (tw >= 0) {
+        const int top = tw * 32 + 31 - __clz(dig[tw]);
+        // the 64 bits that start at the top bit (zeros below bit 0), then the 53-bit mantissa
+        const int sh = 31 - (top & 31);                       // left shift that puts the top bit at bit 31
+        const uint32_t w0 = dig[tw], w1 = tw >= 1 ? dig[tw - 1] : 0u, w2 = tw >= 2 ? dig[tw - 2] : 0u;
+        const unsigned long long hi64 = ((unsigned long long)w0 << 32) | w1;
+        const unsigned long long bits = sh ? ((hi64 << sh) | ((unsigned long long)w2 >> (32 - sh))) : hi64;
+        unsigned long long mant = bits >> 11;
+        const uint32_t guard = (uint32_t)(bits >> 10) & 1u;
+        uint32_t sticky = (bits & 0x3ffull) != 0;
+        if (sh && (w2 << sh)) sticky = 1;                     // bits of the third word not shifted in
+        if (!sh && w2) sticky = 1;
+        for (int j = tw - 3; j >= 0 && !sticky; --j) sticky = dig[j] != 0;
+        if (guard && (sticky || (mant & 1ull))) mant += 1ull;
+        sum = ldexp((double)mant, top - 52 - (l1 ? 149 : 298));
+    }
+    return l1 ? __double2float_rn(sum) : __double2float_rn(sqrt(sum));
+}
+
+// one thread, once per unit (of `count` candidates), after every chunk has added its sums.  The
+// sums were built with atomics in the L2: read them there, and leave them zero.
+__device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count) {
+    Unit& un = P.units[u];
+    const uint32_t emin = __ldcg(&un.emin), emax = __ldcg(&un.emax);
+    if (emin > emax) return;
+    const bool l1 = P.qz == QS_SIGN_L1;
+    auto sums = [&](uint32_t e, unsigned long long* a0, unsigned long long* a1) {
+        const unsigned long long* g = P.eacc + ((size_t)u * 256 + e) * 2;
+        *a0 = __ldcg(g);
+        *a1 = __ldcg(g + 1);
+    };
+    // up to 2^20 values of 24 bits per sum: below 2^44
+    un.norm = (emax - emin <= 12u && count <= (1u << 20)) ? norm_of_sums_near(emin, emax, l1, sums)
+                                                           : norm_of_sums(emin, emax, l1, sums);
+    for (uint32_t e = emin; e <= emax; ++e) {
+        unsigned long long* g = P.eacc + ((size_t)u * 256 + e) * 2;
+        g[0] = 0ull;
+        g[1] = 0ull;
+    }
+}
+
+// ------------------------------------------------------------------ short units: one block does it all
+// A unit with a short candidate list is handled by ONE block from threshold to norm with block
+// barriers only, in the shadow of the first grid-wide stage of the long units' select: every list
+// of at most 256 candidates, and every list (up to UNIT_CAP) of a round that has a block per unit.
+// The block keeps the unit's sort keys in registers (UPT per thread).  Up to 256 candidates the
+// kept set comes from ranks counted directly (key descending, list position ascending: the list
+// is in index order); above that from a four-level radix select over a histogram in shared
+// memory.  Then the tie cut, the next prediction, the exact norm (per-exponent sums in shared
+// memory) and, for the quantizers that send every kept entry, the sender bits and the kept counts
+// per chunk.  Units are handed out by a ticket counter, largest first.
+constexpr int UPT = UNIT_CAP / BT;
+static_assert(UNIT_CAP % CHUNK == 0 && UNIT_CAP / CHUNK <= 16, "kept counts per chunk: sixteen slots");
+
+struct UnitSh {                      // lives in the 8 KB scratch of the persistent kernel
+    uint32_t acc[256][4];            // per-exponent sums (sums_add)
+    uint32_t hist[256];
+    uint32_t keys[256];              // rank path: the candidates' keys
+    uint32_t ctl[8];                 // 0 ticket, 1 prefix, 2 rank wanted, 3 keys equal to tau, 4 tie_max, 5 running ties
+    uint32_t kept[16];               // kept entries per chunk
+};
+
+// Calls f(row, position in the list, key, index, value bits) for the rows of BT consecutive
+// candidates of a unit, in order, every thread of the block taking part in every row (f may vote
+// and meet at barriers).  The reads of NB rows are issued together, so a pass costs a round trip
+// to the L2 per NB rows and not per row; for the same reason what f returns (say the old value
+// of an atomic it started) is handed to g only after f has run for all NB rows.  AUX: the index
+// (and for Rand_k the value) is read; without it f gets zeros.
+template <bool RANDK, int NB, bool AUX, class F, class G>
+__device__ __forceinline__ void unit_rows(const Plan& P, size_t base, uint32_t c, const uint32_t (&key)[UPT], F f, G g) {
+    static_assert(UPT % NB == 0, "whole batches of rows");
+#pragma unroll
+    for (int b = 0; b < UPT / NB; ++b) {
+        if ((uint32_t)(b * NB * BT) < c) {
+            uint32_t ix[NB], vq[NB], tok[NB];
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                const uint32_t off = (uint32_t)((b * NB + j) * BT) + threadIdx.x;
+                ix[j] = (AUX && off < c) ? P.cand_idx[base + off] : 0u;
+                vq[j] = (AUX && RANDK && off < c) ? __float_as_uint(P.cand_val[base + off]) : 0u;
+            }
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                tok[j] = 0u;
+                if ((uint32_t)((b * NB + j) * BT) < c)
+                    tok[j] = f((uint32_t)(b * NB + j), (uint32_t)((b * NB + j) * BT) + threadIdx.x, key[b * NB + j], ix[j], vq[j]);
+            }
+#pragma unroll
+            for (int j = 0; j < NB; ++j)
+                if ((uint32_t)((b * NB + j) * BT) < c) g(ix[j], tok[j]);
+        }
+    }
+}
+
+template <bool RANDK>
+__device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, bool early, UnitSh& S, uint32_t* sh_w) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const uint32_t items = (uint32_t)P.nseg * (uint32_t)act.n;
+    const bool plain = P.qz == QS_NONE, l1 = P.qz == QS_SIGN_L1;
+    const uint32_t lt = (1u << lane) - 1u;
+    if (threadIdx.x == 0) S.ctl[0] = atomicAdd(P.bar + 4, 1u);
+    __syncthreads();
+    for (;;) {
+        const uint32_t item = S.ctl[0];
+        __syncthreads();                                   // everyone has read the ticket
+        if (item >= items) break;
+        if (threadIdx.x == 0) S.ctl[0] = atomicAdd(P.bar + 4, 1u);     // the next one: its round trip is off the path
+        const uint32_t seg = P.seg_order[item / (uint32_t)act.n];
+        const uint32_t r = (uint32_t)act.r[item % (uint32_t)act.n];
+        const uint32_t u = r * (uint32_t)P.nseg + seg;
+        const uint32_t c = tab.c[u], k = P.kseg[seg];
+        if (c == 0 || c > tab.short_c) { __syncthreads(); continue; }     // an idle worker's, or a long unit
+        const size_t base = (size_t)r * P.cap + tab.start[u];
+        uint32_t key[UPT];
+#pragma unroll
+        for (int i = 0; i < UPT; ++i) {
+            const uint32_t off = i * BT + threadIdx.x;
+            key[i] = off < c ? sort_key<RANDK>(P, base + off) : 0u;
+        }
+        *reinterpret_cast<uint4*>(S.acc[threadIdx.x]) = make_uint4(0u, 0u, 0u, 0u);
+        if (threadIdx.x < 16) S.kept[threadIdx.x] = 0u;
+        if (threadIdx.x == 0) { S.ctl[4] = 0xffffffffu; S.ctl[5] = 0u; }
+        uint32_t tau, tie_max;
+        if (c <= (uint32_t)BT) {
+            // ranks by direct counting: candidate j comes before this one if its key is larger, or
+            // equal and earlier in the list
+            const uint32_t my_idx = threadIdx.x < c ? P.cand_idx[base + threadIdx.x] : 0u;
+            S.keys[threadIdx.x] = key[0];
+            __syncthreads();
+            uint32_t rank = 0;
+            for (uint32_t j = 0; j < c; ++j) {
+                const uint32_t kj = S.keys[j];
+                rank += (kj > key[0] || (kj == key[0] && j < threadIdx.x)) ? 1u : 0u;
+            }
+            if (threadIdx.x < c && rank == k - 1u) { S.ctl[1] = key[0]; S.ctl[4] = my_idx; }
+            __syncthreads();
+            tau = S.ctl[1];
+            tie_max = S.ctl[4];
+        } else {
+            if (threadIdx.x == 0) { S.ctl[1] = 0u; S.ctl[2] = k; }
+            for (int level = 0; level < 4; ++level) {
+                const int shift = 24 - 8 * level;
+                S.hist[threadIdx.x] = 0u;
+                __syncthreads();
+                const uint32_t prefix = S.ctl[1];
+                unit_rows<RANDK, 16, false>(P, base, c, key, [&](uint32_t, uint32_t off, uint32_t kv, uint32_t, uint32_t) {
+                    const bool valid = off < c && (level == 0 || (kv >> (32 - 8 * level)) == prefix);
+                    const uint32_t digit = (kv >> shift) & 255u;
+                    const uint32_t live = __ballot_sync(0xffffffffu, valid);
+                    if (valid) {
+                        const uint32_t peers = __match_any_sync(live, digit);
+                        if (lane == __ffs(peers) - 1) atomicAdd(&S.hist[digit], __popc(peers));
+                    }
+                    return 0u;
+                }, [](uint32_t, uint32_t) {});
+                __syncthreads();
+                if (wid == 0) {
+                    uint32_t bin, above;
+                    find_bin(S.hist, S.ctl[2], lane, &bin, &above);
+                    if (lane == 0) {
+                        S.ctl[1] = (prefix << 8) | bin;
+                        S.ctl[2] -= above;
+                        S.ctl[3] = S.hist[bin];
+                    }
+                }
+                __syncthreads();
+            }
+            tau = S.ctl[1];
+            const uint32_t t = S.ctl[2], ceq = S.ctl[3];
+            if (ceq > t) {
+                // more equal keys than slots: the t earliest in the list win
+                unit_rows<RANDK, 8, true>(P, base, c, key, [&](uint32_t, uint32_t off, uint32_t kv, uint32_t idx, uint32_t) {
+                    const bool eq = off < c && kv == tau;
+                    const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+                    if (lane == 0) sh_w[wid] = __popc(bal);
+                    __syncthreads();
+                    uint32_t before = S.ctl[5], row = 0;
+                    for (int w = 0; w < BT / 32; ++w) { if (w < wid) before += sh_w[w]; row += sh_w[w]; }
+                    const uint32_t mine = before + __popc(bal & lt);
+                    if (eq && mine == t - 1u) S.ctl[4] = idx;
+                    __syncthreads();
+                    if (threadIdx.x == 0) S.ctl[5] += row;
+                    return 0u;
+                }, [](uint32_t, uint32_t) {});
+                if (S.ctl[4] == 0xffffffffu) set_status(P, QS_STATE);     // the counts said it is there
+            }
+            tie_max = S.ctl[4];
+        }
+        // the level-0 counts of the order stage are not needed on this path: leave them zero
+        P.hist[(size_t)u * 256 + threadIdx.x] = 0u;
+        // kept entries: exact sums per exponent, sender bits and kept counts per chunk
+        const bool ties = tie_max != 0xffffffffu;
+        auto take = [&](uint32_t i, uint32_t off, uint32_t kv, uint32_t idx, uint32_t vb) {
+            const bool kept = off < c && kv >= tau && !(ties && kv == tau && idx > tie_max);
+            const uint32_t live = __ballot_sync(0xffffffffu, kept);
+            uint32_t seen = 0u;                      // was the coordinate's bit set already (another worker sent it)
+            if (early) {
+                if (lane == 0 && live) atomicAdd(&S.kept[i / PER], __popc(live));
+                if (kept) seen = atomicOr(&P.bm1[idx >> 5], 1u << (idx & 31u)) & (1u << (idx & 31u));
+            }
+            if (kept && !plain) {
+                const uint32_t b = RANDK ? vb : (kv >> 1);
+                const uint32_t e = (b >> 23) & 255u;
+                const uint32_t m = e ? ((b & 0x7fffffu) | 0x800000u) : (b & 0x7fffffu);
+                uint32_t lo, hi;
+                if (l1) { lo = m; hi = 0; }
+                else { const unsigned long long sq = (unsigned long long)m * m; lo = (uint32_t)(sq & 0xffffffu); hi = (uint32_t)(sq >> 24); }
+                sums_add_warp(S.acc, live, e, lo, hi, !l1, lane);
+            }
+            return seen;
+        };
+        auto twice = [&](uint32_t idx, uint32_t seen) { if (seen) atomicOr(&P.bm2[idx >> 5], seen); };
+        // the indices are needed for the sender bits and for a tie cut; Rand_k reads the values too
+        if (early || ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, twice);
+        else unit_rows<RANDK, 16, false>(P, base, c, key, take, twice);
+        __syncthreads();
+        if (wid == 0) {
+            // exponent range of the sums
+            uint32_t lo_e = 256u, hi_e = 0u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t e = (uint32_t)lane * 8u + j;
+                const uint4 a = *reinterpret_cast<const uint4*>(S.acc[e]);
+                if (a.x | a.y | a.z | a.w) { lo_e = lo_e < e ? lo_e : e; hi_e = e; }
+            }
+            lo_e = __reduce_min_sync(0xffffffffu, lo_e);
+            hi_e = __reduce_max_sync(0xffffffffu, hi_e);
+            if (lane == 0) {
+                Unit& out = P.units[u];
+                out.tau = tau;
+                out.tie_max = tie_max;
+                out.tie_t = 0;
+                out.n = 0;
+                out.emin = 255u;
+                out.emax = 0u;
+                auto sums = [&](uint32_t e, unsigned long long* a0, unsigned long long* a1) {
+                    *a0 = ((unsigned long long)S.acc[e][1] << 16) + S.acc[e][0];
+                    *a1 = ((unsigned long long)S.acc[e][3] << 16) + S.acc[e][2];
+                };
+                out.norm = (plain || lo_e > hi_e) ? 0.0f
+                         : hi_e - lo_e <= 12u ? norm_of_sums_near(lo_e, hi_e, l1, sums) : norm_of_sums(lo_e, hi_e, l1, sums);
+                if (!RANDK) predict_floor(P, r, seg, tau, c, k);
+                if (early) {
+                    const uint32_t c0 = tab.cb[u], nch = tab.cb[u + 1] - c0;
+                    for (uint32_t j = 0; j < nch; ++j) P.chunk_cnt[c0 + j] = S.kept[j] | (S.kept[j] << 16);
+                }
             }
         }
-        int tw = ND - 1;
-        while (tw >= 0 && dig[tw] == 0) --tw;
-        double sum = 0.0;
-        if (tw >= 0) {
-            const int top = tw * 32 + 31 - __clz(dig[tw]);
-            // the 64 bits that start at the top bit (zeros below bit 0), then the 53-bit mantissa
-            const int sh = 31 - (top & 31);                       // left shift that puts the top bit at bit 31
-            const uint32_t w0 = dig[tw], w1 = tw >= 1 ? dig[tw - 1] : 0u, w2 = tw >= 2 ? dig[tw - 2] : 0u;
-            const unsigned long long hi64 = ((unsigned long long)w0 << 32) | w1;
-            const unsigned long long bits = sh ? ((hi64 << sh) | ((unsigned long long)w2 >> (32 - sh))) : hi64;
-            unsigned long long mant = bits >> 11;
-            const uint32_t guard = (uint32_t)(bits >> 10) & 1u;
-            uint32_t sticky = (bits & 0x3ffull) != 0;
-            if (sh && (w2 << sh)) sticky = 1;                     // bits of the third word not shifted in
-            if (!sh && w2) sticky = 1;
-            for (int j = tw - 3; j >= 0 && !sticky; --j) sticky = dig[j] != 0;
-            if (guard && (sticky || (mant & 1ull))) mant += 1ull;
-            sum = ldexp((double)mant, top - 52 - (l1 ? 149 : 298));
-        }
-        un.norm = l1 ? __double2float_rn(sum) : __double2float_rn(sqrt(sum));
+        __syncthreads();
     }
 }
 
@@ -1168,16 +1554,21 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge
                 if (i < chunk) { sums[0] += v & 0xffffu; sums[1] += v >> 16; }
             }
             block_sum4(sums, sh);
-            run_k = sums[0]; run_s = sums[1]; unit_n = sums[3]; pay = 2u;
+            run_k = sums[0]; run_s = sums[1]; unit_n = sums[3];
+            pay = P.nseg == 1 ? 2u : P.pay_off[c.u];          // several segments: every kept entry is sent, fixed places
             if (chunk == c.cb && threadIdx.x == 0) {          // the unit's first chunk writes its directory entry
                 P.units[c.u].n = unit_n;
                 if (sums[2] != P.kseg[c.seg]) set_status(P, QS_STATE);
                 uint32_t* row = wire + (size_t)c.r * stride;
-                row[0] = unit_n;
-                row[1] = __float_as_uint(c.un.norm);
-                const long long bits = 64 + (long long)unit_n * entry_bits(bi, (uint32_t)P.bl, P.qz);
-                P.bits[c.r] = bits;
-                if (bits_out) bits_out[c.r] = bits;
+                row[2 * c.seg] = unit_n;
+                row[2 * c.seg + 1] = __float_as_uint(c.un.norm);
+                if (P.nseg == 1) {
+                    const long long bits = 64 + (long long)unit_n * entry_bits(bi, (uint32_t)P.bl, P.qz);
+                    P.bits[c.r] = bits;
+                    if (bits_out) bits_out[c.r] = bits;
+                } else if (c.seg == 0 && bits_out) {
+                    bits_out[c.r] = P.bits[c.r];
+                }
             }
         } else {
             run_k = P.chunk_sel[chunk] - P.chunk_sel[c.cb];
@@ -1489,15 +1880,18 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_small[8];              // unit id, prefix, select scratch
     __shared__ uint32_t sh_w[BT / 32];
     __shared__ uint32_t sh_cnt[2 * 8 * GPW];
-    __shared__ uint32_t sh_flag;
+    __shared__ uint32_t sh_flag[4];
     __shared__ int sh_abort;
     // unit table (three arrays) / candidate-count sums of the order stage / tile buffers of the broadcast
     __shared__ __align__(128) uint32_t sh_tab[ORDER_ITEMS_MAX + 8];
     uint32_t* t_start = sh_tab;
     uint32_t* t_c = sh_tab + UT_MAX;
     uint32_t* t_cb = sh_tab + 2 * UT_MAX;         // UT_MAX + 1 entries
+    uint32_t* t_lb = sh_tab + 3 * UT_MAX + 4;     // UT_MAX + 1 entries
+    static_assert(4 * UT_MAX + 5 <= ORDER_ITEMS_MAX + 8, "the unit table must fit");
     __shared__ __align__(8) uint64_t sh_mbar[3];
-    __shared__ __align__(16) unsigned char sh_big[FB_BINS * 4];   // fallback bins / radix bins / exponent sums
+    __shared__ __align__(16) unsigned char sh_big[FB_BINS * 4];   // fallback bins / radix bins / exponent sums / UnitSh
+    static_assert(sizeof(UnitSh) <= FB_BINS * 4, "the unit stage's scratch must fit");
     const Plan& P = a.P;
     const Active& act = a.act;
     uint32_t* bins = reinterpret_cast<uint32_t*>(sh_big);
@@ -1530,7 +1924,7 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         if (even) stage_order_even<RANDK>(P, act, 0u, bins, sh_tab, sh_scan);
         else stage_order<RANDK>(P, act, 0u, bins);
         QS_BARRIER();
-        const uint32_t missed = build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
+        const uint32_t missed = build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab);
         if (missed) {                              // the same value in every block
             stage_fb_hist<RANDK>(P, act, missed, bins);
             QS_BARRIER();
@@ -1541,7 +1935,7 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
             if (even) stage_order_even<RANDK>(P, act, missed, bins, sh_tab, sh_scan);
             else stage_order<RANDK>(P, act, missed, bins);
             QS_BARRIER();
-            if (build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab)) set_status(P, QS_STATE);   // the exact pass cannot miss
+            if (build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab)) set_status(P, QS_STATE);   // the exact pass cannot miss
             if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd((unsigned long long*)&P.stats[0], (unsigned long long)__popc(missed));
         }
         if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -1552,20 +1946,27 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         // the candidate counts have been consumed: clear them for the next dense pass
         for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nblk; i += gridDim.x * BT) P.blk_count[i] = 0;
         for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nsup; i += gridDim.x * BT) P.sup_count[i] = 0;
-        for (int level = 1; level < 4; ++level) {
-            stage_hist<RANDK>(P, tab, level, bins, &sh_small[0], &sh_small[1]);
+        // select: the first radix level of the long units, and the short units whole, block by block
+        if (tab.total_long) stage_hist<RANDK>(P, tab, 1, bins, &sh_small[0], &sh_small[1]);
+        __syncthreads();                           // the scratch changes hands
+        if (tab.any_short) stage_unit<RANDK>(P, tab, act, merge, *reinterpret_cast<UnitSh*>(sh_big), sh_w);
+        QS_BARRIER();
+        if (tab.total_long) {
+            for (int level = 2; level < 4; ++level) {
+                stage_hist<RANDK>(P, tab, level, bins, &sh_small[0], &sh_small[1]);
+                QS_BARRIER();
+            }
+            stage_final<RANDK>(P, tab, &sh_small[2], sh_w);
+            QS_BARRIER();
+            if (P.fail[0]) {                       // some long list has more equal keys than slots (same in every block)
+                stage_tie_count<RANDK>(P, tab, &sh_small[0], sh_w);
+                QS_BARRIER();
+                stage_tie_find<RANDK>(P, tab, sh_scan, &sh_small[2], sh_w);
+                QS_BARRIER();
+            }
+            stage_norm_accum<RANDK>(P, tab, merge, reinterpret_cast<uint32_t(*)[4]>(sh_big), &sh_small[0], sh_w, sh_cnt);
             QS_BARRIER();
         }
-        stage_final<RANDK>(P, tab, &sh_small[2], sh_w);
-        QS_BARRIER();
-        if (P.fail[0]) {                           // some long list has more equal keys than slots (same in every block)
-            stage_tie_count<RANDK>(P, tab, &sh_small[0], sh_w);
-            QS_BARRIER();
-            stage_tie_find<RANDK>(P, tab, sh_scan, &sh_small[2], sh_w);
-            QS_BARRIER();
-        }
-        stage_norm_accum<RANDK>(P, tab, merge, reinterpret_cast<unsigned long long(*)[2]>(sh_big), &sh_small[0], sh_w);
-        QS_BARRIER();
         if (!merge) {
             stage_quant<RANDK>(P, tab, fused, &sh_small[0], sh_w);
             QS_BARRIER();
@@ -1575,7 +1976,7 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
             QS_BARRIER();
         }
     } else if (a.do_pack) {
-        build_table(P, act, t_start, t_c, t_cb, sh_scan, &sh_flag, &tab);
+        build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab);
         QS_BARRIER();                              // the zeroed records
     }
     if (a.do_pack) {
@@ -1618,6 +2019,7 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
             P.bar[1] = 0;
             P.bar[2] = 0;                            // tile tickets of the broadcast
             P.bar[3] = 0;                            // tile tickets of the next dense pass
+            P.bar[4] = 0;                            // unit tickets
             *P.ncoll = 0;
         }
     }

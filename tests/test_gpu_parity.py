@@ -25,6 +25,18 @@ def setup_module(module):
     B = binding
 
 
+@pytest.fixture(autouse=True, params=["per_unit", "per_level"])
+def selection_path(request, monkeypatch):
+    # Rounds whose units are all short run the threshold, tie cut and norm of a unit inside one
+    # block; QSPARSE_UNIT_CAP=0 (read by qs_init) sends them through the grid-wide radix levels
+    # that long candidate lists take.  Every case below runs both ways.
+    if request.param == "per_level":
+        monkeypatch.setenv("QSPARSE_UNIT_CAP", "0")
+    else:
+        monkeypatch.delenv("QSPARSE_UNIT_CAP", raising=False)
+    yield request.param
+
+
 def bits_equal(a, b):
     a = np.ascontiguousarray(a)
     b = np.ascontiguousarray(b)
@@ -139,16 +151,17 @@ def test_small_and_ragged_sizes(d, k, sp, qz):
     p.close()
 
 
-def test_ties_zeros_and_equal_values():
-    R, d = 2, 5000
+@pytest.mark.parametrize("d", [200, 3000, 5000])     # lists of at most 256, 4096 and more candidates: the three per-unit forms
+def test_ties_zeros_and_equal_values(d):
+    R = 2
     cases = []
     z = np.zeros((R, d), np.float32)
-    cases.append((np.zeros(d, np.float32), z.copy(), z.copy(), 50))                  # everything zero
+    cases.append((np.zeros(d, np.float32), z.copy(), z.copy(), d // 100))             # everything zero
     eq = np.full((R, d), 0.25, np.float32)
-    cases.append((np.zeros(d, np.float32), -eq, z.copy(), 77))                        # all equal
+    cases.append((np.zeros(d, np.float32), -eq, z.copy(), d // 65 + 1))               # all equal
     g = np.random.default_rng(3)
     few = g.choice(np.array([0.0, 1.0, -1.0, 2.0, -0.0], np.float32), size=(R, d)).astype(np.float32)
-    cases.append((np.zeros(d, np.float32), few, z.copy(), 1200))                      # five distinct values
+    cases.append((np.zeros(d, np.float32), few, z.copy(), d * 6 // 25))               # five distinct values
     for x, xw, mem, k in cases:
         for qz in (O.QSGD, O.SIGN_L1):
             p = Pair(R, d, k=k, s=16, quantizer=qz, seed=1, x=x, xw=xw, mem=mem)
