@@ -19,6 +19,8 @@
 //               order, updates x and (fused round) patches the workers' copies
 //
 // Order-dependent results come only from ordered scans, never from the order of atomics.
+#include <cstdlib>
+
 #include "qs_bulk.cuh"
 #include "qs_kernels.h"
 
@@ -164,14 +166,17 @@ __device__ void stage_order(const Plan& P, const Active& act, uint32_t only_mask
                     if (RANDK) P.cand_key[row + base + e] = sk;
                     seg = segment_of(P, idx);
                 }
-                // level 0 of the radix select: count the top key byte per unit
-                const uint32_t tag = (seg << 8) | (sk >> 24);
-                const uint32_t live = __ballot_sync(0xffffffffu, valid);
-                if (valid) {
-                    const uint32_t peers = __match_any_sync(live, tag);
-                    if (lane == __ffs(peers) - 1) {
-                        if (local_bins) atomicAdd(&sh_bins[wslot * 256 + (sk >> 24)], __popc(peers));
-                        else atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
+                // level 0 of the radix select: count the top key byte per unit.  Shared memory takes
+                // an add per lane as it comes (equal addresses cost nothing extra there); adds to
+                // global memory are gathered per warp first
+                if (local_bins) {
+                    if (valid) atomicAdd(&sh_bins[wslot * 256 + (sk >> 24)], 1u);
+                } else {
+                    const uint32_t tag = (seg << 8) | (sk >> 24);
+                    const uint32_t live = __ballot_sync(0xffffffffu, valid);
+                    if (valid) {
+                        const uint32_t peers = __match_any_sync(live, tag);
+                        if (lane == __ffs(peers) - 1) atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
                     }
                 }
             }
@@ -343,15 +348,15 @@ __device__ void stage_order_even(const Plan& P, const Active& act, uint32_t only
                         if (RANDK) P.cand_key[o] = sk;
                         seg = segment_of(P, idx);
                     }
-                    // level 0 of the radix select: count the top key byte per unit
+                    // level 0 of the radix select: count the top key byte per unit (shared memory: an add
+                    // per lane; global memory: gathered per warp first)
+                    const bool local = local_bins && wsl[q] - ws0 < 8u;
+                    if (valid && local) atomicAdd(&sh_bins[(wsl[q] - ws0) * 256 + (sk >> 24)], 1u);
                     const uint32_t tag = (wsl[q] << 24) | (seg << 8) | (sk >> 24);
-                    const uint32_t live = __ballot_sync(0xffffffffu, valid);
-                    if (valid) {
+                    const uint32_t live = __ballot_sync(0xffffffffu, valid && !local);
+                    if (valid && !local) {
                         const uint32_t peers = __match_any_sync(live, tag);
-                        if (lane == __ffs(peers) - 1) {
-                            if (local_bins && wsl[q] - ws0 < 8u) atomicAdd(&sh_bins[(wsl[q] - ws0) * 256 + (sk >> 24)], __popc(peers));
-                            else atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
-                        }
+                        if (lane == __ffs(peers) - 1) atomicAdd(&P.hist[((size_t)r * P.nseg + seg) * 256 + (sk >> 24)], __popc(peers));
                     }
                 }
             }
@@ -460,14 +465,10 @@ __device__ void stage_fb_hist(const Plan& P, const Active& act, uint32_t missed,
         const size_t row = (size_t)r * P.d;
         for (uint32_t base = 0; base < blk.len; base += BT) {
             const uint32_t i = base + threadIdx.x;
-            const bool valid = i < blk.len;
-            const uint32_t live = __ballot_sync(0xffffffffu, valid);
-            if (valid) {
+            if (i < blk.len) {
                 const uint32_t e = blk.start + i;
                 const uint32_t sk = RANDK ? ~philox_word(P, (uint32_t)r, e, 1u) : topk_key(P.mem[row + e]);
-                const uint32_t bin = sk >> FB_SHIFT;
-                const uint32_t peers = __match_any_sync(live, bin);
-                if ((threadIdx.x & 31) == (uint32_t)(__ffs(peers) - 1)) atomicAdd(&sh_bins[bin], __popc(peers));
+                atomicAdd(&sh_bins[sk >> FB_SHIFT], 1u);
             }
         }
         __syncthreads();
@@ -676,12 +677,7 @@ __device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* s
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
             const bool valid = off < c.c && (level == 0 || (sk[i] >> (32 - 8 * level)) == prefix);
-            const uint32_t digit = (sk[i] >> shift) & 255u;
-            const uint32_t live = __ballot_sync(0xffffffffu, valid);
-            if (valid) {
-                const uint32_t peers = __match_any_sync(live, digit);
-                if (lane == __ffs(peers) - 1) atomicAdd(&sh_hist[digit], __popc(peers));
-            }
+            if (valid) atomicAdd(&sh_hist[(sk[i] >> shift) & 255u], 1u);
         }
         __syncthreads();
         const uint32_t v = sh_hist[threadIdx.x];
@@ -865,10 +861,11 @@ __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t id
 
 __device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count);
 
-// Exact per-exponent sums in 32-bit words (shared-memory atomics on 32 bits are single
-// instructions): a value below 2^29 is added as its low 16 bits and the rest; with at most
-// UNIT_CAP / 32 additions per word neither can overflow.  acc[e] = {lo16, rest} of the first sum,
-// {lo16, rest} of the second.
+// Exact per-exponent sums in 32-bit words of shared memory, one add per value and word (adds to
+// shared memory are single instructions on 32 bits, and equal addresses within a warp cost nothing
+// extra, so nothing is gathered per warp first): a value below 2^24 is added as its low 16 bits
+// and the rest; with at most UNIT_CAP additions per word neither can overflow.  acc[e] = {lo16,
+// rest} of the first sum, {lo16, rest} of the second.
 __device__ __forceinline__ void sums_add(uint32_t (*acc)[4], uint32_t e, uint32_t lo, uint32_t hi, bool two) {
     atomicAdd(&acc[e][0], lo & 0xffffu);
     atomicAdd(&acc[e][1], lo >> 16);
@@ -876,28 +873,6 @@ __device__ __forceinline__ void sums_add(uint32_t (*acc)[4], uint32_t e, uint32_
         atomicAdd(&acc[e][2], hi & 0xffffu);
         atomicAdd(&acc[e][3], hi >> 16);
     }
-}
-
-// The same for the lanes of `live`: lanes whose values share an exponent add one sum per warp.
-__device__ __forceinline__ void sums_add_warp(uint32_t (*acc)[4], uint32_t live, uint32_t e, uint32_t lo, uint32_t hi,
-                                              bool two, int lane) {
-    uint32_t rem = live;
-    bool mine = true;
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int ld = __ffs(rem) - 1;
-        const uint32_t e0 = __shfl_sync(live, e, ld);
-        const bool in = mine && e == e0;
-        const uint32_t same = __ballot_sync(live, in);
-        // at most 32 values below 2^24: the 32-bit sums are exact
-        const uint32_t slo = __reduce_add_sync(live, in ? lo : 0u);
-        const uint32_t shi = __reduce_add_sync(live, in ? hi : 0u);
-        if (lane == ld) sums_add(acc, e0, slo, shi, two);
-        if (in) mine = false;
-        rem &= ~same;
-        if (!rem) break;
-    }
-    if (mine) sums_add(acc, e, lo, hi, two);
 }
 
 // Norm from per-exponent sums that span at most 12 exponents, each sum below 2^44: the exact sum
@@ -993,11 +968,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
                 uint32_t lo, hi;
                 if (l1) { lo = m; hi = 0; }
                 else { const unsigned long long sq = (unsigned long long)m * m; lo = (uint32_t)(sq & 0xffffffu); hi = (uint32_t)(sq >> 24); }
-                const uint32_t peers = __match_any_sync(live, e);
-                // at most 32 values below 2^24: the 32-bit sums are exact
-                const uint32_t slo = __reduce_add_sync(peers, lo);
-                const uint32_t shi = __reduce_add_sync(peers, hi);
-                if (lane == __ffs(peers) - 1) sums_add(acc, e, slo, shi, !l1);
+                sums_add(acc, e, lo, hi, !l1);
             }
         }
 #pragma unroll
@@ -1234,12 +1205,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
                 const uint32_t prefix = S.ctl[1];
                 unit_rows<RANDK, 16, false>(P, base, c, key, [&](uint32_t, uint32_t off, uint32_t kv, uint32_t, uint32_t) {
                     const bool valid = off < c && (level == 0 || (kv >> (32 - 8 * level)) == prefix);
-                    const uint32_t digit = (kv >> shift) & 255u;
-                    const uint32_t live = __ballot_sync(0xffffffffu, valid);
-                    if (valid) {
-                        const uint32_t peers = __match_any_sync(live, digit);
-                        if (lane == __ffs(peers) - 1) atomicAdd(&S.hist[digit], __popc(peers));
-                    }
+                    if (valid) atomicAdd(&S.hist[(kv >> shift) & 255u], 1u);
                     return 0u;
                 }, [](uint32_t, uint32_t) {});
                 __syncthreads();
@@ -1294,7 +1260,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
                 uint32_t lo, hi;
                 if (l1) { lo = m; hi = 0; }
                 else { const unsigned long long sq = (unsigned long long)m * m; lo = (uint32_t)(sq & 0xffffffu); hi = (uint32_t)(sq >> 24); }
-                sums_add_warp(S.acc, live, e, lo, hi, !l1, lane);
+                sums_add(S.acc, e, lo, hi, !l1);
             }
             return seen;
         };
@@ -2058,6 +2024,8 @@ cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do
     a.wire = wire; a.stride = stride; a.wire_words = wire_words; a.bits_out = bits_out;
     void* params[] = {&a};
     const void* fn = P.sp == QS_RANDK ? (const void*)mid_kernel<true> : (const void*)mid_kernel<false>;
+    static const bool plain = getenv("QSPARSE_PLAIN_LAUNCH") != nullptr;
+    if (plain) return cudaLaunchKernel(fn, dim3(grid), dim3(BT), params, 0, st);
     return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(BT), params, 0, st);
 }
 
