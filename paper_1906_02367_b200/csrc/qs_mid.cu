@@ -11,7 +11,8 @@
 //               short (histogram of the top key bits, new threshold, candidates found again from
 //               the stored u)
 //   select      radix select over the 32-bit sort key (4 levels of 8 bits), tie cut by lower
-//               index, next round's prediction
+//               index, next round's prediction; units with short candidate lists are selected
+//               from by one block each, with block barriers only, beside the first level
 //   quantize    exact norm of the kept values, levels and signs (Philox stream 0), m <- u - g,
 //               ordered positions of kept and sent entries
 //   pack        directory and the three bit streams of every segment
@@ -19,8 +20,6 @@
 //               order, updates x and (fused round) patches the workers' copies
 //
 // Order-dependent results come only from ordered scans, never from the order of atomics.
-#include <cstdlib>
-
 #include "qs_bulk.cuh"
 #include "qs_kernels.h"
 
@@ -2024,8 +2023,6 @@ cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do
     a.wire = wire; a.stride = stride; a.wire_words = wire_words; a.bits_out = bits_out;
     void* params[] = {&a};
     const void* fn = P.sp == QS_RANDK ? (const void*)mid_kernel<true> : (const void*)mid_kernel<false>;
-    static const bool plain = getenv("QSPARSE_PLAIN_LAUNCH") != nullptr;
-    if (plain) return cudaLaunchKernel(fn, dim3(grid), dim3(BT), params, 0, st);
     return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(BT), params, 0, st);
 }
 
