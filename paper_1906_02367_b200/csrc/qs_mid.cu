@@ -605,16 +605,19 @@ __device__ void derive_prefix(const Plan& P, uint32_t u, uint32_t k, int level, 
     *above_total = at;
 }
 
-struct ChunkCtx { uint32_t u, r, seg, first, c, cb, chunk; Unit un; size_t base; };   // chunk: its number among all chunks
+struct ChunkCtx { uint32_t u = 0xffffffffu, r, seg, first, c, cb, chunk; Unit un; size_t base; };   // chunk: its number among all chunks
 
 // which unit a chunk belongs to (one search per block, shared through sh_u)
-__device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, const Tab& tab, uint32_t chunk, uint32_t* sh_u) {
+// `last`: the context of the block's previous chunk in this stage; a block's consecutive chunks
+// mostly lie in one unit, whose record (unchanged within a stage) is then not read again.
+__device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, const Tab& tab, uint32_t chunk, uint32_t* sh_u,
+                                                  const ChunkCtx* last = nullptr) {
     __syncthreads();
     if (threadIdx.x == 0) *sh_u = unit_of_chunk(P, tab, chunk);
     __syncthreads();
     ChunkCtx c;
     c.u = *sh_u;
-    c.un = P.units[c.u];
+    if (last && last->u == c.u) c.un = last->un; else c.un = P.units[c.u];
     c.r = c.u / P.nseg;
     c.seg = c.u % P.nseg;
     c.c = tab.c[c.u];
@@ -626,7 +629,8 @@ __device__ __forceinline__ ChunkCtx chunk_context(const Plan& P, const Tab& tab,
 }
 
 // the same for chunk q of the long units only (the stages of the grid-wide select walk these)
-__device__ __forceinline__ ChunkCtx long_chunk_context(const Plan& P, const Tab& tab, uint32_t q, uint32_t* sh_u) {
+__device__ __forceinline__ ChunkCtx long_chunk_context(const Plan& P, const Tab& tab, uint32_t q, uint32_t* sh_u,
+                                                       const ChunkCtx* last = nullptr) {
     __syncthreads();
     if (threadIdx.x == 0) {
         uint32_t lo = 0, hi = P.U;               // the last unit with lb <= q: short units before it share its lb
@@ -639,7 +643,7 @@ __device__ __forceinline__ ChunkCtx long_chunk_context(const Plan& P, const Tab&
     __syncthreads();
     ChunkCtx c;
     c.u = *sh_u;
-    c.un = P.units[c.u];
+    if (last && last->u == c.u) c.un = last->un; else c.un = P.units[c.u];
     c.r = c.u / P.nseg;
     c.seg = c.u % P.nseg;
     c.c = tab.c[c.u];
@@ -650,38 +654,51 @@ __device__ __forceinline__ ChunkCtx long_chunk_context(const Plan& P, const Tab&
     return c;
 }
 
-// one level of the radix select: histogram of the level's digit among keys matching the prefix
+// one level of the radix select: histogram of the level's digit among keys matching the prefix.
+// A block takes consecutive chunks; while they lie in one unit the prefix is worked out once and
+// the counts stay in shared memory, to be added to the unit's histogram in one go.
 template <bool RANDK>
 __device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* sh_hist, uint32_t* sh_u, uint32_t* sh_prefix) {
     const int lane = threadIdx.x & 31;
     const uint32_t total = tab.total_long;
     const int shift = 24 - 8 * level;
-    for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = long_chunk_context(P, tab, chunk, sh_u);
+    const uint32_t share = (total + gridDim.x - 1) / gridDim.x;
+    const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
+    uint32_t held = 0xffffffffu, prefix = 0;
+    auto flush = [&]() {
+        __syncthreads();                              // every add of the held chunks has been made
+        const uint32_t v = sh_hist[threadIdx.x];
+        if (v) atomicAdd(&P.hist[((size_t)level * P.U + held) * 256 + threadIdx.x], v);
+    };
+    ChunkCtx c;
+    for (uint32_t chunk = c_lo; chunk < c_hi; ++chunk) {
+        c = long_chunk_context(P, tab, chunk, sh_u, &c);
         uint32_t sk[PER];
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
             sk[i] = off < c.c ? sort_key<RANDK>(P, c.base + off) : 0u;
         }
-        if (threadIdx.x < 32) {
-            uint32_t prefix, at;
-            derive_prefix(P, c.u, P.kseg[c.seg], level, lane, &prefix, &at);
-            if (lane == 0) *sh_prefix = prefix;
+        if (c.u != held) {
+            if (held != 0xffffffffu) flush();
+            held = c.u;
+            if (threadIdx.x < 32) {
+                uint32_t pf, at;
+                derive_prefix(P, c.u, P.kseg[c.seg], level, lane, &pf, &at);
+                if (lane == 0) *sh_prefix = pf;
+            }
+            sh_hist[threadIdx.x] = 0;
+            __syncthreads();
+            prefix = *sh_prefix;
         }
-        sh_hist[threadIdx.x] = 0;
-        __syncthreads();
-        const uint32_t prefix = *sh_prefix;
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
             const bool valid = off < c.c && (level == 0 || (sk[i] >> (32 - 8 * level)) == prefix);
             if (valid) atomicAdd(&sh_hist[(sk[i] >> shift) & 255u], 1u);
         }
-        __syncthreads();
-        const uint32_t v = sh_hist[threadIdx.x];
-        if (v) atomicAdd(&P.hist[((size_t)level * P.U + c.u) * 256 + threadIdx.x], v);
     }
+    if (held != 0xffffffffu) flush();
 }
 
 // Prediction for the next round (Top_k): move the candidate floor so that about `target`
@@ -768,8 +785,9 @@ __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32
 template <bool RANDK>
 __device__ void stage_tie_count(const Plan& P, const Tab& tab, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    ChunkCtx c;
     for (uint32_t chunk = blockIdx.x; chunk < tab.total_long; chunk += gridDim.x) {
-        const ChunkCtx c = long_chunk_context(P, tab, chunk, sh_u);
+        c = long_chunk_context(P, tab, chunk, sh_u, &c);
         if (c.un.tie_t == 0) continue;
         uint32_t cnt = 0;
 #pragma unroll
@@ -858,12 +876,12 @@ __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t id
     return sk > un.tau || (sk == un.tau && idx <= un.tie_max);
 }
 
-__device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count);
+__device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count, uint32_t (*sh)[4]);
 
 // Exact per-exponent sums in 32-bit words of shared memory, one add per value and word (adds to
 // shared memory are single instructions on 32 bits, and equal addresses within a warp cost nothing
 // extra, so nothing is gathered per warp first): a value below 2^24 is added as its low 16 bits
-// and the rest; with at most UNIT_CAP additions per word neither can overflow.  acc[e] = {lo16,
+// and the rest; with at most 2^15 additions per word neither can overflow.  acc[e] = {lo16,
 // rest} of the first sum, {lo16, rest} of the second.
 __device__ __forceinline__ void sums_add(uint32_t (*acc)[4], uint32_t e, uint32_t lo, uint32_t hi, bool two) {
     atomicAdd(&acc[e][0], lo & 0xffffu);
@@ -931,8 +949,58 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
     // the sender bits are known here, and the pack stage does the rest of the quantize stage's work
     const bool early = merge;
     const bool l1 = P.qz == QS_SIGN_L1;
-    for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = long_chunk_context(P, tab, chunk, sh_u);
+    // A block takes consecutive chunks.  While they lie in one unit their sums stay in shared memory
+    // and go out together (at most 32 chunks: 2^15 additions of 16 bits per word): a long list then
+    // costs a block one set of atomic adds on the unit's sums, one fence and one count of finished
+    // chunks, not one per chunk.  Adds from many blocks to the same few 64-bit words of a unit are
+    // what this stage used to wait for.
+    constexpr uint32_t HOLD = 32;
+    ChunkCtx c, held;
+    uint32_t pending = 0;                          // chunks whose sums are held for unit held.u
+    auto flush = [&]() {
+        __syncthreads();                           // every add of the held chunks has been made
+        const uint4 a = *reinterpret_cast<const uint4*>(acc[threadIdx.x]);
+        *reinterpret_cast<uint4*>(acc[threadIdx.x]) = make_uint4(0u, 0u, 0u, 0u);
+        const unsigned long long a0 = ((unsigned long long)a.y << 16) + a.x, a1 = ((unsigned long long)a.w << 16) + a.z;
+        if (a0 | a1) {
+            unsigned long long* g = P.eacc + ((size_t)held.u * 256 + threadIdx.x) * 2;
+            if (a0) atomicAdd(g, a0);
+            if (a1) atomicAdd(g + 1, a1);
+        }
+        // the exponent range of the unit: one update per flush, and only when it widens the range
+        // seen on entry
+        const uint32_t used = __ballot_sync(0xffffffffu, (a0 | a1) != 0ull);
+        if (lane == 0) sh_e[wid] = used;
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t lo_e = 256u, hi_e = 0u;
+            for (int w = 0; w < BT / 32; ++w)
+                if (sh_e[w]) {
+                    const uint32_t first = (uint32_t)w * 32u + (uint32_t)__ffs(sh_e[w]) - 1u, last = (uint32_t)w * 32u + 31u - (uint32_t)__clz(sh_e[w]);
+                    lo_e = lo_e < first ? lo_e : first;
+                    hi_e = hi_e > last ? hi_e : last;
+                }
+            if (lo_e < held.un.emin) atomicMin(&P.units[held.u].emin, lo_e);
+            if (hi_e > held.un.emax) atomicMax(&P.units[held.u].emax, hi_e);
+            __threadfence();
+            // the flush that completes its unit turns the sums into the norm
+            const uint32_t nch = tab.cb[held.u + 1] - held.cb;
+            const bool last = atomicAdd(&P.units[held.u].done, pending) == nch - pending;
+            if (last) __threadfence();
+            sh_e[BT / 32] = last ? 1u : 0u;
+        }
+        __syncthreads();
+        if (sh_e[BT / 32]) unit_norm(P, held.u, held.c, acc);
+        pending = 0;
+    };
+    *reinterpret_cast<uint4*>(acc[threadIdx.x]) = make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t share = (total + gridDim.x - 1) / gridDim.x;
+    const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
+    for (uint32_t chunk = c_lo; chunk < c_hi; ++chunk) {
+        c = long_chunk_context(P, tab, chunk, sh_u, &c);       // (its barriers order the zeroing above)
+        if (pending && (c.u != held.u || pending == HOLD)) flush();
+        held = c;
         float val[PER];
         uint32_t idx[PER], key[PER];
 #pragma unroll
@@ -943,9 +1011,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
             idx[i] = in ? P.cand_idx[c.base + off] : 0xffffffffu;
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
         }
-        *reinterpret_cast<uint4*>(acc[threadIdx.x]) = make_uint4(0u, 0u, 0u, 0u);
         uint32_t nkept = 0;                          // lane 0 of each warp counts
-        __syncthreads();
         // sender bits first, all of them: the answers (was the bit set already) are used further down
         uint32_t seen[PER];
         bool kept[PER];
@@ -973,48 +1039,18 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
 #pragma unroll
         for (int i = 0; i < PER; ++i)
             if (seen[i]) atomicOr(&P.bm2[idx[i] >> 5], seen[i]);
-        if (early && lane == 0) sh_w[wid] = nkept;
-        __syncthreads();
-        if (early && threadIdx.x == 0) {
-            uint32_t t = 0;
-            for (int w = 0; w < BT / 32; ++w) t += sh_w[w];
-            P.chunk_cnt[c.chunk] = t | (t << 16);    // kept | sent << 16
-        }
-        if (plain) continue;
-        const uint4 a = *reinterpret_cast<const uint4*>(acc[threadIdx.x]);
-        const unsigned long long a0 = ((unsigned long long)a.y << 16) + a.x, a1 = ((unsigned long long)a.w << 16) + a.z;
-        if (a0 | a1) {
-            unsigned long long* g = P.eacc + ((size_t)c.u * 256 + threadIdx.x) * 2;
-            if (a0) atomicAdd(g, a0);
-            if (a1) atomicAdd(g + 1, a1);
-        }
-        // The exponent range of the unit: one update per chunk, and only when the chunk widens the
-        // range it saw on entry.  Every block works on the same few units, and the words of a unit
-        // share a line of the L2 that serves one access at a time.
-        const uint32_t used = __ballot_sync(0xffffffffu, (a0 | a1) != 0ull);
-        if (lane == 0) sh_e[wid] = used;
-        // the chunk that completes its unit turns the sums into the norm
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t lo_e = 256u, hi_e = 0u;
-            for (int w = 0; w < BT / 32; ++w)
-                if (sh_e[w]) {
-                    const uint32_t first = (uint32_t)w * 32u + (uint32_t)__ffs(sh_e[w]) - 1u, last = (uint32_t)w * 32u + 31u - (uint32_t)__clz(sh_e[w]);
-                    lo_e = lo_e < first ? lo_e : first;
-                    hi_e = hi_e > last ? hi_e : last;
-                }
-            if (lo_e < c.un.emin) atomicMin(&P.units[c.u].emin, lo_e);
-            if (hi_e > c.un.emax) atomicMax(&P.units[c.u].emax, hi_e);
-            __threadfence();
-            const uint32_t nch = tab.cb[c.u + 1] - c.cb;
-            if (atomicAdd(&P.units[c.u].done, 1u) == nch - 1) {
-                __threadfence();
-                unit_norm(P, c.u, c.c);
-                P.units[c.u].done = 0;
+        if (early) {
+            if (lane == 0) sh_w[wid] = nkept;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                uint32_t t = 0;
+                for (int w = 0; w < BT / 32; ++w) t += sh_w[w];
+                P.chunk_cnt[c.chunk] = t | (t << 16);    // kept | sent << 16
             }
         }
+        if (!plain) ++pending;
     }
+    if (pending) flush();
 }
 
 // adds v * 2^bitpos into a little-endian base-2^32 integer
@@ -1076,26 +1112,40 @@ __device__ float norm_of_sums(uint32_t emin, uint32_t emax, bool l1, Load load) 
     return l1 ? __double2float_rn(sum) : __double2float_rn(sqrt(sum));
 }
 
-// one thread, once per unit (of `count` candidates), after every chunk has added its sums.  The
-// sums were built with atomics in the L2: read them there, and leave them zero.
-__device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count) {
+// The whole block, once per unit (of `count` candidates), after every chunk has added its sums.
+// The sums were built with atomics in the L2: every thread fetches those of one exponent from
+// there (one round trip for all of them, where one thread reading them in turn took one each),
+// leaves them zero and parks them in shared memory (sh: 256 x 16 bytes, zero on entry and on
+// return); one thread then adds them up exactly.
+__device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count, uint32_t (*sh)[4]) {
     Unit& un = P.units[u];
     const uint32_t emin = __ldcg(&un.emin), emax = __ldcg(&un.emax);
-    if (emin > emax) return;
-    const bool l1 = P.qz == QS_SIGN_L1;
-    auto sums = [&](uint32_t e, unsigned long long* a0, unsigned long long* a1) {
-        const unsigned long long* g = P.eacc + ((size_t)u * 256 + e) * 2;
-        *a0 = __ldcg(g);
-        *a1 = __ldcg(g + 1);
-    };
-    // up to 2^20 values of 24 bits per sum: below 2^44
-    un.norm = (emax - emin <= 12u && count <= (1u << 20)) ? norm_of_sums_near(emin, emax, l1, sums)
-                                                           : norm_of_sums(emin, emax, l1, sums);
-    for (uint32_t e = emin; e <= emax; ++e) {
-        unsigned long long* g = P.eacc + ((size_t)u * 256 + e) * 2;
-        g[0] = 0ull;
-        g[1] = 0ull;
+    if (emin <= emax) {                                    // (the same in every thread)
+        const uint32_t e = threadIdx.x;
+        const bool mine = e >= emin && e <= emax;
+        if (mine) {
+            unsigned long long* g = P.eacc + ((size_t)u * 256 + e) * 2;
+            const unsigned long long a0 = __ldcg(g), a1 = __ldcg(g + 1);
+            g[0] = 0ull;
+            g[1] = 0ull;
+            *reinterpret_cast<ulonglong2*>(sh[e]) = make_ulonglong2(a0, a1);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const bool l1 = P.qz == QS_SIGN_L1;
+            auto sums = [&](uint32_t ee, unsigned long long* a0, unsigned long long* a1) {
+                const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(sh[ee]);
+                *a0 = v.x;
+                *a1 = v.y;
+            };
+            // up to 2^20 values of 24 bits per sum: below 2^44
+            un.norm = (emax - emin <= 12u && count <= (1u << 20)) ? norm_of_sums_near(emin, emax, l1, sums)
+                                                                   : norm_of_sums(emin, emax, l1, sums);
+        }
+        __syncthreads();
+        if (mine) *reinterpret_cast<uint4*>(sh[e]) = make_uint4(0u, 0u, 0u, 0u);
     }
+    if (threadIdx.x == 0) un.done = 0;
 }
 
 // ------------------------------------------------------------------ short units: one block does it all
@@ -1310,8 +1360,11 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t*
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_chunks;
     const bool sign_op = qz_is_sign(P.qz), plain = P.qz == QS_NONE;
-    for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+    ChunkCtx c;
+    const uint32_t share = (total + gridDim.x - 1) / gridDim.x;      // consecutive chunks: mostly one unit
+    const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
+    for (uint32_t chunk = c_lo; chunk < c_hi; ++chunk) {
+        c = chunk_context(P, tab, chunk, sh_u, &c);
         const float N = c.un.norm, cs = P.cscale[c.seg];
         const uint32_t k = P.kseg[c.seg];
         float* mem = P.mem + (size_t)c.r * P.d;
@@ -1467,8 +1520,11 @@ template <bool RANDK>
 __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
     const uint32_t total = tab.total_chunks;
     const bool plain = P.qz == QS_NONE, has_lvl = !qz_is_sign(P.qz) && !plain;
-    for (uint32_t chunk = blockIdx.x; chunk < total; chunk += gridDim.x) {
-        const ChunkCtx c = chunk_context(P, tab, chunk, sh_u);
+    ChunkCtx c;
+    const uint32_t share = (total + gridDim.x - 1) / gridDim.x;      // consecutive chunks: mostly one unit
+    const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
+    for (uint32_t chunk = c_lo; chunk < c_hi; ++chunk) {
+        c = chunk_context(P, tab, chunk, sh_u, &c);
         // this thread's candidates first: their reads overlap the sums below
         uint32_t q[PER], e[PER];
         float val[PER];
