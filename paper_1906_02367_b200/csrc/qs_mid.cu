@@ -1415,13 +1415,25 @@ __device__ void stage_chunk_scan(const Plan& P, const Tab& tab, const Active& ac
     if (blockIdx.x != 0) return;
     const uint32_t total = tab.total_chunks;
     uint32_t carry_k = 0, carry_s = 0;
-    for (uint32_t base = 0; base <= total; base += BT) {
-        const uint32_t i = base + threadIdx.x;
-        const uint32_t v = i < total ? P.chunk_cnt[i] : 0u;
+    constexpr uint32_t SC = 16;                   // consecutive chunks per thread and step
+    for (uint32_t base = 0; base <= total; base += BT * SC) {
+        const uint32_t i0 = base + threadIdx.x * SC;
+        uint32_t v[SC], sk = 0, ss = 0;
+#pragma unroll
+        for (uint32_t j = 0; j < SC; ++j) {
+            v[j] = i0 + j < total ? P.chunk_cnt[i0 + j] : 0u;
+            sk += v[j] & 0xffffu;
+            ss += v[j] >> 16;
+        }
         uint32_t tk, ts;
-        const uint32_t ek = block_excl_scan(v & 0xffffu, sh, &tk);
-        const uint32_t es = block_excl_scan(v >> 16, sh, &ts);
-        if (i <= total) { P.chunk_sel[i] = carry_k + ek; P.chunk_nz[i] = carry_s + es; }
+        uint32_t rk = carry_k + block_excl_scan(sk, sh, &tk);
+        uint32_t rs = carry_s + block_excl_scan(ss, sh, &ts);
+#pragma unroll
+        for (uint32_t j = 0; j < SC; ++j) {
+            if (i0 + j <= total) { P.chunk_sel[i0 + j] = rk; P.chunk_nz[i0 + j] = rs; }
+            rk += v[j] & 0xffffu;
+            rs += v[j] >> 16;
+        }
         carry_k += tk; carry_s += ts;
     }
     __syncthreads();
