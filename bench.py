@@ -32,7 +32,7 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dense pass on the bench workload, from the
 # ncu capture summarised in profiles/, scaled from the half-size capture (traffic grows with d)
-DENSE_TRAFFIC_BYTES = 2472900000   # 1236.5 MB measured at half size (profiles/pass_a_tma_kernel_resnet50_half_size.txt) x 2
+DENSE_TRAFFIC_BYTES = 2474800000   # 1237.4 MB measured at half size (profiles/pass_a_tma_kernel_resnet50_half_size.txt) x 2
 
 
 def workload(variant, shrink=1):

@@ -865,10 +865,15 @@ __device__ void stage_tie_find(const Plan& P, const Tab& tab, uint32_t* sh, uint
 // ------------------------------------------------------------------ quantize
 // Fused round, the master's "was this index sent, and by more than one worker": one bit per
 // coordinate in each of two bitmaps that the kernel clears when it starts, small enough to stay
-// in the L2 between the stage that sets them and the stage that reads them.
-__device__ __forceinline__ void mark_sender(const Plan& P, uint32_t idx) {
+// in the L2 between the stage that sets them and the stage that reads them.  Setting a bit takes
+// two steps so that a thread can start the first for all its entries before it needs an answer:
+// sender_mark returns the coordinate's bit if it was set already, sender_again records that.
+__device__ __forceinline__ uint32_t sender_mark(const Plan& P, uint32_t idx) {
     const uint32_t bit = 1u << (idx & 31u);
-    if (atomicOr(&P.bm1[idx >> 5], bit) & bit) atomicOr(&P.bm2[idx >> 5], bit);
+    return atomicOr(&P.bm1[idx >> 5], bit) & bit;
+}
+__device__ __forceinline__ void sender_again(const Plan& P, uint32_t idx, uint32_t seen) {
+    if (seen) atomicOr(&P.bm2[idx >> 5], seen);
 }
 
 template <bool RANDK>
@@ -1020,7 +1025,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
             const uint32_t off = c.first + i * BT + threadIdx.x;
             kept[i] = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
             seen[i] = 0u;
-            if (early && kept[i]) seen[i] = atomicOr(&P.bm1[idx[i] >> 5], 1u << (idx[i] & 31u)) & (1u << (idx[i] & 31u));
+            if (early && kept[i]) seen[i] = sender_mark(P, idx[i]);
         }
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
@@ -1038,7 +1043,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
         }
 #pragma unroll
         for (int i = 0; i < PER; ++i)
-            if (seen[i]) atomicOr(&P.bm2[idx[i] >> 5], seen[i]);
+            sender_again(P, idx[i], seen[i]);
         if (early) {
             if (lane == 0) sh_w[wid] = nkept;
             __syncthreads();
@@ -1300,7 +1305,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             uint32_t seen = 0u;                      // was the coordinate's bit set already (another worker sent it)
             if (early) {
                 if (lane == 0 && live) atomicAdd(&S.kept[i / PER], __popc(live));
-                if (kept) seen = atomicOr(&P.bm1[idx >> 5], 1u << (idx & 31u)) & (1u << (idx & 31u));
+                if (kept) seen = sender_mark(P, idx);
             }
             if (kept && !plain) {
                 const uint32_t b = RANDK ? vb : (kv >> 1);
@@ -1313,7 +1318,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             }
             return seen;
         };
-        auto twice = [&](uint32_t idx, uint32_t seen) { if (seen) atomicOr(&P.bm2[idx >> 5], seen); };
+        auto twice = [&](uint32_t idx, uint32_t seen) { sender_again(P, idx, seen); };
         // the indices are needed for the sender bits and for a tie cut; Rand_k reads the values too
         if (early || ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, twice);
         else unit_rows<RANDK, 16, false>(P, base, c, key, take, twice);
@@ -1379,9 +1384,11 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t*
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
         }
         uint32_t cnt = 0;                            // kept | sent << 16
+        uint32_t seen[PER];                          // sender bit found set already: answers used after the loop
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
+            seen[i] = 0u;
             if (off >= c.c) continue;
             uint32_t q = 0;
             if (is_kept<RANDK>(c.un, key[i], idx[i])) {
@@ -1393,11 +1400,14 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t*
                 if (level) {
                     mem[idx[i]] = val[i] - (plain ? val[i] : coord_value(P, N, level, neg, cs, k));
                     cnt += 1u << 16;
-                    if (fused) mark_sender(P, idx[i]);
+                    if (fused) seen[i] = sender_mark(P, idx[i]);
                 }
             }
             P.cand_q[c.base + off] = q;
         }
+#pragma unroll
+        for (int i = 0; i < PER; ++i)
+            sender_again(P, idx[i], seen[i]);
         cnt = warp_sum(cnt);
         if (lane == 0) sh_w[wid] = cnt;
         __syncthreads();
