@@ -209,9 +209,9 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.nfb = (uint32_t)h_fb.size();
     c->wire_words = words;
     if (nseg > 1) {
-        h_grp.resize(P.ngroups);
+        h_grp.resize((size_t)P.ntile * (STILE / GROUP));     // whole tiles: the dense pass copies a tile's entries at once
         int sg = 0;
-        for (uint32_t g = 0; g < P.ngroups; ++g) {
+        for (uint32_t g = 0; g < (uint32_t)h_grp.size(); ++g) {
             const int64_t e = (int64_t)g * GROUP;
             while (sg + 1 < nseg && e >= offsets[sg + 1]) ++sg;
             h_grp[g] = (uint32_t)sg;

@@ -40,6 +40,7 @@ constexpr int XSLOTS = QS_TMA_XSLOTS;      // x tiles in their ring
 constexpr int MAX_STAGES = STAGES > 4 ? STAGES : 4;
 
 struct TmaCtl {
+    alignas(16) uint32_t gseg[4][STILE / GROUP];   // segment of each group's first coordinate, for the last tile iterations
     uint64_t full[MAX_STAGES];
     uint64_t xfull[XSLOTS];
     uint32_t cnt[2][8 * GPW];              // candidates per group of the current tile (double-buffered)
@@ -118,7 +119,10 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
             mbar_expect(&S.xfull[xsl], bytes);
             bulk_load(xs + (size_t)xsl * TILE, P.x + e0, bytes, &S.xfull[xsl]);
         }
-        mbar_expect(&S.full[s], (uint32_t)NT * bytes);
+        // several segments: the tile's sixteen group-to-segment entries come with its first item
+        const bool segs = w == 0 && P.nseg > 1;
+        mbar_expect(&S.full[s], (uint32_t)NT * bytes + (segs ? (uint32_t)sizeof(S.gseg[0]) : 0u));
+        if (segs) bulk_load(S.gseg[it & 3u], P.grp_seg + (size_t)tile * (STILE / GROUP), (uint32_t)sizeof(S.gseg[0]), &S.full[s]);
         bulk_load(slot(s, 0), P.xw + row, bytes, &S.full[s]);
         bulk_load(slot(s, 1), P.mem + row, bytes, &S.full[s]);
         if (ANCH) bulk_load(slot(s, T_ANCH), P.anchors + row, bytes, &S.full[s]);
@@ -176,15 +180,13 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
             const uint32_t g = tile * (TILE / GROUP) + warp * GP + k;
             const uint32_t q = (warp * GP + k) * GROUP + lane * 4;
             const uint32_t e0 = tile * TILE + q;
-            if (w == 0 && P.nseg > 1) {
-                // segment of the group's first coordinate, from the offsets in shared memory (a load
-                // from global memory here would stall the tile behind the copies in flight)
-                int lo = 0, hi = P.nseg;
+            if (w == 0 && P.nseg > 1 && tile < ntiles) {     // (the end mark brings no entries: nothing to look up)
+                // segment of the group's first coordinate: the table's entries for this tile came in
+                // with the tile's first item (a load from global memory here would stall the tile
+                // behind the copies in flight)
+                const uint32_t ent = S.gseg[it & 3u][warp * GP + k];
+                const int lo = (int)(ent < (uint32_t)P.nseg ? ent : (uint32_t)P.nseg - 1u);
                 const uint32_t first = g * (uint32_t)GROUP;
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (seg_off[mid] <= first) lo = mid; else hi = mid;
-                }
                 sq0[k] = lo;
                 uni[k] = lo + 1 >= P.nseg || seg_off[lo + 1] >= first + (uint32_t)GROUP;
             }
