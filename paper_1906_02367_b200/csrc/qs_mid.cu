@@ -897,6 +897,28 @@ __device__ __forceinline__ void sums_add(uint32_t (*acc)[4], uint32_t e, uint32_
     }
 }
 
+// The norm from the exact sum held as an integer: tot1 x 2^(e_lo - 1 - 149) (magnitudes) or tot2 x
+// 2^(2 (e_lo - 1) - 298) (squares).  One conversion rounds it to fp64, to nearest even.
+__device__ __forceinline__ float norm_of_exact_sum(bool l1, unsigned long long tot1, unsigned __int128 tot2, int e_lo) {
+    double sum;
+    if (l1) {
+        sum = ldexp(__ull2double_rn(tot1), e_lo - 1 - 149);
+    } else {
+        const unsigned long long hi = (unsigned long long)(tot2 >> 64), lo = (unsigned long long)tot2;
+        if (hi == 0ull) {
+            sum = ldexp(__ull2double_rn(lo), 2 * (e_lo - 1) - 298);
+        } else {
+            // the top 64 bits with everything below folded into the lowest one: the conversion then
+            // rounds as if it had seen all the bits
+            const int s = 64 - __clzll(hi);
+            unsigned long long top = (unsigned long long)(tot2 >> s);
+            if ((lo << (64 - s)) != 0ull) top |= 1ull;
+            sum = ldexp(__ull2double_rn(top), s + 2 * (e_lo - 1) - 298);
+        }
+    }
+    return l1 ? __double2float_rn(sum) : __double2float_rn(sqrt(sum));
+}
+
 // Norm from per-exponent sums that span at most 12 exponents, each sum below 2^44: the exact sum
 // fits 64 (magnitudes) or 128 (squares) bits, and one conversion rounds it to fp64 (to nearest
 // even).  Other cases take norm_of_sums; both give the correctly rounded exact sum.  The sums are
@@ -921,23 +943,7 @@ __device__ float norm_of_sums_near(uint32_t emin, uint32_t emax, bool l1, Load l
             else tot2 += ((unsigned __int128)a0[j] + ((unsigned __int128)a1[j] << 24)) << (2 * sh);
         }
     }
-    double sum;
-    if (l1) {
-        sum = ldexp(__ull2double_rn(tot1), e_lo - 1 - 149);
-    } else {
-        const unsigned long long hi = (unsigned long long)(tot2 >> 64), lo = (unsigned long long)tot2;
-        if (hi == 0ull) {
-            sum = ldexp(__ull2double_rn(lo), 2 * (e_lo - 1) - 298);
-        } else {
-            // the top 64 bits with everything below folded into the lowest one: the conversion then
-            // rounds as if it had seen all the bits
-            const int s = 64 - __clzll(hi);
-            unsigned long long top = (unsigned long long)(tot2 >> s);
-            if ((lo << (64 - s)) != 0ull) top |= 1ull;
-            sum = ldexp(__ull2double_rn(top), s + 2 * (e_lo - 1) - 298);
-        }
-    }
-    return l1 ? __double2float_rn(sum) : __double2float_rn(sqrt(sum));
+    return norm_of_exact_sum(l1, tot1, tot2, e_lo);
 }
 
 
@@ -1075,26 +1081,11 @@ __device__ void big_add(uint32_t* dig, int ndig, unsigned long long v, int bitpo
     }
 }
 
-// Exact sum of the per-exponent integer sums (exponents emin .. emax, read through `load`) ->
-// fp64 (round to nearest even) -> norm in fp32.  One thread.
-template <class Load>
-__device__ float norm_of_sums(uint32_t emin, uint32_t emax, bool l1, Load load) {
-    constexpr int ND = 24;                      // 768 bits
-    uint32_t dig[ND];
-    for (int j = 0; j < ND; ++j) dig[j] = 0;
-    // bit 0 stands for 2^-298 (squares) or 2^-149 (magnitudes)
-    for (uint32_t e = emin; e <= emax; ++e) {
-        unsigned long long a0, a1;
-        load(e, &a0, &a1);
-        if (!(a0 | a1)) continue;
-        const int ee = e ? (int)e : 1;          // subnormals share the exponent of e = 1
-        if (l1) {
-            big_add(dig, ND, a0, ee - 1);
-        } else {
-            big_add(dig, ND, a0, 2 * (ee - 1));
-            big_add(dig, ND, a1, 2 * (ee - 1) + 24);
-        }
-    }
+// A 768-bit integer (little-endian base 2^32; bit 0 stands for 2^-298 with squares, 2^-149 with
+// magnitudes) -> fp64 (round to nearest even) -> norm in fp32.  One thread.
+constexpr int NORM_DIGITS = 24;
+__device__ float norm_of_digits(const uint32_t* dig, bool l1) {
+    constexpr int ND = NORM_DIGITS;
     int tw = ND - 1;
     while (tw >= 0 && dig[tw] == 0) --tw;
     double sum = 0.0;
@@ -1115,6 +1106,28 @@ __device__ float norm_of_sums(uint32_t emin, uint32_t emax, bool l1, Load load) 
         sum = ldexp((double)mant, top - 52 - (l1 ? 149 : 298));
     }
     return l1 ? __double2float_rn(sum) : __double2float_rn(sqrt(sum));
+}
+
+// Exact sum of the per-exponent integer sums (exponents emin .. emax, read through `load`) ->
+// norm.  One thread.
+template <class Load>
+__device__ float norm_of_sums(uint32_t emin, uint32_t emax, bool l1, Load load) {
+    constexpr int ND = NORM_DIGITS;
+    uint32_t dig[ND];
+    for (int j = 0; j < ND; ++j) dig[j] = 0;
+    for (uint32_t e = emin; e <= emax; ++e) {
+        unsigned long long a0, a1;
+        load(e, &a0, &a1);
+        if (!(a0 | a1)) continue;
+        const int ee = e ? (int)e : 1;          // subnormals share the exponent of e = 1
+        if (l1) {
+            big_add(dig, ND, a0, ee - 1);
+        } else {
+            big_add(dig, ND, a0, 2 * (ee - 1));
+            big_add(dig, ND, a1, 2 * (ee - 1) + 24);
+        }
+    }
+    return norm_of_digits(dig, l1);
 }
 
 // The whole block, once per unit (of `count` candidates), after every chunk has added its sums.
@@ -1206,12 +1219,139 @@ __device__ __forceinline__ void unit_rows(const Plan& P, size_t base, uint32_t c
     }
 }
 
+// The shortest lists (at most 64 candidates: two per lane) need no block: a warp takes such a
+// unit through the same steps with shuffles only, eight units at a time per block.  Ranks by
+// direct counting; the exact norm as one integer sum over the warp when the kept values' exponents
+// lie within 12 of each other, otherwise value by value into the long accumulator by one lane.
+constexpr uint32_t WARP_C = 64;
+
+__device__ __forceinline__ unsigned long long warp_sum64(unsigned long long v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <bool RANDK>
+__device__ void unit_by_warp(const Plan& P, const Tab& tab, uint32_t u, uint32_t r, uint32_t seg, bool early, int lane) {
+    const uint32_t c = tab.c[u], k = P.kseg[seg];
+    const size_t base = (size_t)r * P.cap + tab.start[u];
+    const bool plain = P.qz == QS_NONE, l1 = P.qz == QS_SIGN_L1;
+    uint32_t key[2], idx[2], vb[2];
+    bool in[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        const uint32_t j = (uint32_t)lane + 32u * q;
+        in[q] = j < c;
+        key[q] = in[q] ? sort_key<RANDK>(P, base + j) : 0u;
+        idx[q] = in[q] ? P.cand_idx[base + j] : 0u;
+        vb[q] = (RANDK && in[q]) ? __float_as_uint(P.cand_val[base + j]) : (key[q] >> 1);
+    }
+    // rank of each candidate: those before it have a larger key, or an equal one earlier in the list
+    uint32_t rank[2] = {0u, 0u};
+    for (uint32_t j = 0; j < c; ++j) {
+        const uint32_t kj = __shfl_sync(0xffffffffu, j < 32u ? key[0] : key[1], (int)(j & 31u));
+        rank[0] += (kj > key[0] || (kj == key[0] && j < (uint32_t)lane)) ? 1u : 0u;
+        rank[1] += (kj > key[1] || (kj == key[1] && j < (uint32_t)lane + 32u)) ? 1u : 0u;
+    }
+    bool kept[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) kept[q] = in[q] && rank[q] < k;
+    // exponent range of the kept values
+    uint32_t e[2], m[2];
+    int lo_e = 255, hi_e = 0;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        e[q] = (vb[q] >> 23) & 255u;
+        m[q] = e[q] ? ((vb[q] & 0x7fffffu) | 0x800000u) : (vb[q] & 0x7fffffu);
+        if (kept[q] && m[q]) {
+            const int ee = e[q] ? (int)e[q] : 1;
+            lo_e = ee < lo_e ? ee : lo_e;
+            hi_e = ee > hi_e ? ee : hi_e;
+        }
+    }
+    lo_e = __reduce_min_sync(0xffffffffu, lo_e);
+    hi_e = __reduce_max_sync(0xffffffffu, hi_e);
+    float norm = 0.0f;
+    if (!plain && hi_e >= lo_e && hi_e - lo_e > 12) {                      // (the same in every lane)
+        uint32_t dig[NORM_DIGITS];
+        for (int j = 0; j < NORM_DIGITS; ++j) dig[j] = 0;
+        for (uint32_t j = 0; j < c; ++j) {
+            const bool second = j >= 32u;
+            const uint32_t kj = __shfl_sync(0xffffffffu, (second ? kept[1] : kept[0]) ? 1u : 0u, (int)(j & 31u));
+            const uint32_t ej = __shfl_sync(0xffffffffu, second ? e[1] : e[0], (int)(j & 31u));
+            const uint32_t mj = __shfl_sync(0xffffffffu, second ? m[1] : m[0], (int)(j & 31u));
+            if (lane == 0 && kj && mj) {
+                const int ee = ej ? (int)ej : 1;
+                if (l1) big_add(dig, NORM_DIGITS, mj, ee - 1);
+                else big_add(dig, NORM_DIGITS, (unsigned long long)mj * mj, 2 * (ee - 1));
+            }
+        }
+        norm = __shfl_sync(0xffffffffu, lane == 0 ? norm_of_digits(dig, l1) : 0.0f, 0);
+    } else if (!plain && hi_e >= lo_e) {
+        // at most 64 terms of 24 (magnitudes) or 48 (squares) bits shifted by at most 12 (24)
+        unsigned long long p1 = 0ull, p2lo = 0ull, p2hi = 0ull;
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+            if (kept[q] && m[q]) {
+                const int sh = (e[q] ? (int)e[q] : 1) - lo_e;
+                if (l1) {
+                    p1 += (unsigned long long)m[q] << sh;
+                } else {
+                    const unsigned __int128 t = (unsigned __int128)((unsigned long long)m[q] * m[q]) << (2 * sh);
+                    p2lo += (unsigned long long)t & 0xffffffffffull;        // low 40 bits
+                    p2hi += (unsigned long long)(t >> 40);
+                }
+            }
+        p1 = warp_sum64(p1);
+        p2lo = warp_sum64(p2lo);
+        p2hi = warp_sum64(p2hi);
+        norm = norm_of_exact_sum(l1, p1, ((unsigned __int128)p2hi << 40) + p2lo, lo_e);
+    }
+    // threshold: the candidate of rank k - 1
+    const uint32_t hit0 = __ballot_sync(0xffffffffu, in[0] && rank[0] == k - 1u);
+    const uint32_t hit1 = __ballot_sync(0xffffffffu, in[1] && rank[1] == k - 1u);
+    const int src = hit0 ? __ffs(hit0) - 1 : __ffs(hit1) - 1;
+    const uint32_t tau = __shfl_sync(0xffffffffu, hit0 ? key[0] : key[1], src);
+    const uint32_t tie_max = __shfl_sync(0xffffffffu, hit0 ? idx[0] : idx[1], src);
+    if (early) {
+        uint32_t seen[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) seen[q] = kept[q] ? sender_mark(P, idx[q]) : 0u;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) sender_again(P, idx[q], seen[q]);
+        const uint32_t n = __popc(__ballot_sync(0xffffffffu, kept[0])) + __popc(__ballot_sync(0xffffffffu, kept[1]));
+        if (lane == 0) P.chunk_cnt[tab.cb[u]] = n | (n << 16);             // a list this short is one chunk
+    }
+    // the level-0 counts of the order stage are not needed on this path: leave them zero
+#pragma unroll
+    for (int i = 0; i < 8; ++i) P.hist[(size_t)u * 256 + (uint32_t)lane + 32u * i] = 0u;
+    if (lane == 0) {
+        Unit& out = P.units[u];
+        out.tau = tau;
+        out.tie_max = tie_max;
+        out.tie_t = 0;
+        out.n = 0;
+        out.emin = 255u;
+        out.emax = 0u;
+        out.norm = norm;
+        if (!RANDK) predict_floor(P, r, seg, tau, c, k);
+    }
+}
+
 template <bool RANDK>
 __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, bool early, UnitSh& S, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t items = (uint32_t)P.nseg * (uint32_t)act.n;
     const bool plain = P.qz == QS_NONE, l1 = P.qz == QS_SIGN_L1;
     const uint32_t lt = (1u << lane) - 1u;
+    // the shortest lists first, a warp each: eight consecutive units of the list to a block
+    for (uint32_t item = blockIdx.x * (BT / 32) + wid; item < items; item += gridDim.x * (BT / 32)) {
+        const uint32_t seg = P.seg_order[item / (uint32_t)act.n];
+        const uint32_t r = (uint32_t)act.r[item % (uint32_t)act.n];
+        const uint32_t u = r * (uint32_t)P.nseg + seg;
+        const uint32_t c = tab.c[u];
+        if (c && c <= WARP_C && c <= tab.short_c) unit_by_warp<RANDK>(P, tab, u, r, seg, early, lane);
+    }
     if (threadIdx.x == 0) S.ctl[0] = atomicAdd(P.bar + 4, 1u);
     __syncthreads();
     for (;;) {
@@ -1223,7 +1363,8 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
         const uint32_t r = (uint32_t)act.r[item % (uint32_t)act.n];
         const uint32_t u = r * (uint32_t)P.nseg + seg;
         const uint32_t c = tab.c[u], k = P.kseg[seg];
-        if (c == 0 || c > tab.short_c) { __syncthreads(); continue; }     // an idle worker's, or a long unit
+        // an idle worker's, a long unit, or one that a warp has done
+        if (c == 0 || c > tab.short_c || c <= WARP_C) { __syncthreads(); continue; }
         const size_t base = (size_t)r * P.cap + tab.start[u];
         uint32_t key[UPT];
 #pragma unroll

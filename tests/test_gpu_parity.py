@@ -151,12 +151,12 @@ def test_small_and_ragged_sizes(d, k, sp, qz):
     p.close()
 
 
-@pytest.mark.parametrize("d", [200, 3000, 5000])     # lists of at most 256, 4096 and more candidates: the three per-unit forms
+@pytest.mark.parametrize("d", [50, 200, 3000, 5000])     # lists of at most 64, 256, 4096 and more candidates: by a warp, by ranks, by radix in a block, by the grid
 def test_ties_zeros_and_equal_values(d):
     R = 2
     cases = []
     z = np.zeros((R, d), np.float32)
-    cases.append((np.zeros(d, np.float32), z.copy(), z.copy(), d // 100))             # everything zero
+    cases.append((np.zeros(d, np.float32), z.copy(), z.copy(), max(1, d // 100)))     # everything zero
     eq = np.full((R, d), 0.25, np.float32)
     cases.append((np.zeros(d, np.float32), -eq, z.copy(), d // 65 + 1))               # all equal
     g = np.random.default_rng(3)
