@@ -62,7 +62,8 @@ __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, in
             }
             __nanosleep(32);
         }
-        __threadfence();
+        // (the acquiring load that saw the last arrival orders this thread behind every block's
+        // writes, and the block barrier below passes that on to the other threads)
         if (P.trace && blockIdx.x == 0) {          // time at which every block has finished the stage
             const uint32_t slot = target / gridDim.x;
             unsigned long long t;
