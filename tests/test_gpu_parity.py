@@ -170,6 +170,26 @@ def test_ties_zeros_and_equal_values(d):
             p.close()
 
 
+@pytest.mark.parametrize("d", [40, 200, 3000, 20000])
+@pytest.mark.parametrize("qz", [O.QSGD, O.SIGN_L1, O.SIGN_L2])
+def test_norm_over_wide_exponent_ranges(d, qz):
+    # kept values spread over sixty binary orders of magnitude (and a few subnormals): the exact sum
+    # cannot take the short 64/128-bit route and goes through the long accumulator, in each of the
+    # forms a unit is handled in (by a warp, by a block, by the grid)
+    R = 3
+    g = np.random.default_rng(d)
+    mag = np.ldexp(g.uniform(1.0, 2.0, size=(R, d)), g.integers(-30, 31, size=(R, d))).astype(np.float32)
+    mag[:, ::17] = np.float32(1e-41)
+    sign = np.where(g.random((R, d)) < 0.5, -1.0, 1.0).astype(np.float32)
+    xw = mag * sign
+    z = np.zeros((R, d), np.float32)
+    p = Pair(R, d, k=max(1, d // 2), s=16, quantizer=qz, seed=7, x=np.zeros(d, np.float32), xw=xw, mem=z)
+    p.round_split(0)
+    p.drift(xw * np.float32(0.25))
+    p.round_fused(1)
+    p.close()
+
+
 def test_ties_in_long_candidate_lists():
     # many equal keys at the threshold of a long list: the cut by lower index is found by all blocks together
     R, d = 3, 200000
