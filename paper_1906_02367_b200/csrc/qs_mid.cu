@@ -1704,8 +1704,7 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge
                 const uint32_t key = RANDK ? P.cand_key[c.base + off] : topk_key(val[i]);
                 if (is_kept<RANDK>(c.un, key, e[i])) {
                     const bool neg = val[i] < 0.0f;
-                    q[i] = Q_SEL | (neg ? Q_NEG : 0u) | 1u;
-                    P.mem[(size_t)c.r * P.d + e[i]] = val[i] - (plain ? val[i] : coord_value(P, c.un.norm, 1, neg, P.cscale[c.seg], P.kseg[c.seg]));
+                    q[i] = Q_SEL | (neg ? Q_NEG : 0u) | 1u;       // (the memory update itself waits until the reads below are out)
                 }
             }
         }
@@ -1726,6 +1725,16 @@ __device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge
 #pragma unroll
             for (int i = 0; i < PER; ++i)
                 if (((sent_mask & ~multi) >> i) & 1u) xv[i] = P.x[e[i]];
+        }
+        if (merge) {
+            // the quantize stage's memory update for level-1 quantizers, behind the reads above: a
+            // wave of scattered stores in front of them would hold them up
+#pragma unroll
+            for (int i = 0; i < PER; ++i)
+                if (q[i] & Q_SEL) {
+                    const bool neg = (q[i] & Q_NEG) != 0;
+                    P.mem[(size_t)c.r * P.d + e[i]] = val[i] - (plain ? val[i] : coord_value(P, c.un.norm, 1, neg, P.cscale[c.seg], P.kseg[c.seg]));
+                }
         }
         uint32_t run_k, run_s, unit_n, pay;
         const uint32_t bi = P.bidx[c.seg], lo = P.seg_off[c.seg];
