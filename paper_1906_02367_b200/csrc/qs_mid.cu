@@ -876,6 +876,10 @@ __device__ __forceinline__ uint32_t sender_mark(const Plan& P, uint32_t idx) {
 __device__ __forceinline__ void sender_again(const Plan& P, uint32_t idx, uint32_t seen) {
     if (seen) atomicOr(&P.bm2[idx >> 5], seen);
 }
+// the pack stage will read x at a sent index: ask for the line now, without waiting for it
+__device__ __forceinline__ void x_ahead(const Plan& P, uint32_t idx) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.x + idx));
+}
 
 template <bool RANDK>
 __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t idx) {
@@ -1032,7 +1036,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
             const uint32_t off = c.first + i * BT + threadIdx.x;
             kept[i] = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
             seen[i] = 0u;
-            if (early && kept[i]) seen[i] = sender_mark(P, idx[i]);
+            if (early && kept[i]) { seen[i] = sender_mark(P, idx[i]); x_ahead(P, idx[i]); }
         }
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
@@ -1317,7 +1321,10 @@ __device__ void unit_by_warp(const Plan& P, const Tab& tab, uint32_t u, uint32_t
     if (early) {
         uint32_t seen[2];
 #pragma unroll
-        for (int q = 0; q < 2; ++q) seen[q] = kept[q] ? sender_mark(P, idx[q]) : 0u;
+        for (int q = 0; q < 2; ++q) {
+            seen[q] = kept[q] ? sender_mark(P, idx[q]) : 0u;
+            if (kept[q]) x_ahead(P, idx[q]);
+        }
 #pragma unroll
         for (int q = 0; q < 2; ++q) sender_again(P, idx[q], seen[q]);
         const uint32_t n = __popc(__ballot_sync(0xffffffffu, kept[0])) + __popc(__ballot_sync(0xffffffffu, kept[1]));
@@ -1447,7 +1454,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             uint32_t seen = 0u;                      // was the coordinate's bit set already (another worker sent it)
             if (early) {
                 if (lane == 0 && live) atomicAdd(&S.kept[i / PER], __popc(live));
-                if (kept) seen = sender_mark(P, idx);
+                if (kept) { seen = sender_mark(P, idx); x_ahead(P, idx); }
             }
             if (kept && !plain) {
                 const uint32_t b = RANDK ? vb : (kv >> 1);
