@@ -98,6 +98,11 @@ enum {
  * Rand_k, plus 4 d bytes of sender bits and small tables); one
  * segment [0, d) with k is installed.  Returns QS_INVALID_ARG, QS_ALLOC or QS_CUDA on
  * failure, in which case *out is NULL.
+ * Read from the environment here, for tuning and tests (results never depend on them):
+ * QSPARSE_UNIT_CAP (0..4096, default 4096: the longest candidate list that one thread
+ * block may select from on its own; 0 sends every list through the grid-wide radix
+ * levels), QSPARSE_MID_PER_SM (thread blocks of the persistent kernel per SM, default
+ * 4), QSPARSE_NO_TMA (dense pass with plain loads), QSPARSE_TMA_DEPTH (its ring depth).
  */
 int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t seed,
             void* cuda_stream);
