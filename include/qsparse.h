@@ -261,8 +261,8 @@ int qs_set_round(qs_ctx* ctx, uint64_t round);
 /*
  * qs_get_stats — host counters since qs_init (synchronises the stream): out[0] rounds
  * compressed, out[1] worker-rounds whose predicted threshold missed and took the exact
- * histogram pass, out[2] candidates examined, out[3] kernels launched.  Writes min(n, 4)
- * values.
+ * histogram pass, out[2] candidates examined, out[3] kernels launched, out[4] blocks of the
+ * persistent kernel (all resident at once).  Writes min(n, 5) values.
  */
 int qs_get_stats(qs_ctx* ctx, int64_t* out, int n);
 

@@ -220,10 +220,10 @@ class Context:
         self._check(lib().qs_set_round(self._h, int(rnd)))
 
     def stats(self):
-        out = np.zeros(4, dtype=np.int64)
-        self._check(lib().qs_get_stats(self._h, out.ctypes.data_as(C.c_void_p), 4))
+        out = np.zeros(5, dtype=np.int64)
+        self._check(lib().qs_get_stats(self._h, out.ctypes.data_as(C.c_void_p), 5))
         return {"rounds": int(out[0]), "fallback_worker_rounds": int(out[1]), "candidates": int(out[2]),
-                "launches": int(out[3])}
+                "launches": int(out[3]), "persistent_blocks": int(out[4])}
 
     def enable_phase_timing(self, on=True):
         self._check(lib().qs_enable_phase_timing(self._h, int(bool(on))))

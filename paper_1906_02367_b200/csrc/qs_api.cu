@@ -119,8 +119,8 @@ uint32_t candidate_target(int sp, uint64_t n, uint64_t k) {
         slack = 6.0 * std::sqrt((double)k) + 32.0;           // the hash is uniform: binomial spread
     } else {
         const double ratio = (double)k / (double)n;
-        const double frac = ratio <= 0.002 ? 1.0 : ratio <= 0.02 ? 0.5 : 0.25;
-        slack = std::fmax(std::fmax(frac * (double)k, 16.0 * std::sqrt((double)k)), 32.0);
+        const double frac = ratio <= 0.02 ? 0.5 : 0.25;
+        slack = std::fmax(std::fmax(frac * (double)k, 16.0 * std::sqrt((double)k)), 16.0);
     }
     const double t = (double)k + slack;
     return (uint32_t)(t >= (double)n ? n : (uint64_t)t);
@@ -253,6 +253,8 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(hist, (size_t)4 * P.U * 256, true);
     AL(eacc, (size_t)P.U * 256 * 2, true);
     AL(chunk_cnt, (size_t)P.maxchunks + 1, true);
+    AL(chunk_dir, (size_t)P.maxchunks + 1, false);
+    AL(unit_tab, P.U, false);
     AL(chunk_sel, (size_t)P.maxchunks + 1, true);
     AL(chunk_nz, (size_t)P.maxchunks + 1, true);
     AL(fb_hist, (size_t)P.U * FB_BINS, true);
@@ -265,10 +267,6 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(dec_ent, (size_t)32 * (nseg + 1), true);
     AL(dec_pay, (size_t)32 * nseg, true);
     AL(touch, (size_t)d, true);
-    AL(bm1, 2 * (((size_t)d + 31) >> 5), true);
-    P.bm2 = P.bm1 + (((size_t)d + 31) >> 5);
-    AL(coll, (size_t)R * P.K, false);
-    AL(ncoll, 1, true);
     AL(status, 1, true);
     AL(bar, 8, true);
     AL(trace, TRACE_SLOTS, true);
@@ -286,7 +284,6 @@ int rezero(qs_ctx* c) {
     QS_CUDA_TRY(c, cudaMemsetAsync(P.fb_hist, 0, sizeof(uint32_t) * P.U * FB_BINS, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.touch, 0, sizeof(uint32_t) * P.d, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.fail, 0, sizeof(uint32_t) * P.R, c->st));
-    QS_CUDA_TRY(c, cudaMemsetAsync(P.ncoll, 0, sizeof(uint32_t), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.units, 0, sizeof(Unit) * P.U, c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.status, 0, sizeof(int), c->st));
     QS_CUDA_TRY(c, cudaMemsetAsync(P.bar, 0, 8 * sizeof(uint32_t), c->st));
@@ -391,6 +388,9 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     P.wbase = 0; P.rdiv = R;
     P.unit_cap = UNIT_CAP;                         // QSPARSE_UNIT_CAP (0 .. 4096) overrides, for tests of both paths
     if (const char* e = std::getenv("QSPARSE_UNIT_CAP")) P.unit_cap = (uint32_t)std::min(std::max(std::atoi(e), 0), UNIT_CAP);
+    P.order_sups_max = ORDER_SUPS_MAX;             // QSPARSE_ORDER_EVEN_MAX (0 .. 2048) overrides, for tests of both order stages
+    if (const char* e = std::getenv("QSPARSE_ORDER_EVEN_MAX")) P.order_sups_max = (uint32_t)std::min(std::max(std::atoi(e), 0), (int)ORDER_SUPS_MAX);
+    P.block_pack = std::getenv("QSPARSE_BLOCK_PACK") != nullptr;   // for tests of both ways of packing in a whole round
     P.seed_lo = (uint32_t)seed; P.seed_hi = (uint32_t)(seed >> 32);
     const int64_t offsets[2] = {0, d};
     const int rc = install_segments(c, 1, offsets, &k);
@@ -585,8 +585,8 @@ int qs_get_stats(qs_ctx* c, int64_t* out, int n) {
     QS_CUDA_TRY(c, cudaStreamSynchronize(c->st));
     long long dev[2] = {0, 0};
     QS_CUDA_TRY(c, cudaMemcpy(dev, c->P.stats, sizeof(dev), cudaMemcpyDeviceToHost));
-    const int64_t v[4] = {c->rounds, (int64_t)dev[0], (int64_t)dev[1], c->launches};
-    for (int i = 0; i < n && i < 4; ++i) out[i] = v[i];
+    const int64_t v[5] = {c->rounds, (int64_t)dev[0], (int64_t)dev[1], c->launches, (int64_t)c->mid_grid};
+    for (int i = 0; i < n && i < 5; ++i) out[i] = v[i];
     return QS_OK;
 }
 

@@ -18,6 +18,7 @@ constexpr int SUP_BLOCKS = 64;       // blocks per super-block of the two-level 
 #endif
 constexpr int CHUNK = QS_CHUNK;     // candidates per selection chunk (a multiple of the 256 threads)
 constexpr int UT_MAX = 2048;         // units whose table fits in the persistent kernel's shared memory
+constexpr uint32_t ORDER_SUPS_MAX = 2048;   // (worker, super-block) sums the order stage can hold in shared memory
 constexpr int UNIT_CAP = 4096;       // candidates of a unit that one block may select from on its own (16 per thread)
 constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (top 11 key bits)
 constexpr int FB_SHIFT = 21;
@@ -64,6 +65,8 @@ struct Plan {
     uint32_t d, ngroups, ntile, nblk, nsup, K, U, nfb, maxchunks;
     uint32_t seed_lo, seed_hi, round_lo, round_hi;
     uint32_t unit_cap;         // a round whose units all have at most this many candidates selects per block (0: never)
+    uint32_t order_sups_max;   // (worker, super-block) pairs up to which the order stage deals its work evenly
+    int block_pack;            // non-zero: every block packs its share before the closing stage (no packing warps beside it)
     uint64_t cap;
     // tables (device)
     const uint32_t* seg_off;   // nseg + 1
@@ -94,6 +97,8 @@ struct Plan {
     uint32_t* hist;            // 4 x U x 256, zero between rounds
     unsigned long long* eacc;  // U x 256 x 2, zero between rounds
     uint32_t* chunk_cnt;       // maxchunks + 1 (kept | sent << 16 per chunk)
+    uint32_t* chunk_dir;       // maxchunks: unit of each chunk, for the packing warps of the closing stage
+    uint4* unit_tab;           // U: (start, candidates, first chunk) of each unit, likewise
     uint32_t* chunk_sel;       // maxchunks + 1 exclusive sums of kept
     uint32_t* chunk_nz;        // maxchunks + 1 exclusive sums of sent
     uint32_t* fb_hist;         // U x FB_BINS, zero between rounds
@@ -103,13 +108,10 @@ struct Plan {
     long long* bits;           // R: bits of the worker's record (likewise)
     uint32_t* dec_ent;         // 32 x (nseg + 1): any worker of a sharded job
     uint32_t* dec_pay;         // 32 x nseg
-    uint32_t* touch;           // d, zero between rounds
-    uint32_t* bm1;             // ceil(d / 32): coordinates some worker sent (fused round)
-    uint32_t* bm2;             // ceil(d / 32): coordinates several workers sent; directly behind bm1
-    uint2* coll;               // R x K: (coordinate, unit) of indices several workers sent, fused round
-    uint32_t* ncoll;           // 1, zero between rounds
+    uint32_t* touch;           // d, zero between rounds: senders of each coordinate (separate master call)
     int* status;
-    uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel, [2], [3] tile tickets, [4] unit tickets
+    uint32_t* bar;             // [0] arrivals of the grid barrier, [1] blocks that left the kernel, [2], [3] tile tickets,
+                               // [4] unit tickets, [6] chunk tickets of the packing warps
     unsigned long long* trace; // TRACE_SLOTS global-timer stamps of the last persistent launch, or null
     long long* stats;          // device counters: [0] fallback worker-rounds, [1] candidates
 };

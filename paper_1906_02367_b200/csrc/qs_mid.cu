@@ -45,8 +45,9 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
     return v;
 }
 
-// All blocks of the cooperative launch meet here.  The wait is bounded: a block that gives up
-// records QS_TIMEOUT and every block leaves the kernel at its next barrier.
+// All blocks of the cooperative launch meet here (every block is resident).  The wait is
+// bounded: a block that gives up records QS_TIMEOUT and every block leaves the stages at its next
+// barrier.
 __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, int* sh_abort) {
     target += gridDim.x;
     __syncthreads();
@@ -68,7 +69,7 @@ __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, in
             const uint32_t slot = target / gridDim.x;
             unsigned long long t;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-            if (slot < TRACE_SLOTS - 1) P.trace[slot] = t;
+            if (slot < TRACE_SLOTS - 4) P.trace[slot] = t;
         }
     }
     __syncthreads();
@@ -250,7 +251,6 @@ __device__ __forceinline__ uint32_t last_not_above(const uint32_t* a, uint32_t n
 // its share touches (a window at a time), and copies: entry -> block by binary search, -> tile by
 // the block's sixteen tile counts, -> its place in the tile's run.  No block reads more counts
 // than its share needs: a table every block reads in full is a hot spot in the L2.
-constexpr uint32_t ORDER_SUPS_MAX = 2048;
 constexpr uint32_t ORDER_WIN = (ORDER_ITEMS_MAX - ORDER_SUPS_MAX - 8) / SUP_BLOCKS;   // super-blocks per window
 
 template <bool RANDK>
@@ -864,23 +864,6 @@ __device__ void stage_tie_find(const Plan& P, const Tab& tab, uint32_t* sh, uint
 }
 
 // ------------------------------------------------------------------ quantize
-// Fused round, the master's "was this index sent, and by more than one worker": one bit per
-// coordinate in each of two bitmaps that the kernel clears when it starts, small enough to stay
-// in the L2 between the stage that sets them and the stage that reads them.  Setting a bit takes
-// two steps so that a thread can start the first for all its entries before it needs an answer:
-// sender_mark returns the coordinate's bit if it was set already, sender_again records that.
-__device__ __forceinline__ uint32_t sender_mark(const Plan& P, uint32_t idx) {
-    const uint32_t bit = 1u << (idx & 31u);
-    return atomicOr(&P.bm1[idx >> 5], bit) & bit;
-}
-__device__ __forceinline__ void sender_again(const Plan& P, uint32_t idx, uint32_t seen) {
-    if (seen) atomicOr(&P.bm2[idx >> 5], seen);
-}
-// the pack stage will read x at a sent index: ask for the line now, without waiting for it
-__device__ __forceinline__ void x_ahead(const Plan& P, uint32_t idx) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.x + idx));
-}
-
 template <bool RANDK>
 __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t idx) {
     return sk > un.tau || (sk == un.tau && idx <= un.tie_max);
@@ -1028,15 +1011,11 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
         }
         uint32_t nkept = 0;                          // lane 0 of each warp counts
-        // sender bits first, all of them: the answers (was the bit set already) are used further down
-        uint32_t seen[PER];
         bool kept[PER];
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
             kept[i] = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
-            seen[i] = 0u;
-            if (early && kept[i]) { seen[i] = sender_mark(P, idx[i]); x_ahead(P, idx[i]); }
         }
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
@@ -1052,9 +1031,6 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
                 sums_add(acc, e, lo, hi, !l1);
             }
         }
-#pragma unroll
-        for (int i = 0; i < PER; ++i)
-            sender_again(P, idx[i], seen[i]);
         if (early) {
             if (lane == 0) sh_w[wid] = nkept;
             __syncthreads();
@@ -1319,14 +1295,6 @@ __device__ void unit_by_warp(const Plan& P, const Tab& tab, uint32_t u, uint32_t
     const uint32_t tau = __shfl_sync(0xffffffffu, hit0 ? key[0] : key[1], src);
     const uint32_t tie_max = __shfl_sync(0xffffffffu, hit0 ? idx[0] : idx[1], src);
     if (early) {
-        uint32_t seen[2];
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            seen[q] = kept[q] ? sender_mark(P, idx[q]) : 0u;
-            if (kept[q]) x_ahead(P, idx[q]);
-        }
-#pragma unroll
-        for (int q = 0; q < 2; ++q) sender_again(P, idx[q], seen[q]);
         const uint32_t n = __popc(__ballot_sync(0xffffffffu, kept[0])) + __popc(__ballot_sync(0xffffffffu, kept[1]));
         if (lane == 0) P.chunk_cnt[tab.cb[u]] = n | (n << 16);             // a list this short is one chunk
     }
@@ -1451,11 +1419,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
         auto take = [&](uint32_t i, uint32_t off, uint32_t kv, uint32_t idx, uint32_t vb) {
             const bool kept = off < c && kv >= tau && !(ties && kv == tau && idx > tie_max);
             const uint32_t live = __ballot_sync(0xffffffffu, kept);
-            uint32_t seen = 0u;                      // was the coordinate's bit set already (another worker sent it)
-            if (early) {
-                if (lane == 0 && live) atomicAdd(&S.kept[i / PER], __popc(live));
-                if (kept) { seen = sender_mark(P, idx); x_ahead(P, idx); }
-            }
+            if (early && lane == 0 && live) atomicAdd(&S.kept[i / PER], __popc(live));
             if (kept && !plain) {
                 const uint32_t b = RANDK ? vb : (kv >> 1);
                 const uint32_t e = (b >> 23) & 255u;
@@ -1465,12 +1429,12 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
                 else { const unsigned long long sq = (unsigned long long)m * m; lo = (uint32_t)(sq & 0xffffffu); hi = (uint32_t)(sq >> 24); }
                 sums_add(S.acc, e, lo, hi, !l1);
             }
-            return seen;
+            return 0u;
         };
-        auto twice = [&](uint32_t idx, uint32_t seen) { sender_again(P, idx, seen); };
-        // the indices are needed for the sender bits and for a tie cut; Rand_k reads the values too
-        if (early || ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, twice);
-        else unit_rows<RANDK, 16, false>(P, base, c, key, take, twice);
+        auto none = [](uint32_t, uint32_t) {};
+        // the indices are needed for a tie cut; Rand_k reads the values too
+        if (ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, none);
+        else unit_rows<RANDK, 16, false>(P, base, c, key, take, none);
         __syncthreads();
         if (wid == 0) {
             // exponent range of the sums
@@ -1510,7 +1474,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
 
 // levels, signs, memory update; kept and sent counts per chunk
 template <bool RANDK>
-__device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t* sh_u, uint32_t* sh_w) {
+__device__ void stage_quant(const Plan& P, const Tab& tab, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_chunks;
     const bool sign_op = qz_is_sign(P.qz), plain = P.qz == QS_NONE;
@@ -1533,11 +1497,9 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t*
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
         }
         uint32_t cnt = 0;                            // kept | sent << 16
-        uint32_t seen[PER];                          // sender bit found set already: answers used after the loop
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
-            seen[i] = 0u;
             if (off >= c.c) continue;
             uint32_t q = 0;
             if (is_kept<RANDK>(c.un, key[i], idx[i])) {
@@ -1549,14 +1511,10 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, bool fused, uint32_t*
                 if (level) {
                     mem[idx[i]] = val[i] - (plain ? val[i] : coord_value(P, N, level, neg, cs, k));
                     cnt += 1u << 16;
-                    if (fused) seen[i] = sender_mark(P, idx[i]);
                 }
             }
             P.cand_q[c.base + off] = q;
         }
-#pragma unroll
-        for (int i = 0; i < PER; ++i)
-            sender_again(P, idx[i], seen[i]);
         cnt = warp_sum(cnt);
         if (lane == 0) sh_w[wid] = cnt;
         __syncthreads();
@@ -1686,153 +1644,202 @@ __device__ __forceinline__ void block_sum4(uint32_t v[4], uint32_t* sh) {
 }
 
 // streams of every segment, and the ordered kept list kept for inspection.  A thread takes PER
-// consecutive candidates, so one scan over the block places them all.
+// consecutive candidates, so one scan over the block places them all.  One chunk; `c` carries the
+// context of the block's previous chunk in and this one's out.
 template <bool RANDK>
-__device__ void stage_pack(const Plan& P, const Tab& tab, bool fused, bool merge, uint32_t* wire, long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
-    const uint32_t total = tab.total_chunks;
+__device__ void pack_chunk(const Plan& P, const Tab& tab, uint32_t chunk, ChunkCtx& c, bool merge, uint32_t* wire,
+                           long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
     const bool plain = P.qz == QS_NONE, has_lvl = !qz_is_sign(P.qz) && !plain;
-    ChunkCtx c;
-    const uint32_t share = (total + gridDim.x - 1) / gridDim.x;      // consecutive chunks: mostly one unit
-    const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
-    for (uint32_t chunk = c_lo; chunk < c_hi; ++chunk) {
-        c = chunk_context(P, tab, chunk, sh_u, &c);
-        // this thread's candidates first: their reads overlap the sums below
-        uint32_t q[PER], e[PER];
-        float val[PER];
+    c = chunk_context(P, tab, chunk, sh_u, &c);
+    // this thread's candidates first: their reads overlap the sums below
+    uint32_t q[PER], e[PER];
+    float val[PER];
 #pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            const uint32_t off = c.first + threadIdx.x * PER + i;
-            const bool in = off < c.c;
-            e[i] = in ? P.cand_idx[c.base + off] : 0u;
-            q[i] = (in && !merge) ? P.cand_q[c.base + off] : 0u;
-            val[i] = (in && (merge || plain)) ? P.cand_val[c.base + off] : 0.0f;
-            if (merge && in) {
-                // the quantize stage's part for level-1 quantizers: sign, and the memory update
-                const uint32_t key = RANDK ? P.cand_key[c.base + off] : topk_key(val[i]);
-                if (is_kept<RANDK>(c.un, key, e[i])) {
-                    const bool neg = val[i] < 0.0f;
-                    q[i] = Q_SEL | (neg ? Q_NEG : 0u) | 1u;       // (the memory update itself waits until the reads below are out)
-                }
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t off = c.first + threadIdx.x * PER + i;
+        const bool in = off < c.c;
+        e[i] = in ? P.cand_idx[c.base + off] : 0u;
+        q[i] = (in && !merge) ? P.cand_q[c.base + off] : 0u;
+        val[i] = (in && (merge || plain)) ? P.cand_val[c.base + off] : 0.0f;
+        if (merge && in) {
+            // the quantize stage's part for level-1 quantizers: the sign (the memory update is the closing stage's)
+            const uint32_t key = RANDK ? P.cand_key[c.base + off] : topk_key(val[i]);
+            if (is_kept<RANDK>(c.un, key, e[i])) {
+                const bool neg = val[i] < 0.0f;
+                q[i] = Q_SEL | (neg ? Q_NEG : 0u) | 1u;
             }
         }
-        // Master update riding along (whole round): which of this thread's entries are sent is known
-        // from q alone, so the reads it needs (was the index sent by several workers; x) start now
-        // and are in flight while the positions are worked out.
-        uint32_t sent_mask = 0, multi = 0;
-        float xv[PER];
-#pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            if ((q[i] & Q_SEL) && (q[i] & 0xffffu)) sent_mask |= 1u << i;
-            xv[i] = 0.0f;
+    }
+    uint32_t run_k, run_s, unit_n, pay;
+    const uint32_t bi = P.bidx[c.seg], lo = P.seg_off[c.seg];
+    if (tab.fast) {
+        // positions from the chunk counts of the unit directly (no scan stage ran)
+        const uint32_t c1 = tab.cb[c.u + 1];
+        uint32_t sums[4] = {0u, 0u, 0u, 0u};          // kept before, sent before, kept in all, sent in all
+        for (uint32_t i = c.cb + threadIdx.x; i < c1; i += BT) {
+            const uint32_t v = P.chunk_cnt[i];
+            sums[2] += v & 0xffffu; sums[3] += v >> 16;
+            if (i < chunk) { sums[0] += v & 0xffffu; sums[1] += v >> 16; }
         }
-        if (fused) {
-#pragma unroll
-            for (int i = 0; i < PER; ++i)
-                if (((sent_mask >> i) & 1u) && ((P.bm2[e[i] >> 5] >> (e[i] & 31u)) & 1u)) multi |= 1u << i;
-#pragma unroll
-            for (int i = 0; i < PER; ++i)
-                if (((sent_mask & ~multi) >> i) & 1u) xv[i] = P.x[e[i]];
-        }
-        if (merge) {
-            // the quantize stage's memory update for level-1 quantizers, behind the reads above: a
-            // wave of scattered stores in front of them would hold them up
-#pragma unroll
-            for (int i = 0; i < PER; ++i)
-                if (q[i] & Q_SEL) {
-                    const bool neg = (q[i] & Q_NEG) != 0;
-                    P.mem[(size_t)c.r * P.d + e[i]] = val[i] - (plain ? val[i] : coord_value(P, c.un.norm, 1, neg, P.cscale[c.seg], P.kseg[c.seg]));
-                }
-        }
-        uint32_t run_k, run_s, unit_n, pay;
-        const uint32_t bi = P.bidx[c.seg], lo = P.seg_off[c.seg];
-        if (tab.fast) {
-            // positions from the chunk counts of the unit directly (no scan stage ran)
-            const uint32_t c1 = tab.cb[c.u + 1];
-            uint32_t sums[4] = {0u, 0u, 0u, 0u};          // kept before, sent before, kept in all, sent in all
-            for (uint32_t i = c.cb + threadIdx.x; i < c1; i += BT) {
-                const uint32_t v = P.chunk_cnt[i];
-                sums[2] += v & 0xffffu; sums[3] += v >> 16;
-                if (i < chunk) { sums[0] += v & 0xffffu; sums[1] += v >> 16; }
+        block_sum4(sums, sh);
+        run_k = sums[0]; run_s = sums[1]; unit_n = sums[3];
+        pay = P.nseg == 1 ? 2u : P.pay_off[c.u];          // several segments: every kept entry is sent, fixed places
+        if (chunk == c.cb && threadIdx.x == 0) {          // the unit's first chunk writes its directory entry
+            P.units[c.u].n = unit_n;
+            if (sums[2] != P.kseg[c.seg]) set_status(P, QS_STATE);
+            uint32_t* row = wire + (size_t)c.r * stride;
+            row[2 * c.seg] = unit_n;
+            row[2 * c.seg + 1] = __float_as_uint(c.un.norm);
+            if (P.nseg == 1) {
+                const long long bits = 64 + (long long)unit_n * entry_bits(bi, (uint32_t)P.bl, P.qz);
+                P.bits[c.r] = bits;
+                if (bits_out) bits_out[c.r] = bits;
+            } else if (c.seg == 0 && bits_out) {
+                bits_out[c.r] = P.bits[c.r];
             }
-            block_sum4(sums, sh);
-            run_k = sums[0]; run_s = sums[1]; unit_n = sums[3];
-            pay = P.nseg == 1 ? 2u : P.pay_off[c.u];          // several segments: every kept entry is sent, fixed places
-            if (chunk == c.cb && threadIdx.x == 0) {          // the unit's first chunk writes its directory entry
-                P.units[c.u].n = unit_n;
-                if (sums[2] != P.kseg[c.seg]) set_status(P, QS_STATE);
-                uint32_t* row = wire + (size_t)c.r * stride;
-                row[2 * c.seg] = unit_n;
-                row[2 * c.seg + 1] = __float_as_uint(c.un.norm);
-                if (P.nseg == 1) {
-                    const long long bits = 64 + (long long)unit_n * entry_bits(bi, (uint32_t)P.bl, P.qz);
-                    P.bits[c.r] = bits;
-                    if (bits_out) bits_out[c.r] = bits;
-                } else if (c.seg == 0 && bits_out) {
-                    bits_out[c.r] = P.bits[c.r];
-                }
-            }
-        } else {
-            run_k = P.chunk_sel[chunk] - P.chunk_sel[c.cb];
-            run_s = P.chunk_nz[chunk] - P.chunk_nz[c.cb];
-            unit_n = c.un.n;
-            pay = P.pay_off[c.u];
         }
-        uint32_t* w_idx = wire + (size_t)c.r * stride + pay;
-        uint32_t* w_sgn = w_idx + words_for(unit_n, bi);
-        uint32_t* w_lvl = w_sgn + words_for(unit_n, 1);
-        uint32_t* o_idx = P.sel_idx + (size_t)c.r * P.K + P.kprefix[c.seg];
-        uint32_t* o_q = P.sel_q + (size_t)c.r * P.K + P.kprefix[c.seg];
-        uint32_t mine = 0;                            // kept | sent << 16 among this thread's candidates
+    } else {
+        run_k = P.chunk_sel[chunk] - P.chunk_sel[c.cb];
+        run_s = P.chunk_nz[chunk] - P.chunk_nz[c.cb];
+        unit_n = c.un.n;
+        pay = P.pay_off[c.u];
+    }
+    uint32_t* w_idx = wire + (size_t)c.r * stride + pay;
+    uint32_t* w_sgn = w_idx + words_for(unit_n, bi);
+    uint32_t* w_lvl = w_sgn + words_for(unit_n, 1);
+    uint32_t* o_idx = P.sel_idx + (size_t)c.r * P.K + P.kprefix[c.seg];
+    uint32_t* o_q = P.sel_q + (size_t)c.r * P.K + P.kprefix[c.seg];
+    uint32_t mine = 0;                            // kept | sent << 16 among this thread's candidates
 #pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
-            mine += kept | (sent << 16);
-        }
-        uint32_t tot;
-        const uint32_t ex = block_excl_scan(mine, sh, &tot);
-        uint32_t jk = run_k + (ex & 0xffffu), js0 = run_s + (ex >> 16);
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
+        mine += kept | (sent << 16);
+    }
+    uint32_t tot;
+    const uint32_t ex = block_excl_scan(mine, sh, &tot);
+    uint32_t jk = run_k + (ex & 0xffffu), js0 = run_s + (ex >> 16);
 #pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
-            if (kept && jk < P.kseg[c.seg]) {                          // (the bound holds by construction)
-                o_idx[jk] = e[i];
-                o_q[jk] = q[i];
-                if (sent && js0 < unit_n) {
-                    const uint64_t js = js0;
-                    or_bits(w_idx, js * bi, bi, e[i] - lo);
-                    if (plain) {
-                        w_sgn[js] = __float_as_uint(val[i]);                   // value stream
-                    } else {
-                        if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
-                        if (has_lvl) or_bits(w_lvl, js * P.bl, P.bl, (q[i] & 0xffffu) - 1u);
-                    }
-                }
-            }
-            jk += kept;
-            js0 += sent;
-        }
-        if (fused) {
-            // an index only this worker sent gets acc = 0 + g, x <- x - acc / R right here; an index
-            // with several senders has each sender leave its value at (worker, coordinate) and set
-            // its bit in the index's word of sender bits; whoever finds that word empty lists the
-            // index for the next stage.
-            float* gval = reinterpret_cast<float*>(P.stage);
-#pragma unroll
-            for (int i = 0; i < PER; ++i) {
-                if (!((sent_mask >> i) & 1u)) continue;
-                const float g = plain ? val[i]
-                                      : coord_value(P, c.un.norm, (int)(q[i] & 0xffffu), (q[i] & Q_NEG) != 0,
-                                                    P.cscale[c.seg], P.kseg[c.seg]);
-                if (!((multi >> i) & 1u)) {
-                    float acc = 0.0f;
-                    acc = acc + g;
-                    P.x[e[i]] = xv[i] - acc / (float)P.rdiv;
+    for (int i = 0; i < PER; ++i) {
+        const uint32_t kept = (q[i] & Q_SEL) ? 1u : 0u, sent = (kept && (q[i] & 0xffffu)) ? 1u : 0u;
+        if (kept && jk < P.kseg[c.seg]) {                          // (the bound holds by construction)
+            o_idx[jk] = e[i];
+            o_q[jk] = q[i];
+            if (sent && js0 < unit_n) {
+                const uint64_t js = js0;
+                or_bits(w_idx, js * bi, bi, e[i] - lo);
+                if (plain) {
+                    w_sgn[js] = __float_as_uint(val[i]);                   // value stream
                 } else {
-                    gval[(size_t)c.r * P.cap + e[i]] = g;
-                    if (atomicOr(&P.touch[e[i]], 1u << c.r) == 0u) P.coll[atomicAdd(P.ncoll, 1u)] = make_uint2(e[i], c.u);
+                    if (q[i] & Q_NEG) atomicOr(&w_sgn[js >> 5], 1u << (js & 31u));
+                    if (has_lvl) or_bits(w_lvl, js * P.bl, P.bl, (q[i] & 0xffffu) - 1u);
                 }
             }
         }
+        jk += kept;
+        js0 += sent;
+    }
+}
+
+// every chunk, the blocks taking equal shares of consecutive chunks (mostly one unit each)
+template <bool RANDK>
+__device__ void stage_pack(const Plan& P, const Tab& tab, bool merge, uint32_t* wire, long long stride,
+                           long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
+    const uint32_t total = tab.total_chunks;
+    ChunkCtx c;
+    const uint32_t share = (total + gridDim.x - 1) / gridDim.x;
+    const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
+    for (uint32_t chunk = c_lo; chunk < c_hi; ++chunk) pack_chunk<RANDK>(P, tab, chunk, c, merge, wire, stride, bits_out, sh_u, sh);
+}
+
+// The unit table as the packing warps of the closing stage need it (their block's copy in shared
+// memory is gone by then): unit of every chunk, and (start, candidates, first chunk) of every unit.
+__device__ void publish_table(const Plan& P, const Tab& tab) {
+    for (uint32_t q = blockIdx.x * BT + threadIdx.x; q < tab.total_chunks; q += gridDim.x * BT) P.chunk_dir[q] = unit_of_chunk(P, tab, q);
+    for (uint32_t u = blockIdx.x * BT + threadIdx.x; u < P.U; u += gridDim.x * BT) P.unit_tab[u] = make_uint4(tab.start[u], tab.c[u], tab.cb[u], 0u);
+}
+
+// One chunk packed by one warp: the quantizers that send every kept entry at level 1 (whole round;
+// the memory update is the closing stage's).  32 rows of 32 candidates; a row's kept entries get
+// consecutive places behind those of the rows and chunks before it.
+template <bool RANDK>
+__device__ void pack_chunk_warp(const Plan& P, uint32_t q, uint32_t* wire, long long stride, long long* bits_out, int lane) {
+    const uint32_t u = P.chunk_dir[q];
+    const uint4 ut = P.unit_tab[u];                   // start, candidates, first chunk
+    const Unit un = P.units[u];
+    const uint32_t r = u / P.nseg, seg = u % P.nseg;
+    const uint32_t k = P.kseg[seg], bi = P.bidx[seg], lo = P.seg_off[seg];
+    const uint32_t j = q - ut.z, first = j * (uint32_t)CHUNK;
+    const size_t base = (size_t)r * P.cap + ut.x;
+    const bool plain = P.qz == QS_NONE;
+    uint32_t before = 0;                              // kept in the unit's earlier chunks
+    for (uint32_t i = lane; i < j; i += 32) before += P.chunk_cnt[ut.z + i] & 0xffffu;
+    before = warp_sum(before);
+    uint32_t* row = wire + (size_t)r * stride;
+    uint32_t* w_idx = row + (P.nseg == 1 ? 2u : P.pay_off[u]);
+    uint32_t* w_sgn = w_idx + words_for(k, bi);
+    uint32_t* o_idx = P.sel_idx + (size_t)r * P.K + P.kprefix[seg];
+    uint32_t* o_q = P.sel_q + (size_t)r * P.K + P.kprefix[seg];
+    if (j == 0) {                                     // the unit's first chunk writes its directory entry
+        const uint32_t nch = (ut.y + CHUNK - 1) / CHUNK;
+        uint32_t tot = 0;
+        for (uint32_t i = lane; i < nch; i += 32) tot += P.chunk_cnt[ut.z + i] & 0xffffu;
+        tot = warp_sum(tot);
+        if (lane == 0) {
+            if (tot != k) set_status(P, QS_STATE);
+            P.units[u].n = k;
+            row[2 * seg] = k;
+            row[2 * seg + 1] = __float_as_uint(un.norm);
+            if (P.nseg == 1) {
+                const long long bits = 64 + (long long)k * entry_bits(bi, (uint32_t)P.bl, P.qz);
+                P.bits[r] = bits;
+                if (bits_out) bits_out[r] = bits;
+            } else if (seg == 0 && bits_out) {
+                bits_out[r] = P.bits[r];
+            }
+        }
+    }
+    uint32_t run = before;
+    const uint32_t lt = (1u << lane) - 1u;
+    constexpr int RB = 4;                             // rows whose reads are issued together
+    for (uint32_t rb = 0; rb < (uint32_t)(CHUNK / 32) && first + rb * 32u < ut.y; rb += RB) {
+        uint32_t idx[RB], key[RB];
+        float val[RB];
+        bool in[RB];
+#pragma unroll
+        for (int t = 0; t < RB; ++t) {
+            const uint32_t off = first + (rb + t) * 32u + (uint32_t)lane;
+            in[t] = off < ut.y;
+            idx[t] = in[t] ? P.cand_idx[base + off] : 0u;
+            val[t] = in[t] ? P.cand_val[base + off] : 0.0f;
+            key[t] = RANDK ? (in[t] ? P.cand_key[base + off] : 0u) : topk_key(val[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < RB; ++t) {
+            const bool kept = in[t] && is_kept<RANDK>(un, key[t], idx[t]);
+            const uint32_t bal = __ballot_sync(0xffffffffu, kept);
+            const uint32_t pos = run + __popc(bal & lt);
+            if (kept && pos < k) {                                     // (the bound holds by construction)
+                const bool neg = val[t] < 0.0f;
+                o_idx[pos] = idx[t];
+                o_q[pos] = Q_SEL | (neg ? Q_NEG : 0u) | 1u;
+                or_bits(w_idx, (uint64_t)pos * bi, bi, idx[t] - lo);
+                if (plain) w_sgn[pos] = __float_as_uint(val[t]);       // value stream
+                else if (neg) atomicOr(&w_sgn[pos >> 5], 1u << (pos & 31u));
+            }
+            run += __popc(bal);
+        }
+    }
+}
+
+// chunks handed out to packing warps by a ticket counter
+template <bool RANDK>
+__device__ void pack_by_warps(const Plan& P, uint32_t total_chunks, uint32_t* wire, long long stride, long long* bits_out, int lane) {
+    for (;;) {
+        uint32_t q = 0;
+        if (lane == 0) q = atomicAdd(P.bar + 6, 1u);
+        q = __shfl_sync(0xffffffffu, q, 0);
+        if (q >= total_chunks) break;
+        pack_chunk_warp<RANDK>(P, q, wire, stride, bits_out, lane);
     }
 }
 
@@ -1972,109 +1979,488 @@ __device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t
     }
 }
 
-// Fused round: indices that several workers sent.  Their lowest sender listed them and every sender
-// left its value at (worker, coordinate); here they are added in increasing worker order.
-__device__ void stage_coll_apply(const Plan& P) {
-    const uint32_t n = *P.ncoll;
-    const float* gval = reinterpret_cast<const float*>(P.stage);
-    for (uint32_t id = blockIdx.x * BT + threadIdx.x; id < n; id += gridDim.x * BT) {
-        const uint32_t coord = P.coll[id].x;
-        uint32_t rest = P.touch[coord];
-        float acc = 0.0f;
-        while (rest) {
-            const int r2 = __ffs(rest) - 1;
-            rest &= rest - 1u;
-            acc = acc + gval[(size_t)r2 * P.cap + coord];
-        }
-        P.x[coord] = P.x[coord] - acc / (float)P.rdiv;
-        P.touch[coord] = 0u;
-    }
+// ------------------------------------------------------------------ master update + broadcast
+// Closing stage of a whole round: x <- x - (1/R) sum_r g_r and xw_r <- x in ONE pass over x.
+//
+// Tiles of x (2048 coordinates) are handed out by a ticket counter.  In every block one warp keeps
+// the copies going through a ring of slots in shared memory: a tile of x comes in with one bulk
+// copy and with it, one more bulk copy per active worker, the tile's candidate runs as the dense
+// pass left them ((index, value) pairs; their counts were read a tile ahead); when a tile has been
+// worked on it goes out to every active worker's row (and anchor row) as bulk stores.  Four
+// other warps, one per slot, work on the tiles that have landed: from the unit's
+// threshold, tie cut and norm a warp decides which candidates were kept and sent and what value
+// g each stands for (the same expression the worker used for its memory), and applies them to
+// the tile in shared memory:
+//   - a coordinate with one sender: x - (0 + g) / R, on the spot;
+//   - a coordinate with several senders (found with two bitmaps of the tile in shared memory):
+//     the entries are listed, and the entry of the lowest worker adds the values in increasing
+//     worker order before it updates x.  The list is bounded: positions are taken in windows of
+//     as many as fit.
+// Updated coordinates are also written to x in global memory.  No sender bitmaps over d, no
+// scattered reads of x, no stage for shared indices: everything the update needs is in the
+// tile's runs, and the copies never wait for the arithmetic as long as the working warps keep up.
+// Rows that are not 16-byte aligned take the same steps with ordinary loads and stores, a warp
+// per tile; so do the candidates of a tile that has more of them than the buffer holds.
+constexpr int NSLOT = 4;           // tiles of a block in shared memory: coming in, worked on, going out
+constexpr int NWORK = NSLOT;       // warps that work on landed tiles (warps 1 .. NWORK; warp 0 copies): one per slot, so
+                                   // that each sees every phase of its slot's barrier in turn
+constexpr int ML_CAP = 160;        // listed entries of coordinates with several senders
+constexpr int CB = 416;            // candidates of a tile (all workers) held in shared memory
+constexpr uint32_t NO_TILE = 0xffffffffu;
+
+struct BcSlot {
+    float xs[STILE];               // a tile of x
+    uint2 cb[CB];                  // its candidates, worker after worker (each run padded to an even count);
+                                   // once looked at, an entry holds (position | sent << 31, value)
+    uint32_t cnt[32];              // candidates of each active worker (slot order)
+    uint32_t pbefore[32];          // where its run starts in cb
+    uint32_t gseg[STILE / GROUP];  // segment of the first coordinate of each 128-coordinate group
+    uint32_t tile, staged;
+    uint32_t whole;                // the working warp asks for the whole tile to be stored to x (many coordinates changed)
+    uint32_t pad;
+};
+
+struct BcScratch {                 // of one working warp
+    uint32_t bm1[STILE / 32];      // coordinates of the tile some worker sent
+    uint32_t bm2[STILE / 32];      // coordinates several workers sent
+    uint32_t pref[STILE / 32];     // such coordinates before each word of bm2
+    uint32_t mpos[ML_CAP];         // listed entry: position in the tile | worker slot << 16
+    float mg[ML_CAP];              // its value
+    uint32_t nm, pad[3];
+};
+
+struct BcBlock {
+    BcSlot slot[NSLOT];
+    BcScratch scr[NWORK];
+    uint64_t full[NSLOT];          // the slot's copies have landed (or the end mark is in place)
+    uint64_t done[NSLOT];          // the slot's tile has been worked on
+    int abort, pad[3];
+};
+static_assert(sizeof(BcSlot) % 16 == 0 && sizeof(BcScratch) % 16 == 0, "tile buffers are the targets of bulk copies");
+constexpr size_t MID_SCRATCH_BYTES = (ORDER_ITEMS_MAX + 8) * sizeof(uint32_t) + FB_BINS * 4;
+constexpr size_t MID_POOL_BYTES = sizeof(BcBlock) > MID_SCRATCH_BYTES ? sizeof(BcBlock) : MID_SCRATCH_BYTES;
+
+// what a lane keeps about the unit (its worker, a segment) its candidates mostly belong to
+struct UnitLite { uint32_t tau, tie_max, k, end; float norm, c; };
+
+// Lanes to workers: the warp is cut into as many equal parts as the next power of two of the
+// active workers; part j of worker slot w (lane w + j * parts) walks entries j, j + J, .. of the
+// worker's run.  Everything a lane needs about its worker sits in its own registers: no shuffles
+// or searches per candidate.
+struct LaneMap {
+    int nact, my_w;
+    uint32_t J, my_j, my_r;
+    bool live;
+};
+
+__device__ __forceinline__ LaneMap lane_map(const Active& act, int lane) {
+    LaneMap L;
+    L.nact = act.n;
+    int parts = 1;
+    while (parts < L.nact) parts <<= 1;               // nact <= 32
+    L.J = 32u / (uint32_t)parts;
+    L.my_w = lane & (parts - 1);
+    L.my_j = (uint32_t)lane / (uint32_t)parts;
+    L.live = L.my_w < L.nact;
+    L.my_r = L.live ? (uint32_t)act.r[L.my_w] : 0u;
+    return L;
 }
 
-// xw_r <- x (and the anchors) for the active workers: the closing dense stage of a fused round
-template <bool ALIGNED>
-__device__ void stage_broadcast(const Plan& P, const Active& act) {
-    const int lane = threadIdx.x & 31;
-    for (uint32_t g = blockIdx.x * (BT / 32) + (threadIdx.x >> 5); g < P.ngroups; g += gridDim.x * (BT / 32)) {
-        const uint32_t e0 = g * (uint32_t)GROUP + (uint32_t)lane * 4u;
-        if (e0 >= P.d) continue;
-        if (ALIGNED) {
-            const float4 v = *reinterpret_cast<const float4*>(P.x + e0);
-            for (int w = 0; w < act.n; ++w) {
-                __stcs(reinterpret_cast<float4*>(P.xw + (size_t)act.r[w] * P.d + e0), v);
-                if (P.anchors) __stcs(reinterpret_cast<float4*>(P.anchors + (size_t)act.r[w] * P.d + e0), v);
+__device__ __forceinline__ UnitLite unit_lite(const Plan& P, const LaneMap& L, uint32_t seg) {
+    UnitLite u = {0u, 0u, 0u, 0u, 0.0f, 0.0f};
+    if (L.live) {
+        const Unit& g = P.units[(size_t)L.my_r * P.nseg + seg];
+        u.tau = g.tau; u.tie_max = g.tie_max; u.norm = g.norm;
+        u.k = P.kseg[seg]; u.c = P.cscale[seg]; u.end = P.seg_off[seg + 1];
+    }
+    return u;
+}
+
+// The update of one tile by one warp.  xs: the tile in shared memory; cnt: candidates of this
+// lane's worker in the tile; cb + pbefore: where they are in shared memory (staged), otherwise they
+// are read from the run in global memory; gseg: the tile's group-to-segment entries.  mem_update:
+// the warp also writes m <- u - g at the sent coordinates (level-1 quantizers in a whole round).
+// Returns true when it leaves the tile's write-back to x to the caller (can_whole: the caller can
+// store the whole tile; taken when so many coordinates changed that one sequential store is cheaper
+// than their scattered sectors).
+constexpr uint32_t WHOLE_TILE_MIN = 64;
+
+template <bool RANDK>
+__device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t tile, uint32_t cnt, bool staged, uint2* cb,
+                           uint32_t pbefore, const uint32_t* gseg, float* xs, BcScratch& W, const UnitLite& un, bool mem_update,
+                           bool can_whole) {
+    const uint32_t e0 = tile * (uint32_t)STILE;
+    const uint32_t nel = P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE;
+    const float rdiv = (float)P.rdiv;
+    const uint32_t wp = (uint32_t)(ML_CAP / (L.nact > 0 ? L.nact : 1));   // positions with several senders per window
+    const uint32_t J = L.J, my_j = L.my_j, my_r = L.my_r;
+    const uint2* run = P.stage + (size_t)my_r * P.cap + (size_t)tile * STILE;
+    // What will be read from global memory is asked for now, all of it at once (one round trip in
+    // place of one per entry): the run itself when it is not in shared memory, and the units of
+    // the next few segments when the tile may hold more than one.
+    if (!staged)
+        for (uint32_t line = my_j; line * 16u < cnt; line += J) asm volatile("prefetch.global.L1 [%0];" ::"l"(run + line * 16u));
+    if (un.end < e0 + nel && L.live) {
+        const uint32_t s0 = gseg[0];
+        for (uint32_t j = 1 + my_j; j <= 4u * J && s0 + j < (uint32_t)P.nseg; j += J)
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(&P.units[(size_t)my_r * P.nseg + s0 + j].tau));
+    }
+    // Entry i of this lane's worker's run: sent?  position in the tile and value.  The first look
+    // at a staged entry leaves the answer in its place.
+    auto cand = [&](uint32_t i, bool first, uint32_t* pos, float* g) -> bool {
+        uint2* home = &cb[staged ? pbefore + i : 0u];
+        const uint2 ent = staged ? *home : run[i];
+        if (staged && !first) {                       // looked at before: the answer is in place
+            *pos = ent.x & (uint32_t)(STILE - 1);
+            *g = __uint_as_float(ent.y);
+            return (ent.x >> 31) != 0u;
+        }
+        const uint32_t idx = ent.x;
+        bool sent = idx >= e0 && idx - e0 < nel;                    // (an entry outside its tile is never written by the dense pass)
+        float gv = 0.0f;
+        if (sent) {
+            UnitLite u = un;
+            if (idx >= un.end) {                      // a later segment of the tile: look its unit up
+                uint32_t seg = gseg[(idx - e0) >> 7];
+                while (seg + 1 < (uint32_t)P.nseg && idx >= P.seg_off[seg + 1]) ++seg;
+                u = unit_lite(P, L, seg);
             }
-        } else {
-            for (uint32_t j = 0; j < 4 && e0 + j < P.d; ++j) {
-                const float v = P.x[e0 + j];
-                for (int w = 0; w < act.n; ++w) {
-                    P.xw[(size_t)act.r[w] * P.d + e0 + j] = v;
-                    if (P.anchors) P.anchors[(size_t)act.r[w] * P.d + e0 + j] = v;
+            const float val = __uint_as_float(ent.y);
+            const uint32_t key = RANDK ? ~philox_word(P, my_r, idx, 1u) : topk_key(val);
+            sent = key > u.tau || (key == u.tau && idx <= u.tie_max);
+            if (sent) {
+                if (P.qz == QS_NONE) {
+                    gv = val;
+                } else {
+                    int level = 1;
+                    if (!qz_is_sign(P.qz)) level = qsgd_level(val, u.norm, P.s, philox_word(P, my_r, idx, 0u));
+                    sent = level != 0;                             // (level 0: kept, not sent)
+                    if (sent) {                                    // the value as coord_value forms it
+                        if (qz_is_sign(P.qz)) {
+                            gv = u.norm / (float)u.k;
+                        } else {
+                            gv = (u.norm * (float)level) / (float)P.s;
+                            if (P.qz == QS_QSGD_SCALED) gv = gv * u.c;
+                        }
+                        if (val < 0.0f) gv = -gv;
+                    }
+                }
+            }
+        }
+        *pos = sent ? idx - e0 : 0u;
+        *g = gv;
+        // the worker's memory at a sent coordinate (quantizers that have no quantize stage of their own)
+        if (mem_update && sent && first) P.mem[(size_t)my_r * P.d + idx] = __uint_as_float(ent.y) - gv;
+        if (staged) *home = make_uint2(*pos | (sent ? 0x80000000u : 0u), __float_as_uint(gv));
+        return sent;
+    };
+    // senders per coordinate
+    for (uint32_t i = my_j; i < cnt; i += J) {
+        uint32_t pos = 0;
+        float g = 0.0f;
+        if (cand(i, true, &pos, &g)) {
+            const uint32_t bit = 1u << (pos & 31u);
+            if (atomicOr(&W.bm1[pos >> 5], bit) & bit) atomicOr(&W.bm2[pos >> 5], bit);
+        }
+    }
+    __syncwarp();
+    const uint32_t m_lo = W.bm2[lane], m_hi = W.bm2[lane + 32];
+    const bool any_multi = __any_sync(0xffffffffu, (m_lo | m_hi) != 0u);
+    // coordinates with one sender
+    for (uint32_t i = my_j; i < cnt; i += J) {
+        uint32_t pos = 0;
+        float g = 0.0f;
+        if (cand(i, false, &pos, &g) && !((W.bm2[pos >> 5] >> (pos & 31u)) & 1u)) {
+            float acc = 0.0f;
+            acc = acc + g;
+            xs[pos] = xs[pos] - acc / rdiv;
+        }
+    }
+    if (any_multi) {
+        // rank of a coordinate among those with several senders: popcounts before its word
+        const uint32_t c_lo = __popc(m_lo), c_hi = __popc(m_hi);
+        const uint32_t i_lo = warp_incl_scan(c_lo, lane), i_hi = warp_incl_scan(c_hi, lane);
+        const uint32_t n_lo = __shfl_sync(0xffffffffu, i_lo, 31);
+        const uint32_t npos = n_lo + __shfl_sync(0xffffffffu, i_hi, 31);
+        W.pref[lane] = i_lo - c_lo;
+        W.pref[lane + 32] = n_lo + i_hi - c_hi;
+        __syncwarp();
+        for (uint32_t w0 = 0; w0 < npos; w0 += wp) {
+            for (uint32_t i = my_j; i < cnt; i += J) {
+                uint32_t pos = 0;
+                float g = 0.0f;
+                if (!cand(i, false, &pos, &g)) continue;
+                const uint32_t wbits = W.bm2[pos >> 5];
+                if (!((wbits >> (pos & 31u)) & 1u)) continue;
+                const uint32_t rank = W.pref[pos >> 5] + __popc(wbits & ((1u << (pos & 31u)) - 1u));
+                if (rank < w0 || rank >= w0 + wp) continue;
+                const uint32_t at = atomicAdd(&W.nm, 1u);
+                if (at < (uint32_t)ML_CAP) { W.mpos[at] = pos | ((uint32_t)L.my_w << 16); W.mg[at] = g; }
+            }
+            __syncwarp();
+            const uint32_t n = W.nm < (uint32_t)ML_CAP ? W.nm : (uint32_t)ML_CAP;
+            if (W.nm > (uint32_t)ML_CAP) set_status(P, QS_STATE);          // a window holds at most wp x nact entries
+            for (uint32_t j = lane; j < n; j += 32) {
+                const uint32_t me = W.mpos[j], pos = me & 0xffffu, slot = me >> 16;
+                bool owner = true;
+                for (uint32_t i = 0; i < n; ++i) {
+                    const uint32_t o = W.mpos[i];
+                    if ((o & 0xffffu) == pos && (o >> 16) < slot) owner = false;
+                }
+                if (!owner) continue;
+                float acc = 0.0f;
+                int last = -1;
+                for (;;) {                            // the senders in increasing worker order
+                    int best = 1 << 30;
+                    float gb = 0.0f;
+                    for (uint32_t i = 0; i < n; ++i) {
+                        const uint32_t o = W.mpos[i];
+                        const int so = (int)(o >> 16);
+                        if ((o & 0xffffu) == pos && so > last && so < best) { best = so; gb = W.mg[i]; }
+                    }
+                    if (best == (1 << 30)) break;
+                    acc = acc + gb;
+                    last = best;
+                }
+                xs[pos] = xs[pos] - acc / rdiv;
+            }
+            __syncwarp();
+            if (lane == 0) W.nm = 0u;
+            __syncwarp();
+        }
+    }
+    __syncwarp();                                     // every lane is done with the tile and the bitmaps
+    // x in global memory: every changed coordinate's 32-byte sector, whole and once (a sector
+    // written in full needs no read of what it held), or the whole tile by the caller
+    const uint32_t b_lo = W.bm1[lane], b_hi = W.bm1[lane + 32];
+    const uint32_t changed = warp_sum(__popc(b_lo) + __popc(b_hi));
+    const bool whole = can_whole && changed >= WHOLE_TILE_MIN;
+    if (!whole && changed) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t bits = h ? b_hi : b_lo;
+            const uint32_t p0 = ((uint32_t)lane + 32u * h) * 32u;      // first position of the word
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (!((bits >> (8 * q)) & 0xffu)) continue;
+                const uint32_t p = p0 + 8u * q;
+                if (((reinterpret_cast<uintptr_t>(P.x + e0 + p)) & 31u) == 0 && p + 8u <= nel) {
+                    const float4 a = *reinterpret_cast<const float4*>(xs + p), b = *reinterpret_cast<const float4*>(xs + p + 4);
+                    *reinterpret_cast<float4*>(P.x + e0 + p) = a;
+                    *reinterpret_cast<float4*>(P.x + e0 + p + 4) = b;
+                } else {                              // rows off the 32-byte grid, or the ragged end: the changed coordinates alone
+                    for (uint32_t i = 0; i < 8u; ++i)
+                        if ((bits >> (8 * q + i)) & 1u) P.x[e0 + p + i] = xs[p + i];
                 }
             }
         }
     }
+    W.bm1[lane] = 0u; W.bm1[lane + 32] = 0u; W.bm2[lane] = 0u; W.bm2[lane + 32] = 0u;
+    return whole;
 }
 
-// The same broadcast through the bulk-copy engine (16-byte-aligned rows): one thread per block
-// brings tiles of x into a ring of three shared-memory buffers and sends each out to every active
-// worker's row; no data passes through registers.  Waits are bounded.
-__device__ void stage_broadcast_bulk(const Plan& P, const Active& act, float* buf0, float* buf1, float* buf2,
-                                     uint64_t* mbar, int* sh_abort) {
-    if (threadIdx.x != 0) return;
-    float* buf[3] = {buf0, buf1, buf2};
-    for (int b = 0; b < 3; ++b) mbar_init(&mbar[b], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    fence_async_smem();                              // the buffers were ordinary shared memory until now
-    // Tiles are handed out by a ticket counter: blocks that sit closer to the memory they touch
-    // take more of them, and all blocks finish together.  The next ticket is drawn one tile ahead
-    // so that its round trip is off the path.
-    const uint32_t ntiles = P.ntile;
-    uint32_t ticket = atomicAdd(P.bar + 2, 1u);
-    uint32_t t0 = 0, t1 = 0, t2 = 0, issued = 0;
-    bool more = true;
-    auto load = [&]() {                              // next tile into buffer issued % 3
-        if (!more) return;
-        const uint32_t t = ticket;
-        if (t >= ntiles) { more = false; return; }
-        ticket = atomicAdd(P.bar + 2, 1u);
-        const uint32_t b = issued % 3;
-        if (b == 0) t0 = t; else if (b == 1) t1 = t; else t2 = t;
-        const uint32_t e0 = t * (uint32_t)STILE;
-        const uint32_t bytes = (P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE) * 4u;
-        mbar_expect(&mbar[b], bytes);
-        bulk_load(buf[b], P.x + e0, bytes, &mbar[b]);
-        ++issued;
-    };
-    load();
-    load();
-    uint32_t done = 0;
-    for (uint32_t i = 0; i < issued; ++i) {
-        const uint32_t b = i % 3;
-        if (!mbar_wait(&mbar[b], (i / 3) & 1u)) { *sh_abort = 1; break; }
-        done = i + 1;
-        const uint32_t t = b == 0 ? t0 : b == 1 ? t1 : t2;
-        const uint32_t e0 = t * (uint32_t)STILE;
-        const uint32_t bytes = (P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE) * 4u;
-        for (int w = 0; w < act.n; ++w) {
-            bulk_store(P.xw + (size_t)act.r[w] * P.d + e0, buf[b], bytes);
-            if (P.anchors) bulk_store(P.anchors + (size_t)act.r[w] * P.d + e0, buf[b], bytes);
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+// bounded wait that also gives up when another warp of the block has
+__device__ __forceinline__ bool mbar_wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+    }
+}
+
+__device__ __forceinline__ uint32_t tile_count(const Plan& P, const LaneMap& L, uint32_t tile) {
+    uint32_t c = (L.live && tile < P.ntile) ? P.tile_cnt[(size_t)L.my_r * P.nblk * BLK_TILES + tile] : 0u;
+    return c < (uint32_t)STILE ? c : (uint32_t)STILE;
+}
+
+// 16-byte-aligned rows: warp 0 copies, warps 1 .. NWORK work on the tiles
+// pack_chunks > 0: the block's other warps write the records meanwhile (pack_by_warps)
+template <bool RANDK>
+__device__ void stage_update_broadcast(const Plan& P, const Active& act, BcBlock& B, bool mem_update, uint32_t pack_chunks,
+                                       uint32_t* wire, long long stride, long long* bits_out) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NSLOT; ++i) { mbar_init(&B.full[i], 1); mbar_init(&B.done[i], 1); }
+        B.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (wid >= 1 && wid <= NWORK) {
+        BcScratch& W = B.scr[wid - 1];
+        W.bm1[lane] = 0u; W.bm1[lane + 32] = 0u; W.bm2[lane] = 0u; W.bm2[lane + 32] = 0u;
+        if (lane == 0) W.nm = 0u;
+    }
+    fence_async_smem();                               // the buffers were ordinary shared memory until now
+    __syncthreads();
+    if (wid > NWORK) {
+        if (pack_chunks) pack_by_warps<RANDK>(P, pack_chunks, wire, stride, bits_out, lane);
+        return;
+    }
+    const LaneMap L = lane_map(act, lane);
+    const bool one_seg = P.nseg == 1;
+    const uint32_t ntile = P.ntile;
+    volatile int* abort_flag = &B.abort;
+    if (wid == 0) {
+        // ---- the copying warp
+        asm volatile("fence.proxy.async.global;" ::: "memory");   // x and the runs may have been written with ordinary stores
+        // tickets are drawn two tiles ahead of the copies and counts read one tile ahead, so that
+        // neither round trip is on the path
+        uint32_t tA = 0, tB = 0;
+        if (lane == 0) { tA = atomicAdd(P.bar + 2, 1u); tB = atomicAdd(P.bar + 2, 1u); }
+        tA = __shfl_sync(0xffffffffu, tA, 0);
+        tB = __shfl_sync(0xffffffffu, tB, 0);
+        auto gseg_of = [&](uint32_t tile) -> uint32_t {
+            return (!one_seg && lane < STILE / GROUP && tile < ntile) ? P.grp_seg[(size_t)tile * (STILE / GROUP) + lane] : 0u;
+        };
+        uint32_t cntA = tile_count(P, L, tA), gsA = gseg_of(tA);
+        // starts the copies of the next tile into slot s (or leaves the end mark there)
+        auto arm = [&](uint32_t s) {
+            BcSlot& S = B.slot[s];
+            const uint32_t tile = tA;
+            uint32_t tC = 0;
+            if (lane == 0) tC = atomicAdd(P.bar + 2, 1u);
+            const uint32_t cntB = tile_count(P, L, tB), gsB = gseg_of(tB);
+            if (tile >= ntile) {
+                if (lane == 0) { S.tile = NO_TILE; mbar_expect(&B.full[s], 0u); }
+            } else {
+                const uint32_t e0 = tile * (uint32_t)STILE;
+                const uint32_t nel = P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE;
+                const uint32_t padded = L.my_j == 0u ? (cntA + 1u) & ~1u : 0u;
+                const uint32_t pincl = warp_incl_scan(padded, lane);
+                const uint32_t ptotal = __shfl_sync(0xffffffffu, pincl, 31);
+                const bool staged = ptotal <= (uint32_t)CB;
+                if (L.my_j == 0u) { S.cnt[L.my_w] = cntA; S.pbefore[L.my_w] = pincl - padded; }
+                if (lane < STILE / GROUP) S.gseg[lane] = gsA;
+                if (lane == 0) {
+                    S.tile = tile;
+                    S.staged = staged ? 1u : 0u;
+                    mbar_expect(&B.full[s], nel * 4u + (staged ? ptotal * 8u : 0u));
+                    bulk_load(S.xs, P.x + e0, nel * 4u, &B.full[s]);
+                }
+                __syncwarp();                         // the bytes are announced before any run's copy starts
+                if (staged && cntA && L.my_j == 0u)
+                    bulk_load(&S.cb[pincl - padded], P.stage + (size_t)L.my_r * P.cap + (size_t)tile * STILE, padded * 8u, &B.full[s]);
+            }
+            tA = tB; cntA = cntB; gsA = gsB;
+            tB = __shfl_sync(0xffffffffu, tC, 0);
+            __syncwarp();                             // the slot's header is visible to the whole warp
+        };
+        uint32_t armed = 0;                           // tiles (or end marks) whose slot has been armed
+        for (; armed < (uint32_t)(NSLOT - 1); ++armed) arm(armed);
+        uint32_t si = 0;
+        for (;; ++si) {
+            const uint32_t s = si % NSLOT;
+            BcSlot& S = B.slot[s];
+            const uint32_t tile = S.tile;             // written by this warp
+            if (tile == NO_TILE) break;
+            const bool ok = mbar_wait_or_abort(&B.done[s], (si / NSLOT) & 1u, abort_flag);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            if (lane == 0) {
+                const uint32_t e0 = tile * (uint32_t)STILE;
+                const uint32_t nel = P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE;
+                if (S.whole) bulk_store(P.x + e0, S.xs, nel * 4u);
+                for (int w = 0; w < act.n; ++w) {
+                    bulk_store(P.xw + (size_t)act.r[w] * P.d + e0, S.xs, nel * 4u);
+                    if (P.anchors) bulk_store(P.anchors + (size_t)act.r[w] * P.d + e0, S.xs, nel * 4u);
+                }
+                bulk_commit();
+                bulk_wait_read<1>();                  // the stores of the tile before have read their slot: it is armed next
+            }
+            __syncwarp();
+            arm(armed % NSLOT);
+            ++armed;
         }
-        bulk_commit();
-        if (more) {
-            bulk_wait_read<1>();                     // the buffer of tile i - 1 has been read by its stores
-            load();
+        if (!*abort_flag) {
+            // the slot that has not seen an end mark yet (only its header is written: the stores that
+            // may still be reading its tile are not disturbed)
+            arm(armed % NSLOT);
+            ++armed;
+        }
+        if (*abort_flag) {
+            // copies already started get a bounded chance to land before the block leaves
+            for (uint32_t i = si; i < armed; ++i) mbar_wait(&B.full[i % NSLOT], (i / NSLOT) & 1u);
+            if (lane == 0) set_status(P, QS_TIMEOUT);
+        }
+        if (lane == 0) bulk_wait_all();               // nothing of this block may still be reading shared memory
+    } else {
+        // ---- a working warp: the tiles that come through slot wid - 1
+        BcScratch& W = B.scr[wid - 1];
+        UnitLite un = unit_lite(P, L, 0u);
+        const uint32_t s = (uint32_t)(wid - 1);
+        BcSlot& S = B.slot[s];
+        for (uint32_t use = 0;; ++use) {
+            const bool ok = mbar_wait_or_abort(&B.full[s], use & 1u, abort_flag);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            const uint32_t tile = S.tile;
+            if (tile == NO_TILE) break;
+            if (!one_seg) un = unit_lite(P, L, S.gseg[0]);
+            const uint32_t cnt = L.live ? S.cnt[L.my_w] : 0u;
+            const bool whole = apply_tile<RANDK>(P, L, lane, tile, cnt, S.staged != 0u, S.cb, L.live ? S.pbefore[L.my_w] : 0u, S.gseg, S.xs,
+                                                 W, un, mem_update, true);
+            if (lane == 0) S.whole = whole ? 1u : 0u;
+            fence_async_smem();                       // the tile as updated must be what the bulk stores read
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&B.done[s]);
         }
     }
-    if (*sh_abort) {
-        // loads already issued get a bounded chance to land before the block leaves
-        for (uint32_t i = done; i < issued; ++i) mbar_wait(&mbar[i % 3], (i / 3) & 1u);
-        set_status(P, QS_TIMEOUT);
+}
+
+// rows that are not 16-byte aligned: warps 0 .. NWORK - 1 take a tile each by ticket, ordinary loads and stores
+template <bool RANDK>
+__device__ void stage_update_broadcast_plain(const Plan& P, const Active& act, BcBlock& B, bool mem_update, uint32_t pack_chunks,
+                                             uint32_t* wire, long long stride, long long* bits_out) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (wid >= NWORK) {
+        if (pack_chunks) pack_by_warps<RANDK>(P, pack_chunks, wire, stride, bits_out, lane);
+        return;
     }
-    bulk_wait_all();
+    BcScratch& W = B.scr[wid];
+    float* xs = B.slot[wid].xs;
+    uint32_t* gseg = B.slot[wid].gseg;
+    W.bm1[lane] = 0u; W.bm1[lane + 32] = 0u; W.bm2[lane] = 0u; W.bm2[lane + 32] = 0u;
+    if (lane == 0) W.nm = 0u;
+    __syncwarp();
+    const LaneMap L = lane_map(act, lane);
+    const bool one_seg = P.nseg == 1;
+    UnitLite un = unit_lite(P, L, 0u);
+    for (;;) {
+        uint32_t tile = 0;
+        if (lane == 0) tile = atomicAdd(P.bar + 2, 1u);
+        tile = __shfl_sync(0xffffffffu, tile, 0);
+        if (tile >= P.ntile) break;
+        const uint32_t e0 = tile * (uint32_t)STILE;
+        const uint32_t nel = P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE;
+        for (uint32_t i = lane; i < nel; i += 32) xs[i] = P.x[e0 + i];
+        if (lane < STILE / GROUP) gseg[lane] = one_seg ? 0u : P.grp_seg[(size_t)tile * (STILE / GROUP) + lane];
+        __syncwarp();
+        if (!one_seg) un = unit_lite(P, L, gseg[0]);
+        apply_tile<RANDK>(P, L, lane, tile, tile_count(P, L, tile), false, nullptr, 0u, gseg, xs, W, un, mem_update, false);
+        __syncwarp();
+        for (int w = 0; w < act.n; ++w)
+            for (uint32_t i = lane; i < nel; i += 32) {
+                const float v = xs[i];
+                P.xw[(size_t)act.r[w] * P.d + e0 + i] = v;
+                if (P.anchors) P.anchors[(size_t)act.r[w] * P.d + e0 + i] = v;
+            }
+        __syncwarp();
+    }
 }
 
 // ------------------------------------------------------------------ the persistent kernel
+// In a whole round with a level-1 quantizer (sign, none) nothing of the records depends on the
+// closing stage and nothing of the closing stage on the records: both start from the thresholds
+// and norms.  When the chunks are few enough (a couple per packing warp) the records are written
+// by the warps that have no part in the closing stage, in its shadow; otherwise, and for QSGD
+// (whose levels need a stage of their own first), every block packs its share before it.
+constexpr uint32_t PACK_WARPS = BT / 32 - 1 - NWORK;      // warps of a block free to pack during the closing stage
+constexpr uint32_t PACK_CHUNKS_PER_WARP = 2;
+
 template <bool RANDK>
 __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_scan[33];
@@ -2083,15 +2469,19 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
     __shared__ uint32_t sh_cnt[2 * 8 * GPW];
     __shared__ uint32_t sh_flag[4];
     __shared__ int sh_abort;
-    // unit table (three arrays) / candidate-count sums of the order stage / tile buffers of the broadcast
-    __shared__ __align__(128) uint32_t sh_tab[ORDER_ITEMS_MAX + 8];
+    // One pool of dynamic shared memory (MID_POOL_BYTES).  Its first part is the unit table (four
+    // arrays) / the candidate-count sums of the order stage, then 8 KB of stage scratch (fallback
+    // bins / radix bins / exponent sums / UnitSh); the closing stage takes all of it for its warps'
+    // buffers.
+    extern __shared__ __align__(128) unsigned char sh_pool[];
+    uint32_t* sh_tab = reinterpret_cast<uint32_t*>(sh_pool);
+    unsigned char* sh_big = sh_pool + (ORDER_ITEMS_MAX + 8) * sizeof(uint32_t);
+    static_assert(MID_SCRATCH_BYTES <= MID_POOL_BYTES, "the stages' scratch must fit the pool");
     uint32_t* t_start = sh_tab;
     uint32_t* t_c = sh_tab + UT_MAX;
     uint32_t* t_cb = sh_tab + 2 * UT_MAX;         // UT_MAX + 1 entries
     uint32_t* t_lb = sh_tab + 3 * UT_MAX + 4;     // UT_MAX + 1 entries
     static_assert(4 * UT_MAX + 5 <= ORDER_ITEMS_MAX + 8, "the unit table must fit");
-    __shared__ __align__(8) uint64_t sh_mbar[3];
-    __shared__ __align__(16) unsigned char sh_big[FB_BINS * 4];   // fallback bins / radix bins / exponent sums / UnitSh
     static_assert(sizeof(UnitSh) <= FB_BINS * 4, "the unit stage's scratch must fit");
     const Plan& P = a.P;
     const Active& act = a.act;
@@ -2104,8 +2494,10 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         P.trace[0] = t;
         for (int i = 1; i < TRACE_SLOTS; ++i) P.trace[i] = 0;
     }
-#define QS_BARRIER() do { if (!grid_barrier(P, target, &sh_abort)) return; } while (0)
+    // a barrier that gives up ends the stages; the block still takes part in the closing count below
+#define QS_BARRIER() if (!grid_barrier(P, target, &sh_abort)) break
 
+    do {
     if (a.do_pack) {
         // the records are built with OR: start from zero words (a later barrier precedes their use)
         for (int w = 0; w < act.n; ++w) {
@@ -2114,14 +2506,11 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         }
     }
     Tab tab;
-    const bool fused = a.do_compress && a.do_pack && a.do_decode;   // whole round: the master update rides along
-    if (fused) {
-        const uint32_t nw = 2u * ((P.d + 31u) >> 5);          // the two bitmaps are one allocation
-        for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < nw; i += gridDim.x * BT) P.bm1[i] = 0u;
-    }
+    const bool fused = a.do_compress && a.do_pack && a.do_decode;   // whole round: the master update is part of the closing stage
     const bool merge = fused && qz_early(P.qz);                     // level-1 quantizers: no quantize stage of its own
+    bool warp_pack = false;                                          // the records are written in the closing stage's shadow
     if (a.do_compress) {
-        const bool even = P.nsup * (uint32_t)act.n <= ORDER_SUPS_MAX;
+        const bool even = P.nsup * (uint32_t)act.n <= P.order_sups_max;
         if (even) stage_order_even<RANDK>(P, act, 0u, bins, sh_tab, sh_scan);
         else stage_order<RANDK>(P, act, 0u, bins);
         QS_BARRIER();
@@ -2144,6 +2533,8 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
             for (int w = 0; w < act.n; ++w) cands += P.seg_start[(size_t)act.r[w] * (P.nseg + 1) + P.nseg];
             atomicAdd((unsigned long long*)&P.stats[1], cands);
         }
+        warp_pack = merge && tab.fast && !P.block_pack && tab.total_chunks <= PACK_CHUNKS_PER_WARP * PACK_WARPS * gridDim.x;
+        if (warp_pack) publish_table(P, tab);
         // the candidate counts have been consumed: clear them for the next dense pass
         for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nblk; i += gridDim.x * BT) P.blk_count[i] = 0;
         for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nsup; i += gridDim.x * BT) P.sup_count[i] = 0;
@@ -2153,10 +2544,12 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         if (tab.any_short) stage_unit<RANDK>(P, tab, act, merge, *reinterpret_cast<UnitSh*>(sh_big), sh_w);
         QS_BARRIER();
         if (tab.total_long) {
+            bool gave_up = false;
             for (int level = 2; level < 4; ++level) {
                 stage_hist<RANDK>(P, tab, level, bins, &sh_small[0], &sh_small[1]);
-                QS_BARRIER();
+                if (!grid_barrier(P, target, &sh_abort)) { gave_up = true; break; }
             }
+            if (gave_up) break;
             stage_final<RANDK>(P, tab, &sh_small[2], sh_w);
             QS_BARRIER();
             if (P.fail[0]) {                       // some long list has more equal keys than slots (same in every block)
@@ -2168,26 +2561,32 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
             stage_norm_accum<RANDK>(P, tab, merge, reinterpret_cast<uint32_t(*)[4]>(sh_big), &sh_small[0], sh_w, sh_cnt);
             QS_BARRIER();
         }
+    } else if (a.do_pack) {
+        build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab);
+        QS_BARRIER();                              // the zeroed records
+    }
+    // Thresholds, tie cuts and norms are known.
+    if (a.do_compress) {
         if (!merge) {
-            stage_quant<RANDK>(P, tab, fused, &sh_small[0], sh_w);
+            stage_quant<RANDK>(P, tab, &sh_small[0], sh_w);
             QS_BARRIER();
         }
         if (!tab.fast) {
             stage_chunk_scan(P, tab, act, sh_scan);
             QS_BARRIER();
         }
-    } else if (a.do_pack) {
-        build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab);
-        QS_BARRIER();                              // the zeroed records
     }
-    if (a.do_pack) {
+    if (a.do_pack && !warp_pack) {
         if (!tab.fast) stage_pack_dir(P, act, a.wire, a.stride, a.bits_out);
-        stage_pack<RANDK>(P, tab, fused, merge, a.wire, a.stride, a.bits_out, &sh_small[0], sh_scan);
-        if (a.do_decode) QS_BARRIER();
+        stage_pack<RANDK>(P, tab, merge, a.wire, a.stride, a.bits_out, &sh_small[0], sh_scan);
     }
     if (fused) {
-        stage_coll_apply(P);
+        const uint32_t pack_chunks = warp_pack ? tab.total_chunks : 0u;
+        __syncthreads();                           // the unit table and the scratch change hands: the closing stage's buffers now
+        if (a.aligned) stage_update_broadcast<RANDK>(P, act, *reinterpret_cast<BcBlock*>(sh_pool), merge, pack_chunks, a.wire, a.stride, a.bits_out);
+        else stage_update_broadcast_plain<RANDK>(P, act, *reinterpret_cast<BcBlock*>(sh_pool), merge, pack_chunks, a.wire, a.stride, a.bits_out);
     } else if (a.do_decode) {
+        if (a.do_pack) QS_BARRIER();
         if (P.nseg > 1) {
             stage_dec_prep(P, act, a.wire, a.stride, sh_scan);
             QS_BARRIER();
@@ -2196,32 +2595,24 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         QS_BARRIER();
         stage_dec_apply(P, act, a.wire, a.stride, a.patch);
     }
-    if (a.do_broadcast) {
-        QS_BARRIER();
-        if (a.aligned) {
-            // the unit table is no longer needed: its three arrays are the tile buffers
-            stage_broadcast_bulk(P, act, reinterpret_cast<float*>(t_start), reinterpret_cast<float*>(t_c),
-                                 reinterpret_cast<float*>(t_cb), sh_mbar, &sh_abort);
-        } else {
-            stage_broadcast<false>(P, act);
-        }
-    }
+    } while (0);
 #undef QS_BARRIER
     // the last block to leave resets the barrier for the next launch
     __syncthreads();
-    if (P.trace && blockIdx.x == 0 && threadIdx.x == 0) {
+    if (P.trace && threadIdx.x == 0) {             // when block 0 was done, and when the last block was
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        P.trace[TRACE_SLOTS - 1] = t;
+        if (blockIdx.x == 0) P.trace[TRACE_SLOTS - 2] = t;
+        atomicMax(P.trace + TRACE_SLOTS - 1, t);
     }
     if (threadIdx.x == 0) {
         if (atomicAdd(P.bar + 1, 1u) == gridDim.x - 1) {
             P.bar[0] = 0;
             P.bar[1] = 0;
-            P.bar[2] = 0;                            // tile tickets of the broadcast
+            P.bar[2] = 0;                            // tile tickets of the closing stage
             P.bar[3] = 0;                            // tile tickets of the next dense pass
             P.bar[4] = 0;                            // unit tickets
-            *P.ncoll = 0;
+            P.bar[6] = 0;                            // chunk tickets of the packing warps
         }
     }
 }
@@ -2244,8 +2635,11 @@ __global__ void __launch_bounds__(256) export_kernel(const Plan P, long long* se
 // ------------------------------------------------------------------ launchers
 int mid_blocks_per_sm(bool randk) {
     int per_sm = 0;
-    const cudaError_t e = randk ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mid_kernel<true>, BT, 0)
-                                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mid_kernel<false>, BT, 0);
+    cudaError_t e = randk ? cudaFuncSetAttribute(mid_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MID_POOL_BYTES)
+                          : cudaFuncSetAttribute(mid_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MID_POOL_BYTES);
+    if (e != cudaSuccess) return 0;
+    e = randk ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mid_kernel<true>, BT, MID_POOL_BYTES)
+              : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mid_kernel<false>, BT, MID_POOL_BYTES);
     return e == cudaSuccess ? per_sm : 0;
 }
 
@@ -2259,7 +2653,7 @@ cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do
     a.wire = wire; a.stride = stride; a.wire_words = wire_words; a.bits_out = bits_out;
     void* params[] = {&a};
     const void* fn = P.sp == QS_RANDK ? (const void*)mid_kernel<true> : (const void*)mid_kernel<false>;
-    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(BT), params, 0, st);
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(BT), params, MID_POOL_BYTES, st);
 }
 
 void launch_export(const Plan& P, long long* sel_idx, int* level, uint8_t* sign, float* norm, long long* n,
