@@ -659,17 +659,37 @@ __device__ __forceinline__ ChunkCtx long_chunk_context(const Plan& P, const Tab&
 // A block takes consecutive chunks; while they lie in one unit the prefix is worked out once and
 // the counts stay in shared memory, to be added to the unit's histogram in one go.
 template <bool RANDK>
-__device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* sh_hist, uint32_t* sh_u, uint32_t* sh_prefix) {
+__device__ void final_unit(const Plan& P, const Tab& tab, uint32_t u, uint32_t* sh4, uint32_t* sh_w);
+
+// At the last level the block whose counts complete a unit (a count of finished chunks per unit)
+// goes on to the unit's threshold, tie cut and prediction at once: no stage of its own for that.
+template <bool RANDK>
+__device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* sh_hist, uint32_t* sh_u, uint32_t* sh_prefix,
+                           uint32_t* sh4, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31;
     const uint32_t total = tab.total_long;
     const int shift = 24 - 8 * level;
     const uint32_t share = (total + gridDim.x - 1) / gridDim.x;
     const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
-    uint32_t held = 0xffffffffu, prefix = 0;
+    uint32_t held = 0xffffffffu, prefix = 0, nheld = 0;
     auto flush = [&]() {
         __syncthreads();                              // every add of the held chunks has been made
         const uint32_t v = sh_hist[threadIdx.x];
         if (v) atomicAdd(&P.hist[((size_t)level * P.U + held) * 256 + threadIdx.x], v);
+        if (level == 3) {
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const uint32_t nch = tab.cb[held + 1] - tab.cb[held];
+                const bool last = atomicAdd(&P.units[held].done, nheld) == nch - nheld;
+                if (last) __threadfence();
+                *sh_prefix = last ? 1u : 0u;
+            }
+            __syncthreads();
+            if (*sh_prefix) final_unit<RANDK>(P, tab, held, sh4, sh_w);
+            __syncthreads();
+        }
+        nheld = 0;
     };
     ChunkCtx c;
     for (uint32_t chunk = c_lo; chunk < c_hi; ++chunk) {
@@ -692,6 +712,7 @@ __device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* s
             __syncthreads();
             prefix = *sh_prefix;
         }
+        ++nheld;
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
@@ -720,13 +741,13 @@ __device__ void predict_floor(const Plan& P, uint32_t r, uint32_t seg, uint32_t 
     *gp = __float_as_uint(tn) << 1;
 }
 
-// threshold key, tie cut and next prediction of each unit; clears its histograms
+// threshold key, tie cut and next prediction of one long unit, by the whole block, once every
+// level of its select has been counted; clears its histograms
 template <bool RANDK>
-__device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32_t* sh_w) {
+__device__ void final_unit(const Plan& P, const Tab& tab, uint32_t u, uint32_t* sh4, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (uint32_t u = blockIdx.x; u < P.U; u += gridDim.x) {
+    {
         const uint32_t uc = tab.c[u];
-        if (uc <= tab.short_c) continue;           // no candidates (idle worker), or a block did the unit on its own
         const uint32_t seg = u % P.nseg, r = u / P.nseg, k = P.kseg[seg];
         __syncthreads();
         if (wid == 0) {
@@ -777,6 +798,7 @@ __device__ void stage_final(const Plan& P, const Tab& tab, uint32_t* sh4, uint32
             out.emin = 255u;
             out.emax = 0u;
             out.norm = 0.0f;
+            out.done = 0;
             if (!RANDK) predict_floor(P, r, seg, tau, uc, k);
         }
     }
@@ -864,6 +886,12 @@ __device__ void stage_tie_find(const Plan& P, const Tab& tab, uint32_t* sh, uint
 }
 
 // ------------------------------------------------------------------ quantize
+// The closing stage will change the worker's memory at a kept coordinate while the memory system
+// is busy with its copies: ask for the sector now, while it is idle, and to keep it in the L2.
+__device__ __forceinline__ void mem_ahead(const Plan& P, uint32_t r, uint32_t idx) {
+    asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(P.mem + (size_t)r * P.d + idx));
+}
+
 template <bool RANDK>
 __device__ __forceinline__ bool is_kept(const Unit& un, uint32_t sk, uint32_t idx) {
     return sk > un.tau || (sk == un.tau && idx <= un.tie_max);
@@ -1016,6 +1044,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
         for (int i = 0; i < PER; ++i) {
             const uint32_t off = c.first + i * BT + threadIdx.x;
             kept[i] = off < c.c && is_kept<RANDK>(c.un, key[i], idx[i]);
+            if (early && kept[i]) mem_ahead(P, c.r, idx[i]);
         }
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
@@ -1295,6 +1324,9 @@ __device__ void unit_by_warp(const Plan& P, const Tab& tab, uint32_t u, uint32_t
     const uint32_t tau = __shfl_sync(0xffffffffu, hit0 ? key[0] : key[1], src);
     const uint32_t tie_max = __shfl_sync(0xffffffffu, hit0 ? idx[0] : idx[1], src);
     if (early) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+            if (kept[q]) mem_ahead(P, r, idx[q]);
         const uint32_t n = __popc(__ballot_sync(0xffffffffu, kept[0])) + __popc(__ballot_sync(0xffffffffu, kept[1]));
         if (lane == 0) P.chunk_cnt[tab.cb[u]] = n | (n << 16);             // a list this short is one chunk
     }
@@ -1420,6 +1452,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             const bool kept = off < c && kv >= tau && !(ties && kv == tau && idx > tie_max);
             const uint32_t live = __ballot_sync(0xffffffffu, kept);
             if (early && lane == 0 && live) atomicAdd(&S.kept[i / PER], __popc(live));
+            if (early && kept) mem_ahead(P, r, idx);
             if (kept && !plain) {
                 const uint32_t b = RANDK ? vb : (kv >> 1);
                 const uint32_t e = (b >> 23) & 255u;
@@ -1432,8 +1465,8 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             return 0u;
         };
         auto none = [](uint32_t, uint32_t) {};
-        // the indices are needed for a tie cut; Rand_k reads the values too
-        if (ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, none);
+        // the indices are needed for a tie cut and for the request above; Rand_k reads the values too
+        if (early || ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, none);
         else unit_rows<RANDK, 16, false>(P, base, c, key, take, none);
         __syncthreads();
         if (wid == 0) {
@@ -2539,19 +2572,17 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nblk; i += gridDim.x * BT) P.blk_count[i] = 0;
         for (uint32_t i = blockIdx.x * BT + threadIdx.x; i < (uint32_t)P.R * P.nsup; i += gridDim.x * BT) P.sup_count[i] = 0;
         // select: the first radix level of the long units, and the short units whole, block by block
-        if (tab.total_long) stage_hist<RANDK>(P, tab, 1, bins, &sh_small[0], &sh_small[1]);
+        if (tab.total_long) stage_hist<RANDK>(P, tab, 1, bins, &sh_small[0], &sh_small[1], &sh_small[2], sh_w);
         __syncthreads();                           // the scratch changes hands
         if (tab.any_short) stage_unit<RANDK>(P, tab, act, merge, *reinterpret_cast<UnitSh*>(sh_big), sh_w);
         QS_BARRIER();
         if (tab.total_long) {
             bool gave_up = false;
-            for (int level = 2; level < 4; ++level) {
-                stage_hist<RANDK>(P, tab, level, bins, &sh_small[0], &sh_small[1]);
+            for (int level = 2; level < 4; ++level) {          // (the last level ends with each unit's threshold and tie cut)
+                stage_hist<RANDK>(P, tab, level, bins, &sh_small[0], &sh_small[1], &sh_small[2], sh_w);
                 if (!grid_barrier(P, target, &sh_abort)) { gave_up = true; break; }
             }
             if (gave_up) break;
-            stage_final<RANDK>(P, tab, &sh_small[2], sh_w);
-            QS_BARRIER();
             if (P.fail[0]) {                       // some long list has more equal keys than slots (same in every block)
                 stage_tie_count<RANDK>(P, tab, &sh_small[0], sh_w);
                 QS_BARRIER();
