@@ -19,7 +19,7 @@ constexpr int SUP_BLOCKS = 64;       // blocks per super-block of the two-level 
 constexpr int CHUNK = QS_CHUNK;     // candidates per selection chunk (a multiple of the 256 threads)
 constexpr int UT_MAX = 2048;         // units whose table fits in the persistent kernel's shared memory
 constexpr uint32_t ORDER_SUPS_MAX = 2048;   // (worker, super-block) sums the order stage can hold in shared memory
-constexpr int UNIT_CAP = 4096;       // candidates of a unit that one block may select from on its own (16 per thread)
+constexpr int UNIT_CAP = 6144;       // candidates of a unit that one block may select from on its own (16 per thread)
 constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (top 11 key bits)
 constexpr int FB_SHIFT = 21;
 constexpr int FB_CHUNK = 65536;      // coordinates per fallback-histogram block

@@ -412,7 +412,7 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
                 c = ss[seg + 1] - start;
                 if (c < P.kseg[seg]) atomicOr(sh_flag, 1u << r);
                 atomicMax(sh_flag + 1, c);
-                if (c) atomicAdd(sh_flag + 2, 1u);
+                if (c > (uint32_t)BT && c <= P.unit_cap) atomicAdd(sh_flag + 2, 1u);   // lists that would keep a block busy for a while
             }
         }
         uint32_t total;
@@ -427,11 +427,12 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
     // the streams' places: one segment, or a quantizer that sends every kept entry (fixed places)
     tab->fast = (P.nseg == 1 || qz_early(P.qz)) && (longest + CHUNK - 1) / CHUNK <= 1024u;
     // Which units one block selects from on its own (block barriers only), and which take the
-    // grid-wide radix levels: all of them in a block each when every list is short and there is a
-    // block per unit; otherwise only the lists of at most one candidate per thread.
+    // grid-wide radix levels: every list up to the cap when there is a block for each list that
+    // would keep one busy for a while (lists are dealt largest first); otherwise only the lists of
+    // at most one candidate per thread.
     uint32_t short_c = 0;
     if (P.unit_cap) {
-        const bool all = longest <= P.unit_cap && sh_flag[2] <= gridDim.x;
+        const bool all = sh_flag[2] <= gridDim.x;
         short_c = all ? P.unit_cap : (P.unit_cap < (uint32_t)BT ? P.unit_cap : (uint32_t)BT);
     }
     tab->short_c = short_c;
@@ -1406,7 +1407,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
                 S.hist[threadIdx.x] = 0u;
                 __syncthreads();
                 const uint32_t prefix = S.ctl[1];
-                unit_rows<RANDK, 16, false>(P, base, c, key, [&](uint32_t, uint32_t off, uint32_t kv, uint32_t, uint32_t) {
+                unit_rows<RANDK, 8, false>(P, base, c, key, [&](uint32_t, uint32_t off, uint32_t kv, uint32_t, uint32_t) {
                     const bool valid = off < c && (level == 0 || (kv >> (32 - 8 * level)) == prefix);
                     if (valid) atomicAdd(&S.hist[(kv >> shift) & 255u], 1u);
                     return 0u;
@@ -1467,7 +1468,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
         auto none = [](uint32_t, uint32_t) {};
         // the indices are needed for a tie cut and for the request above; Rand_k reads the values too
         if (early || ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, none);
-        else unit_rows<RANDK, 16, false>(P, base, c, key, take, none);
+        else unit_rows<RANDK, 8, false>(P, base, c, key, take, none);
         __syncthreads();
         if (wid == 0) {
             // exponent range of the sums
