@@ -30,7 +30,8 @@
  *     word that qs_sync_status reads after synchronising the stream.
  *   - Status codes: QS_OK = 0, negative = error.  Nothing is printed, nothing aborts.
  *   - worker_mask: host array of R bytes, non-zero = worker takes part; NULL = all.
- *   - R <= 32, 1 <= k <= d < 2^32, 1 <= s <= 65535, round < 2^56, R x nseg <= 2048.
+ *   - R <= 32, 1 <= k <= d <= 2^32 - 4096 (coordinates are counted in 32 bits, in tiles of
+ *     2048), 1 <= s <= 65535, round < 2^56, R x nseg <= 2048.
  *
  * Arithmetic (identical, operation for operation, to the CPU checker under oracle/):
  *   fp32 with no fused multiply-add; u = mem + (x - xw); Top_k orders by the bit
@@ -99,10 +100,17 @@ enum {
  * segment [0, d) with k is installed.  Returns QS_INVALID_ARG, QS_ALLOC or QS_CUDA on
  * failure, in which case *out is NULL.
  * Read from the environment here, for tuning and tests (results never depend on them):
- * QSPARSE_UNIT_CAP (0..4096, default 4096: the longest candidate list that one thread
+ * QSPARSE_UNIT_CAP (0..6144, default 6144: the longest candidate list that one thread
  * block may select from on its own; 0 sends every list through the grid-wide radix
- * levels), QSPARSE_MID_PER_SM (thread blocks of the persistent kernel per SM, default
- * 4), QSPARSE_NO_TMA (dense pass with plain loads), QSPARSE_TMA_DEPTH (its ring depth).
+ * levels), QSPARSE_ORDER_EVEN_MAX (0..2048, default 2048: (worker, super-block) pairs up to
+ * which the order stage deals candidates evenly; 0 = always by region), QSPARSE_BLOCK_PACK
+ * (whole rounds pack the records block by block before the closing stage, not by spare warps
+ * beside it), QSPARSE_MID_PER_SM (thread blocks of the persistent kernel per SM, default
+ * 4), QSPARSE_NO_TMA (dense pass with plain loads), QSPARSE_TMA_DEPTH (its ring depth),
+ * QSPARSE_SPIN_LIMIT (polls a grid barrier waits before it gives up with QS_TIMEOUT; default
+ * 2^22, about a second) and QSPARSE_TEST_MISS_BARRIER (test of that path: in the first
+ * persistent launch of the context one block stays away from the first barrier, so that every
+ * other block's bounded wait runs out).
  */
 int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t seed,
             void* cuda_stream);
@@ -248,7 +256,10 @@ int64_t qs_record_bits(const qs_ctx* ctx, const int64_t* n);
 int64_t qs_total_k(const qs_ctx* ctx);
 
 /* Synchronises the stream and returns the first error recorded on the device since the
- * last call (QS_OK if none), clearing it. */
+ * last call (QS_OK if none), clearing it.  After a device-side error (QS_NONFINITE,
+ * QS_TIMEOUT, QS_STATE) the round that hit it is void: its outputs are undefined, and this call
+ * also puts the library's scratch back into its starting state, so call it before the next
+ * round. */
 int qs_sync_status(qs_ctx* ctx);
 /* Text of the last host-side error of this context (never NULL). */
 const char* qs_last_error(const qs_ctx* ctx);
@@ -270,9 +281,9 @@ int qs_get_stats(qs_ctx* ctx, int64_t* out, int n);
  * qs_enable_phase_timing / qs_get_phase_timing — measurement aid, not part of the method:
  * when on, qs_sync_round records CUDA events on the context's stream around its dense pass.
  * qs_get_phase_timing synchronises and returns, summed over the rounds since the last call
- * and then cleared: ms[0] the dense pass (form u, candidate flags, old-model broadcast: one
- * kernel launch per round), ms[1] the rest of the round (selection, quantizer, memory update,
- * pack, decode, update: one persistent kernel), ms[2] the number of rounds.  Writes
+ * and then cleared: ms[0] the dense pass (form u, candidate flags and runs: one kernel launch
+ * per round), ms[1] the rest of the round (selection, quantizer, memory update, pack, master
+ * update and broadcast: one persistent kernel), ms[2] the number of rounds.  Writes
  * min(n, 3) values.
  */
 int qs_enable_phase_timing(qs_ctx* ctx, int on);
@@ -281,8 +292,8 @@ int qs_get_phase_timing(qs_ctx* ctx, double* ms, int n);
 /*
  * qs_get_stage_trace — measurement aid: microseconds, from the start of the last persistent
  * kernel of this context, at which each of its grid barriers completed (us[1], us[2], ...,
- * -1 = not reached) and left the kernel (us[31]); us[0] = 0.  Synchronises the stream.
- * Writes min(n, 32) values.
+ * -1 = not reached), block 0 left the kernel (us[30]) and the last block did (us[31]);
+ * us[0] = 0.  Synchronises the stream.  Writes min(n, 32) values.
  */
 int qs_get_stage_trace(qs_ctx* ctx, double* us, int n);
 
@@ -300,7 +311,9 @@ int qs_get_stage_trace(qs_ctx* ctx, double* us, int n);
  * that loads the library therefore holds QS_STATIC_MAX_D words (4 MiB) until the process ends.
  *
  *   R, d, k, s, quantizer   as in qs_init, one segment [0, d); d <= QS_STATIC_MAX_D, else
- *                           QS_TOO_LARGE is returned and nothing is enqueued.
+ *                           QS_TOO_LARGE is returned and nothing is enqueued.  QS_NONE (the
+ *                           sparsifier alone, 32-bit values in the record) is not decoded
+ *                           by this call: QS_INVALID_ARG.
  *   x (device, d)           updated in place: acc = 0; acc += g_r in increasing r;
  *                           x <- x - acc / R, at every index some masked worker sent.
  *   wire (device), stride_words, worker_mask (host, R bytes or NULL)

@@ -302,6 +302,7 @@ int run_mid(qs_ctx* c, const Active& act, int do_compress, int do_pack, int do_d
             uint32_t* wire, int64_t stride, int64_t* bits_out) {
     const cudaError_t e = launch_mid(c->P, act, do_compress, do_pack, do_decode, 0, do_broadcast, c->aligned ? 1 : 0,
                                      wire, stride, (long long)c->wire_words, (long long*)bits_out, c->mid_grid, c->st);
+    c->P.test_miss_barrier = 0;                    // the test of the bounded wait concerns one launch
     if (e != cudaSuccess) return cuda_fail(c, e, "persistent kernel");
     return after_launch(c, 1, "persistent kernel");
 }
@@ -358,7 +359,7 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     if (!out) return QS_INVALID_ARG;
     *out = nullptr;
     const int sp = op & 15, qz = op >> 4;
-    if (R < 1 || R > MAX_R || d < 1 || d >= (1ll << 32) || k < 1 || k > d || s < 1 || s > 65535) return QS_INVALID_ARG;
+    if (R < 1 || R > MAX_R || d < 1 || d > (1ll << 32) - 4096 || k < 1 || k > d || s < 1 || s > 65535) return QS_INVALID_ARG;   // (32-bit tile arithmetic on the device)
     if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1 && qz != QS_NONE && qz != QS_SIGN_L2)) return QS_INVALID_ARG;
     qs_ctx* c = new qs_ctx();
     std::memset(&c->P, 0, sizeof(Plan));
@@ -391,6 +392,9 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     P.order_sups_max = ORDER_SUPS_MAX;             // QSPARSE_ORDER_EVEN_MAX (0 .. 2048) overrides, for tests of both order stages
     if (const char* e = std::getenv("QSPARSE_ORDER_EVEN_MAX")) P.order_sups_max = (uint32_t)std::min(std::max(std::atoi(e), 0), (int)ORDER_SUPS_MAX);
     P.block_pack = std::getenv("QSPARSE_BLOCK_PACK") != nullptr;   // for tests of both ways of packing in a whole round
+    P.spin_limit = 1u << 22;                       // barrier polls before giving up (about a second)
+    if (const char* e = std::getenv("QSPARSE_SPIN_LIMIT")) P.spin_limit = (uint32_t)std::max(std::atoi(e), 16);
+    P.test_miss_barrier = std::getenv("QSPARSE_TEST_MISS_BARRIER") != nullptr;   // one launch only, see run_mid
     P.seed_lo = (uint32_t)seed; P.seed_hi = (uint32_t)(seed >> 32);
     const int64_t offsets[2] = {0, d};
     const int rc = install_segments(c, 1, offsets, &k);

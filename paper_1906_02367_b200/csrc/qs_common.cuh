@@ -66,6 +66,8 @@ struct Plan {
     uint32_t seed_lo, seed_hi, round_lo, round_hi;
     uint32_t unit_cap;         // a round whose units all have at most this many candidates selects per block (0: never)
     uint32_t order_sups_max;   // (worker, super-block) pairs up to which the order stage deals its work evenly
+    uint32_t spin_limit;       // polls a grid barrier waits before it records QS_TIMEOUT
+    int test_miss_barrier;     // test of that path: block 0 stays away from the launch's first barrier
     int block_pack;            // non-zero: every block packs its share before the closing stage (no packing warps beside it)
     uint64_t cap;
     // tables (device)

@@ -27,7 +27,6 @@ namespace qs {
 
 constexpr int BT = 256;                    // threads per block of the persistent kernel
 constexpr int PER = CHUNK / BT;            // candidates per thread and chunk
-constexpr uint32_t SPIN_LIMIT = 1u << 22;  // barrier polls before giving up (about a second)
 
 struct MidArgs {
     Plan P;
@@ -49,14 +48,16 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
 // bounded: a block that gives up records QS_TIMEOUT and every block leaves the stages at its next
 // barrier.
 __device__ __forceinline__ bool grid_barrier(const Plan& P, uint32_t& target, int* sh_abort) {
+    const bool first = target == 0;
     target += gridDim.x;
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        atomicAdd(P.bar, 1u);
+        // (test of the bounded wait: one block stays away once, the others' waits run out)
+        if (!(P.test_miss_barrier && first && blockIdx.x == 0)) atomicAdd(P.bar, 1u);
         uint32_t spins = 0;
         while (ld_acquire(P.bar) < target) {
-            if (++spins > SPIN_LIMIT) {
+            if (++spins > P.spin_limit) {
                 atomicCAS(P.status, 0, QS_TIMEOUT);
                 *sh_abort = 1;
                 break;

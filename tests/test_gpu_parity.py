@@ -25,15 +25,25 @@ def setup_module(module):
     B = binding
 
 
-@pytest.fixture(autouse=True, params=["per_unit", "per_level"])
+@pytest.fixture(autouse=True, params=["per_unit", "per_level", "uneven_order", "block_pack"])
 def selection_path(request, monkeypatch):
-    # Rounds whose units are all short run the threshold, tie cut and norm of a unit inside one
-    # block; QSPARSE_UNIT_CAP=0 (read by qs_init) sends them through the grid-wide radix levels
-    # that long candidate lists take.  Every case below runs both ways.
+    # The library picks among several ways of doing the same stage by the size of the round; switches
+    # read by qs_init force the ones that small inputs would not reach.  Results never depend on them,
+    # and every case below runs all four ways:
+    #   per_unit      the defaults: short candidate lists are selected from by one block (or warp) each
+    #   per_level     QSPARSE_UNIT_CAP=0: every list goes through the grid-wide radix levels
+    #   uneven_order  QSPARSE_ORDER_EVEN_MAX=0: the order stage that deals candidates by region, which
+    #                 the default only takes for very many (worker, super-block) pairs
+    #   block_pack    QSPARSE_BLOCK_PACK=1: in a whole round every block packs its share of the records
+    #                 before the closing stage instead of packing warps beside it
+    for name in ("QSPARSE_UNIT_CAP", "QSPARSE_ORDER_EVEN_MAX", "QSPARSE_BLOCK_PACK"):
+        monkeypatch.delenv(name, raising=False)
     if request.param == "per_level":
         monkeypatch.setenv("QSPARSE_UNIT_CAP", "0")
-    else:
-        monkeypatch.delenv("QSPARSE_UNIT_CAP", raising=False)
+    elif request.param == "uneven_order":
+        monkeypatch.setenv("QSPARSE_ORDER_EVEN_MAX", "0")
+    elif request.param == "block_pack":
+        monkeypatch.setenv("QSPARSE_BLOCK_PACK", "1")
     yield request.param
 
 
@@ -455,4 +465,60 @@ def test_errors_are_reported_not_thrown_on_the_device():
         B.Context(33, 100, 1, 4)
     with pytest.raises(B.QsError):
         B.Context(2, 100, 101, 4)
+    p.close()
+
+
+def test_resume_from_saved_state_and_round_counter():
+    """The state of a run is (x, xw, mem, round counter, seed): a fresh context fed the saved buffers
+    and qs_set_round continues with identical bytes, and the automatic counter matches explicit rounds."""
+    R, d, k = 4, 50000, 500
+    x, xw, mem = I.gaussian_round(R, d, seed=31)
+    drifts = [I.gaussian_drift(R, d, 12, rnd, std=1e-2) for rnd in range(6)]
+    full = Pair(R, d, k=k, s=16, quantizer=O.QSGD, seed=21, x=x, xw=xw, mem=mem)
+    saved = None
+    for rnd in range(6):
+        if rnd == 3:
+            assert full.ctx.get_round() == 3
+            saved = [t.cpu().numpy().copy() for t in (full.gx, full.gxw, full.gmem)]
+        full.drift(drifts[rnd])
+        out = O.sync_round(full.plan, rnd, full.x, full.xw, full.mem)
+        assert out["rc"] == 0
+        full.ctx.sync_round(full.wire, B.QS_ROUND_AUTO, None, full.gbits)      # the context counts the rounds itself
+        full.check_state(f"automatic round {rnd}")
+        assert np.array_equal(full.wire.cpu().numpy().view(np.uint32), out["wire"])
+    assert full.ctx.get_round() == 6
+    end = [t.cpu().numpy().copy() for t in (full.wire, full.gx, full.gxw, full.gmem)]
+    full.close()
+    again = Pair(R, d, k=k, s=16, quantizer=O.QSGD, seed=21, x=saved[0], xw=saved[1], mem=saved[2])
+    again.ctx.set_round(3)
+    for rnd in range(3, 6):
+        again.gxw += torch.from_numpy(drifts[rnd]).to(again.gxw.device)
+        again.ctx.sync_round(again.wire, B.QS_ROUND_AUTO, None, again.gbits)
+    assert again.ctx.sync_status() == 0, again.ctx.last_error()
+    assert again.ctx.get_round() == 6
+    for a, b in zip(end, (again.wire, again.gx, again.gxw, again.gmem)):
+        assert np.array_equal(a.view(np.uint32), b.cpu().numpy().view(np.uint32))
+    again.close()
+
+
+def test_bounded_wait_runs_out_and_the_context_recovers(monkeypatch):
+    """A grid barrier that does not complete ends the launch with QS_TIMEOUT instead of hanging: in the
+    context's first persistent launch one block stays away from the first barrier (a switch read by
+    qs_init), the other blocks' bounded waits run out, and after qs_sync_status the context runs
+    rounds that match the oracle again."""
+    R, d, k = 3, 40000, 400
+    x, xw, mem = I.gaussian_round(R, d, seed=37)
+    monkeypatch.setenv("QSPARSE_SPIN_LIMIT", "4096")          # a few milliseconds
+    monkeypatch.setenv("QSPARSE_TEST_MISS_BARRIER", "1")
+    p = Pair(R, d, k=k, s=16, quantizer=O.QSGD, seed=8, x=x, xw=xw, mem=mem)
+    monkeypatch.delenv("QSPARSE_TEST_MISS_BARRIER")
+    p.ctx.sync_round(p.wire, 0, None, p.gbits)
+    assert p.ctx.sync_status() == B.QS_TIMEOUT
+    assert p.ctx.sync_status() == 0                           # reported once, then cleared
+    # the interrupted round is void: put the state back and go on
+    for t, a in ((p.gx, x), (p.gxw, xw), (p.gmem, mem)):
+        t.copy_(torch.from_numpy(a))
+    p.round_fused(0)
+    p.drift(I.gaussian_drift(R, d, 5, 1, std=1e-2))
+    p.round_split(1)
     p.close()

@@ -29,7 +29,8 @@ def test_null_and_bad_arguments_are_rejected_on_the_host():
     assert L.qs_init(None, 1, 10, 1, 4, 0, 0, None) == B.QS_INVALID_ARG
     h = C.c_void_p()
     for args in [(0, 10, 1, 4, 0), (33, 10, 1, 4, 0), (2, 0, 1, 4, 0), (2, 10, 11, 4, 0), (2, 10, 0, 4, 0),
-                 (2, 10, 1, 0, 0), (2, 10, 1, 70000, 0), (2, 10, 1, 4, 7), (2, 2**32, 1, 4, 0)]:
+                 (2, 10, 1, 0, 0), (2, 10, 1, 70000, 0), (2, 10, 1, 4, 7), (2, 2**32, 1, 4, 0),
+                 (2, 2**32 - 4095, 1, 4, 0)]:          # d beyond what the 32-bit tile arithmetic of the kernels covers
         R, d, k, s, op = args
         assert L.qs_init(C.byref(h), R, d, k, s, op, 0, None) == B.QS_INVALID_ARG and not h.value
     assert L.qs_wire_words(None) < 0 and L.qs_total_k(None) < 0

@@ -1,17 +1,20 @@
-"""The allocation-free master update (qs_unpack_accumulate_static) against the regular one.
+"""The allocation-free master update (qs_unpack_accumulate_static) against the regular one and the oracle.
 
 Some users of the library may not allocate device memory at the moment the update runs (their
 memory is handed out once by another component, or an allocation would stall the device in the
 middle of a serving loop), so that entry point keeps its scratch in a fixed array inside the
 library.  This file checks, through the C boundary, that it changes x exactly as
-qs_unpack_accumulate does, twice in a row on the same array (the second call meets whatever the
-first one left behind), and that it refuses sizes its array cannot hold.  It is collected last on
+qs_unpack_accumulate and the CPU oracle's master update do, twice in a row on the same array (the
+second call meets whatever the first one left behind), that the call leaves the amount of free
+device memory as it found it, and that it refuses what it cannot take: sizes its array cannot
+hold, and the plain sparsifier (32-bit values in the record), which it does not decode.  It is collected last on
 purpose: a run that stops at the first failure has then already run every other test.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as O
 from paper_1906_02367_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
@@ -40,12 +43,21 @@ def test_static_update_matches_the_regular_one_twice(quantizer, s):
         ctx.compress_feedback(rnd, mask)
         ctx.pack(wire)
         x_static = gx.clone()
+        x_oracle = gx.cpu().numpy().copy()
         ctx.unpack_accumulate(wire, mask)                              # regular entry point
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         rc = B.unpack_accumulate_static(R, d, k, s, quantizer, x_static, wire, mask)
         assert rc == 0
         assert ctx.sync_status() == 0, ctx.last_error()
         torch.cuda.synchronize()
+        if rnd:                                                        # (the first call on a device may load the module)
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call must not allocate device memory"
         assert np.array_equal(_bits(x_static), _bits(gx)), f"call {rnd}"
+        # the oracle's master update on the same records
+        plan = O.Plan(R, d, k=k, s=s, quantizer=quantizer, seed=5)
+        assert O.unpack_accumulate(plan, x_oracle, wire.cpu().numpy().view(np.uint32), mask=mask) == 0
+        assert np.array_equal(_bits(x_static), x_oracle.view(np.uint32)), f"call {rnd} against the oracle"
         assert not np.array_equal(_bits(gx), x.view(np.uint32))        # the update did something
         ctx.broadcast(mask)
     ctx.destroy()
@@ -60,6 +72,7 @@ def test_static_update_rejects_what_it_cannot_hold():
     assert B.unpack_accumulate_static(2, B.QS_STATIC_MAX_D + 1, 4, 16, 0, x, wire) == B.QS_TOO_LARGE
     assert B.unpack_accumulate_static(2, 16, 17, 16, 0, x, wire) == B.QS_INVALID_ARG
     assert B.unpack_accumulate_static(33, 16, 4, 16, 0, x, wire) == B.QS_INVALID_ARG
+    assert B.unpack_accumulate_static(2, 16, 4, 16, B.QS_NONE, x, wire) == B.QS_INVALID_ARG   # values in the record: not decoded here
     small = torch.zeros((2, 3), dtype=torch.int32, device="cuda")
     assert B.unpack_accumulate_static(2, 16, 4, 16, 0, x, small) == B.QS_CAPACITY
     assert B.unpack_accumulate_static(2, 16, 4, 16, 0, x, wire) == 0   # empty records: nothing to add
