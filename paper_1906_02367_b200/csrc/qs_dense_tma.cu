@@ -155,6 +155,17 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
             else bulk_wait_read<0>();
             issue();
         }
+        // Rand_k: the keys do not depend on the data, only on (worker, coordinate): their ten Philox
+        // rounds are worked out before the wait for the item's copies, in its shadow.  (The item's
+        // tile was noted by the producer at least one iteration, and block barrier, ago.)
+        uint4 hq[GP];
+        uint32_t tile_pre = tile;
+        if (RANDK) {
+            if (w == 0) tile_pre = *reinterpret_cast<volatile uint32_t*>(&S.tiles[it & 3u]);
+#pragma unroll
+            for (int k = 0; k < GP; ++k)
+                hq[k] = philox_quad(P, (uint32_t)r, (tile_pre * TILE + (warp * GP + k) * GROUP + lane * 4) >> 2, 1u);
+        }
         bool ok = mbar_wait(&S.full[s], ph);
         if (w == 0 && ok) tile = S.tiles[it & 3u];       // written by the producer before it armed the barrier
         if (!ANCH && w == 0 && tile < ntiles) ok = ok && mbar_wait(&S.xfull[xsl], (uint32_t)((it / XSLOTS) & 1));   // no x tile comes with the end mark
@@ -216,7 +227,7 @@ __global__ void __launch_bounds__(256) pass_a_tma_kernel(const Plan P, const Act
                 if (in) bad |= sk[jj] >= 0xFF000000u;
             }
             if (RANDK) {
-                const uint4 h = philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
+                const uint4 h = tile == tile_pre ? hq[k] : philox_quad(P, (uint32_t)r, e0 >> 2, 1u);
                 sk[0] = ~h.x; sk[1] = ~h.y; sk[2] = ~h.z; sk[3] = ~h.w;
             }
             if (uni[k]) {                    // one threshold for the whole group (the same branch in every lane)

@@ -2129,7 +2129,7 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
     const float rdiv = (float)P.rdiv;
     const uint32_t wp = (uint32_t)(ML_CAP / (L.nact > 0 ? L.nact : 1));   // positions with several senders per window
     const uint32_t J = L.J, my_j = L.my_j, my_r = L.my_r;
-    const uint2* run = P.stage + (size_t)my_r * P.cap + (size_t)tile * STILE;
+    uint2* run = P.stage + (size_t)my_r * P.cap + (size_t)tile * STILE;
     // What will be read from global memory is asked for now, all of it at once (one round trip in
     // place of one per entry): the run itself when it is not in shared memory, and the units of
     // the next few segments when the tile may hold more than one.
@@ -2141,11 +2141,12 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
             asm volatile("prefetch.global.L1 [%0];" ::"l"(&P.units[(size_t)my_r * P.nseg + s0 + j].tau));
     }
     // Entry i of this lane's worker's run: sent?  position in the tile and value.  The first look
-    // at a staged entry leaves the answer in its place.
+    // at an entry leaves the answer in its place (in shared memory, or in the run itself, which
+    // nothing reads after this stage), so that the random draws and the division are made once.
     auto cand = [&](uint32_t i, bool first, uint32_t* pos, float* g) -> bool {
-        uint2* home = &cb[staged ? pbefore + i : 0u];
-        const uint2 ent = staged ? *home : run[i];
-        if (staged && !first) {                       // looked at before: the answer is in place
+        uint2* home = staged ? &cb[pbefore + i] : &run[i];
+        const uint2 ent = *home;
+        if (!first) {                                 // looked at before: the answer is in place
             *pos = ent.x & (uint32_t)(STILE - 1);
             *g = __uint_as_float(ent.y);
             return (ent.x >> 31) != 0u;
@@ -2186,7 +2187,7 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
         *g = gv;
         // the worker's memory at a sent coordinate (quantizers that have no quantize stage of their own)
         if (mem_update && sent && first) P.mem[(size_t)my_r * P.d + idx] = __uint_as_float(ent.y) - gv;
-        if (staged) *home = make_uint2(*pos | (sent ? 0x80000000u : 0u), __float_as_uint(gv));
+        *home = make_uint2(*pos | (sent ? 0x80000000u : 0u), __float_as_uint(gv));
         return sent;
     };
     // senders per coordinate

@@ -41,6 +41,31 @@ def test_single_process_needs_no_group():
     assert bench.workload("per_tensor")[2] == 25557032 and len(bench.workload("per_tensor")[4]) == 161
 
 
+def test_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` with no launcher around it starts two ranks (torch.distributed.run on 127.0.0.1) and
+    reports n_gpus = 2; here through the launch-path self-test, which needs no GPU (gloo, no kernels).  Asked
+    for more GPUs than the machine has, the real run exits non-zero and prints no result line."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    bench_py = os.path.join(ROOT, "bench.py")
+    run = subprocess.run([sys.executable, bench_py, "--gpus", "2", "--selftest-cpu", "--steps", "3", "--warmup", "3"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert run.returncode == 0, run.stderr[-2000:]
+    lines = [l for l in run.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["ms_per_step"] == 2.0  # the slowest rank's (made-up) time
+    if not torch.cuda.is_available():
+        run = subprocess.run([sys.executable, bench_py, "--gpus", "2", "--steps", "3"], capture_output=True, text=True, env=env,
+                             timeout=300)
+        assert run.returncode != 0 and not [l for l in run.stdout.splitlines() if l.startswith("{")]
+    # a launcher that started a different number of ranks than --gpus says is an error, not a line with n_gpus = 1
+    env1 = dict(env, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    run = subprocess.run([sys.executable, bench_py, "--gpus", "2", "--selftest-cpu"], capture_output=True, text=True, env=env1, timeout=300)
+    assert run.returncode != 0 and not run.stdout.strip()
+
+
 # ---------------------------------------------------------------- sharded round (records all-gathered), 2 ranks
 class _OracleEngine:
     """Stands in for the CUDA context on a machine without a GPU: same calls, the oracle's arithmetic."""
