@@ -11,7 +11,7 @@ import numpy as np
 from . import build as _build
 
 TOPK, RANDK = 0, 1
-QSGD, QSGD_SCALED, SIGN_L1, NONE, SIGN_L2 = 0, 1, 2, 3, 4
+QSGD, QSGD_SCALED, SIGN_L1, NONE, SIGN_L2, MINMAX = 0, 1, 2, 3, 4, 5
 SORT, NTH = 0, 1
 
 _lib = None
@@ -27,6 +27,10 @@ def lib():
         _lib.qso_norm_l1.restype = C.c_float
         _lib.qso_qsgd_level.restype = C.c_int
         _lib.qso_qsgd_level.argtypes = [C.c_float, C.c_float, C.c_int, C.c_uint32]
+        _lib.qso_minmax_level.restype = C.c_int
+        _lib.qso_minmax_level.argtypes = [C.c_float, C.c_float, C.c_float, C.c_int, C.c_uint32]
+        _lib.qso_value_minmax.restype = C.c_float
+        _lib.qso_value_minmax.argtypes = [C.c_float, C.c_float, C.c_int, C.c_int]
         _lib.qso_beta_qsgd.restype = C.c_double
         _lib.qso_beta_qsgd.argtypes = [C.c_int64, C.c_int]
         _lib.qso_wire_words.restype = C.c_int64
@@ -80,6 +84,14 @@ def select_randk(seed, rnd, worker, lo, n, k, mode=SORT):
 
 def qsgd_level(u, N, s, w):
     return int(lib().qso_qsgd_level(C.c_float(u), C.c_float(N), s, w))
+
+
+def minmax_level(v, lo, hi, s, w):
+    return int(lib().qso_minmax_level(C.c_float(v), C.c_float(lo), C.c_float(hi), s, w))
+
+
+def value_minmax(lo, hi, s, level):
+    return float(lib().qso_value_minmax(C.c_float(lo), C.c_float(hi), s, level))
 
 
 def beta_qsgd(k, s):

@@ -45,6 +45,19 @@
 //   [sign-l2] quantizer 4 is Lemma 3's operator with m = 2: g = N2/k with N2 the l2 norm of
 //             the kept vector ([norm]); record as for quantizer 2.  m >= 3 is not provided (its
 //             sum of m-th powers has no exact fp64 terms, and gamma_m only shrinks with m).
+//   [min-max] quantizer 5 is the stochastic s-level quantizer of Definition 1's example 2: s levels
+//             between the smallest entry lo and the largest entry hi of the kept vector (signed
+//             values), lo + j D, j = 0 .. s-1, D = (hi - lo)/(s - 1); an entry goes to the level
+//             below or above it, up with probability (v - lo)/D - floor((v - lo)/D) (unbiased,
+//             independently per component; error at most k/(2 (s-1)^2) ||v||^2 in expectation, the
+//             bound of the mean-estimation paper the text cites; the text's d/(2 s^2) counts the
+//             intervals as s).  fp32 recipe: D = (hi - lo)/(s-1); p = (v - lo)/D; l = floor(p);
+//             f = p - l; U as for [qsgd]; j = min(l + (U < f), s - 1); g = lo + j * D (product and
+//             sum rounded on their own); hi == lo: every entry gets j = 0.  Needs s >= 2.  Every
+//             kept entry is sent (j = 0 stands for lo, not for nothing): in the record the count
+//             is implied (n = k), the header pair carries (lo, hi), there is no sign stream and the
+//             level stream holds j; bits = sum_seg 64 + k (b_idx + b_lvl).  Levels are reported
+//             as j + 1 (1 .. s), like QSGD's.
 //   [pieces]  Corollary 1: each segment has its own k, norm, beta.
 //   [momentum] Section 5.1 applies momentum 0.9 on the local iterations and prints no
 //             formula: the heavy-ball form v <- mu v + grad, xhat <- xhat - eta v is taken,
@@ -83,7 +96,7 @@
 namespace {
 
 enum { SP_TOPK = 0, SP_RANDK = 1 };
-enum { QZ_QSGD = 0, QZ_QSGD_SCALED = 1, QZ_SIGN_L1 = 2, QZ_NONE = 3, QZ_SIGN_L2 = 4 };
+enum { QZ_QSGD = 0, QZ_QSGD_SCALED = 1, QZ_SIGN_L1 = 2, QZ_NONE = 3, QZ_SIGN_L2 = 4, QZ_MINMAX = 5 };
 inline bool is_sign(int quantizer) { return quantizer == QZ_SIGN_L1 || quantizer == QZ_SIGN_L2; }
 enum { ERR_OK = 0, ERR_ARG = -1, ERR_CAPACITY = -4, ERR_NONFINITE = -5 };
 
@@ -263,6 +276,31 @@ float value_qsgd(float N, int level, int s, int scaled, float c, int negative) {
     return negative ? -g : g;
 }
 
+// Stochastic s-level quantizer between the smallest and the largest entry of the kept vector
+// (Section 2.1, Definition 1, example 2): s levels lo, lo + D, .., lo + (s-1) D with D = (hi - lo) /
+// (s - 1); an entry between two levels goes to the upper one with the probability that makes the
+// result unbiased.  Levels are numbered 1 .. s here (level l stands for lo + (l - 1) D), so that
+// the record's level field holds l - 1 as for QSGD.  fp32, every operation rounded on its own; the
+// uniform draw is the top 24 bits of the Philox word, as for QSGD.  hi == lo: one level.
+int minmax_level(float v, float lo, float hi, int s, uint32_t w) {
+    float D = (hi - lo) / (float)(s - 1);
+    if (!(D > 0.0f)) return 1;
+    float p = (v - lo) / D;
+    float l = std::floor(p);
+    float f = p - l;
+    float U = (float)(w >> 8) * 5.9604644775390625e-08f;  // 2^-24
+    int j = (int)l + (U < f ? 1 : 0);
+    if (j < 0) j = 0;
+    if (j > s - 1) j = s - 1;
+    return j + 1;
+}
+
+float value_minmax(float lo, float hi, int s, int level) {
+    float D = (hi - lo) / (float)(s - 1);
+    float step = (float)(level - 1) * D;
+    return lo + step;
+}
+
 float value_sign(float N1, int64_t k, int negative) {
     float g = N1 / (float)k;
     return negative ? -g : g;
@@ -292,10 +330,12 @@ uint32_t get_bits(const uint32_t* w, int64_t bitpos, int width) {
 // words of the streams of a segment that sends n entries, and bits per entry
 int64_t payload_words(int64_t n, int bi, int bl, int quantizer) {
     if (quantizer == QZ_NONE) return words_for(n, bi) + n;                 // indices, then 32-bit values
+    if (quantizer == QZ_MINMAX) return words_for(n, bi) + words_for(n, bl); // indices, then levels (no signs)
     return words_for(n, bi) + words_for(n, 1) + (!is_sign(quantizer) ? words_for(n, bl) : 0);
 }
 int entry_bits(int bi, int bl, int quantizer) {
     if (quantizer == QZ_NONE) return bi + 32;
+    if (quantizer == QZ_MINMAX) return bi + bl;
     return bi + 1 + (!is_sign(quantizer) ? bl : 0);
 }
 
@@ -327,6 +367,7 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
     }
     const int has_levels = P.quantizer == QZ_QSGD || P.quantizer == QZ_QSGD_SCALED;
     const int plain = P.quantizer == QZ_NONE;   // sparsifier alone: the kept values travel as they are
+    const int minmax = P.quantizer == QZ_MINMAX;
     const int bl = bits_lvl(P.s);
     int64_t payload = 2 * (int64_t)P.nseg;  // word offset of the next segment's streams
     int64_t bits = 0, selpos = 0;
@@ -338,7 +379,9 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
         else select_randk(P.seed, round, (uint32_t)r, lo, n_el, k, mode, idx.data());
         std::vector<float> kept(k);
         for (int64_t j = 0; j < k; ++j) kept[j] = u[lo + idx[j]];
-        const float N = plain ? 0.0f
+        float vlo = kept[0], vhi = kept[0];     // smallest and largest kept entry (min/max quantizer)
+        for (int64_t j = 1; j < k; ++j) { if (kept[j] < vlo) vlo = kept[j]; if (kept[j] > vhi) vhi = kept[j]; }
+        const float N = (plain || minmax) ? 0.0f
                       : (has_levels || P.quantizer == QZ_SIGN_L2) ? norm_l2_exact(kept.data(), k) : norm_l1_exact(kept.data(), k);
         const float c = (float)(1.0 / (1.0 + beta_qsgd(k, P.s)));
         std::vector<int64_t> s_idx; std::vector<int> s_lvl, s_neg; std::vector<float> s_val;
@@ -354,6 +397,9 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
             } else if (plain) {
                 level = 1;
                 gval = v;
+            } else if (minmax) {
+                level = minmax_level(v, vlo, vhi, P.s, philox_word(P.seed, round, (uint32_t)r, (uint64_t)gi, 0u));
+                gval = value_minmax(vlo, vhi, P.s, level);
             } else {
                 level = 1;
                 gval = value_sign(N, k, neg);
@@ -376,6 +422,10 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
         uint32_t nb; std::memcpy(&nb, &N, 4);
         wire[2 * g] = (uint32_t)n;
         wire[2 * g + 1] = nb;
+        if (minmax) {   // every kept entry is sent, so the count is implied (n = k): the pair carries (min, max)
+            std::memcpy(&wire[2 * g], &vlo, 4);
+            std::memcpy(&wire[2 * g + 1], &vhi, 4);
+        }
         uint32_t* w_idx = wire + payload;
         uint32_t* w_sgn = w_idx + words_for(n, bi);
         uint32_t* w_lvl = w_sgn + words_for(n, 1);
@@ -383,6 +433,8 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
             put_bits(w_idx, j * bi, bi, (uint32_t)s_idx[j]);
             if (plain) {
                 std::memcpy(&w_sgn[j], &s_val[j], 4);          // the value stream follows the indices
+            } else if (minmax) {
+                put_bits(w_sgn, j * bl, bl, (uint32_t)(s_lvl[j] - 1));   // the level stream follows the indices
             } else {
                 put_bits(w_sgn, j, 1, (uint32_t)s_neg[j]);
                 if (has_levels) put_bits(w_lvl, j * bl, bl, (uint32_t)(s_lvl[j] - 1));
@@ -390,7 +442,7 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
         }
         payload += payload_words(n, bi, bl, P.quantizer);
         bits += 64 + n * entry_bits(bi, bl, P.quantizer);
-        if (norm_out) norm_out[g] = N;
+        if (norm_out) norm_out[g] = minmax ? vhi : N;
         if (n_out) n_out[g] = n;
     }
     if (bits_out) *bits_out = bits;
@@ -402,12 +454,14 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
 void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
     const int has_levels = P.quantizer == QZ_QSGD || P.quantizer == QZ_QSGD_SCALED;
     const int plain = P.quantizer == QZ_NONE;
+    const int minmax = P.quantizer == QZ_MINMAX;
     const int bl = bits_lvl(P.s);
     int64_t payload = 2 * (int64_t)P.nseg;
     for (int g = 0; g < P.nseg; ++g) {
         const int64_t lo = P.off[g], n_el = P.off[g + 1] - lo, k = P.kseg[g];
-        const int64_t n = wire[2 * g];
+        const int64_t n = minmax ? k : wire[2 * g];
         float N; std::memcpy(&N, &wire[2 * g + 1], 4);
+        float vlo; std::memcpy(&vlo, &wire[2 * g], 4);    // (min, max) in the header pair of the min/max quantizer
         const int bi = bits_idx(n_el);
         const float c = (float)(1.0 / (1.0 + beta_qsgd(k, P.s)));
         const uint32_t* w_idx = wire + payload;
@@ -415,10 +469,12 @@ void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
         const uint32_t* w_lvl = w_sgn + words_for(n, 1);
         for (int64_t j = 0; j < n; ++j) {
             const int64_t i = lo + (int64_t)get_bits(w_idx, j * bi, bi);
-            const int neg = plain ? 0 : (int)get_bits(w_sgn, j, 1);
+            const int neg = (plain || minmax) ? 0 : (int)get_bits(w_sgn, j, 1);
             float gval;
             if (plain) {
                 std::memcpy(&gval, &w_sgn[j], 4);
+            } else if (minmax) {
+                gval = value_minmax(vlo, N, P.s, (int)get_bits(w_sgn, j * bl, bl) + 1);
             } else if (has_levels) {
                 const int level = (int)get_bits(w_lvl, j * bl, bl) + 1;
                 gval = value_qsgd(N, level, P.s, P.quantizer == QZ_QSGD_SCALED, c, neg);
@@ -433,6 +489,7 @@ void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
 
 bool valid_plan(const Plan& P) {
     if (P.R < 1 || P.d < 1 || P.nseg < 1 || P.s < 1 || P.s > 65535) return false;
+    if (P.quantizer == QZ_MINMAX && P.s < 2) return false;
     if (P.off[0] != 0 || P.off[P.nseg] != P.d) return false;
     for (int g = 0; g < P.nseg; ++g) {
         int64_t n = P.off[g + 1] - P.off[g];
@@ -462,6 +519,8 @@ void qso_select_randk(uint64_t seed, uint64_t round, uint32_t worker, int64_t lo
     select_randk(seed, round, worker, lo, n, k, mode, idx_out);
 }
 int qso_qsgd_level(float u, float N, int s, uint32_t w) { return qsgd_level(u, N, s, w); }
+int qso_minmax_level(float v, float lo, float hi, int s, uint32_t w) { return minmax_level(v, lo, hi, s, w); }
+float qso_value_minmax(float lo, float hi, int s, int level) { return value_minmax(lo, hi, s, level); }
 double qso_beta_qsgd(int64_t k, int s) { return beta_qsgd(k, s); }
 
 int64_t qso_wire_words(int R, int64_t d, int nseg, const int64_t* off, const int64_t* kseg, int s,
