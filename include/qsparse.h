@@ -78,6 +78,16 @@ enum {
 /* Sign scaled by the l2 norm over k (Lemma 3 with m = 2; gamma_2 = 1/d): g = +-N2/k with N2 the
  * exactly summed l2 norm of the kept vector; record as for QS_SIGN_L1.  m >= 3 is not provided. */
 #define QS_SIGN_L2 4
+/* Stochastic s-level quantizer between the smallest entry lo and the largest entry hi of the kept
+ * vector (Definition 1, example 2): levels lo + j D, j = 0 .. s-1, D = (hi - lo)/(s - 1); an entry
+ * goes to the level below or above it, up with probability (v - lo)/D - floor((v - lo)/D)
+ * (unbiased).  fp32: p = (v - lo)/D; j = min(floor(p) + (U < p - floor(p)), s - 1) with U the top
+ * 24 bits of the Philox word of stream 0; g = lo + j * D (product and sum rounded on their own);
+ * hi == lo gives j = 0.  Needs s >= 2.  Every kept entry is sent: in the record the count is
+ * implied (n = k_seg), the segment's header pair carries (lo, hi), there is no sign stream and
+ * the level stream holds j; bits = 64 + k (b_idx + b_lvl) per segment.  qs_export_selection
+ * reports the levels as j + 1 and hi as the norm. */
+#define QS_MINMAX 5
 /* op argument of qs_init */
 #define QS_OP(sparsifier, quantizer) ((sparsifier) | ((quantizer) << 4))
 

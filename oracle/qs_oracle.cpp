@@ -407,7 +407,7 @@ int worker_compress(const Plan& P, uint64_t round, int r, const float* anchor, c
             mem[gi] = v - gval;
             if (sel_out) sel_out[selpos + j] = gi;
             if (lvl_out) lvl_out[selpos + j] = level;
-            if (sgn_out) sgn_out[selpos + j] = (uint8_t)neg;
+            if (sgn_out) sgn_out[selpos + j] = (uint8_t)(minmax ? 0 : neg);   // (no sign travels with the min/max quantizer)
             if (level != 0) { s_idx.push_back(idx[j]); s_lvl.push_back(level); s_neg.push_back(neg); s_val.push_back(v); }
         }
         // coordinates outside the kept set: C(u) = 0 there, so m <- u

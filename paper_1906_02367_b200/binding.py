@@ -17,7 +17,7 @@ QS_INVALID_ARG, QS_ALLOC, QS_CUDA, QS_CAPACITY, QS_NONFINITE, QS_STATE, QS_TIMEO
 QS_TOO_LARGE = -8
 QS_STATIC_MAX_D = 1 << 20
 QS_TOPK, QS_RANDK = 0, 1
-QS_QSGD, QS_QSGD_SCALED, QS_SIGN_L1, QS_NONE, QS_SIGN_L2 = 0, 1, 2, 3, 4
+QS_QSGD, QS_QSGD_SCALED, QS_SIGN_L1, QS_NONE, QS_SIGN_L2, QS_MINMAX = 0, 1, 2, 3, 4, 5
 QS_ROUND_AUTO = 2**64 - 1
 
 EXPORTS = [

@@ -193,7 +193,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
         h_c[g] = (float)(1.0 / (1.0 + (a < b ? a : b)));
         h_bi[g] = (uint8_t)std::max(1, ceil_log2(n));
         // quantizers that send every kept entry: the streams' places and the bit count never change
-        if (qz_is_sign(P.qz) || P.qz == QS_NONE)
+        if (qz_sends_all(P.qz))
             for (int r = 0; r < R; ++r) {
                 h_pay[(size_t)r * nseg + g] = (uint32_t)words;
                 h_bits[r] += 64 + (long long)k * entry_bits(h_bi[g], (uint32_t)P.bl, P.qz);
@@ -360,7 +360,8 @@ int qs_init(qs_ctx** out, int R, int64_t d, int64_t k, int s, int op, uint64_t s
     *out = nullptr;
     const int sp = op & 15, qz = op >> 4;
     if (R < 1 || R > MAX_R || d < 1 || d > (1ll << 32) - 4096 || k < 1 || k > d || s < 1 || s > 65535) return QS_INVALID_ARG;   // (32-bit tile arithmetic on the device)
-    if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1 && qz != QS_NONE && qz != QS_SIGN_L2)) return QS_INVALID_ARG;
+    if ((sp != QS_TOPK && sp != QS_RANDK) || (qz != QS_QSGD && qz != QS_QSGD_SCALED && qz != QS_SIGN_L1 && qz != QS_NONE && qz != QS_SIGN_L2 && qz != QS_MINMAX)) return QS_INVALID_ARG;
+    if (qz == QS_MINMAX && s < 2) return QS_INVALID_ARG;      // two levels at least: the smallest and the largest entry
     qs_ctx* c = new qs_ctx();
     std::memset(&c->P, 0, sizeof(Plan));
     c->st = static_cast<cudaStream_t>(cuda_stream);

@@ -238,6 +238,10 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* sh, ui
 __device__ __forceinline__ void set_status(const Plan& P, int code) { atomicCAS(P.status, 0, code); }
 
 __host__ __device__ __forceinline__ bool qz_is_sign(int qz) { return qz == QS_SIGN_L1 || qz == QS_SIGN_L2; }
+// quantizers that send every kept entry: the streams' places and the bit count never change
+__host__ __device__ __forceinline__ bool qz_sends_all(int qz) { return qz_is_sign(qz) || qz == QS_NONE || qz == QS_MINMAX; }
+// quantizers whose record has a level stream
+__host__ __device__ __forceinline__ bool qz_has_levels(int qz) { return qz == QS_QSGD || qz == QS_QSGD_SCALED || qz == QS_MINMAX; }
 
 __host__ __device__ __forceinline__ uint32_t words_for(uint32_t nfields, uint32_t width) {
     return (uint32_t)(((uint64_t)nfields * width + 31u) >> 5);
@@ -246,10 +250,12 @@ __host__ __device__ __forceinline__ uint32_t words_for(uint32_t nfields, uint32_
 // words of the streams of a segment that sends n entries, and bits per entry
 __host__ __device__ __forceinline__ uint32_t streams_words(uint32_t n, uint32_t bi, uint32_t bl, int qz) {
     if (qz == QS_NONE) return words_for(n, bi) + n;                     // indices, then 32-bit values
+    if (qz == QS_MINMAX) return words_for(n, bi) + words_for(n, bl);    // indices, then levels (no signs)
     return words_for(n, bi) + words_for(n, 1) + (!qz_is_sign(qz) ? words_for(n, bl) : 0u);
 }
 __host__ __device__ __forceinline__ uint32_t entry_bits(uint32_t bi, uint32_t bl, int qz) {
     if (qz == QS_NONE) return bi + 32u;
+    if (qz == QS_MINMAX) return bi + bl;
     return bi + 1u + (!qz_is_sign(qz) ? bl : 0u);
 }
 
@@ -263,6 +269,34 @@ __device__ __forceinline__ int qsgd_level(float u, float N, int s, uint32_t w) {
     const float U = (float)(w >> 8) * 5.9604644775390625e-08f;
     const int level = (int)l + (U < f ? 1 : 0);
     return level < s ? level : s;
+}
+
+// The min/max quantizer: smallest and largest kept value travel as ordered 32-bit keys (larger
+// float = larger key), which atomicMin / atomicMax can work on.
+__device__ __forceinline__ uint32_t float_order(float v) {
+    const uint32_t b = __float_as_uint(v);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float order_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+// level 1 .. s of the min/max quantizer (level l stands for lo + (l - 1) D) and the value
+__device__ __forceinline__ int minmax_level(float v, float lo, float hi, int s, uint32_t w) {
+    const float D = (hi - lo) / (float)(s - 1);
+    if (!(D > 0.0f)) return 1;
+    const float p = (v - lo) / D;
+    const float l = floorf(p);
+    const float f = p - l;
+    const float U = (float)(w >> 8) * 5.9604644775390625e-08f;
+    int j = (int)l + (U < f ? 1 : 0);
+    j = j < 0 ? 0 : j;
+    j = j > s - 1 ? s - 1 : j;
+    return j + 1;
+}
+__device__ __forceinline__ float minmax_value(float lo, float hi, int s, int level) {
+    const float D = (hi - lo) / (float)(s - 1);
+    const float step = (float)(level - 1) * D;
+    return lo + step;
 }
 
 __device__ __forceinline__ float coord_value(const Plan& P, float N, int level, bool neg, float c,

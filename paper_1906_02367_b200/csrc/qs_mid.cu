@@ -426,7 +426,7 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
     tab->start = t_start; tab->c = t_c; tab->cb = t_cb; tab->lb = t_lb; tab->total_chunks = carry;
     const uint32_t longest = sh_flag[1];
     // the streams' places: one segment, or a quantizer that sends every kept entry (fixed places)
-    tab->fast = (P.nseg == 1 || qz_early(P.qz)) && (longest + CHUNK - 1) / CHUNK <= 1024u;
+    tab->fast = (P.nseg == 1 || qz_sends_all(P.qz)) && (longest + CHUNK - 1) / CHUNK <= 1024u;
     // Which units one block selects from on its own (block barriers only), and which take the
     // grid-wide radix levels: every list up to the cap when there is a block for each list that
     // would keep one busy for a while (lists are dealt largest first); otherwise only the lists of
@@ -797,7 +797,7 @@ __device__ void final_unit(const Plan& P, const Tab& tab, uint32_t u, uint32_t* 
             out.tie_max = tie_max;
             out.tie_t = tie_t;
             out.n = 0;
-            out.emin = 255u;
+            out.emin = P.qz == QS_MINMAX ? 0xffffffffu : 255u;    // (min/max quantizer: ordered keys of the smallest and largest kept value)
             out.emax = 0u;
             out.norm = 0.0f;
             out.done = 0;
@@ -974,6 +974,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_long;
     const bool plain = P.qz == QS_NONE;            // the plain sparsifier sends the values: no norm
+    const bool mm = P.qz == QS_MINMAX;             // smallest and largest kept value in place of a norm
     // merge: a whole round with a quantizer that sends every kept entry at level 1; the counts and
     // the sender bits are known here, and the pack stage does the rest of the quantize stage's work
     const bool early = merge;
@@ -1041,6 +1042,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
             key[i] = RANDK ? (in ? P.cand_key[c.base + off] : 0u) : topk_key(val[i]);
         }
         uint32_t nkept = 0;                          // lane 0 of each warp counts
+        uint32_t mm_lo = 0xffffffffu, mm_hi = 0u;
         bool kept[PER];
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
@@ -1052,7 +1054,11 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
         for (int i = 0; i < PER; ++i) {
             const uint32_t live = __ballot_sync(0xffffffffu, kept[i]);
             if (early && lane == 0) nkept += __popc(live);
-            if (kept[i] && !plain) {
+            if (kept[i] && mm) {
+                const uint32_t ok = float_order(val[i]);
+                mm_lo = ok < mm_lo ? ok : mm_lo;
+                mm_hi = ok > mm_hi ? ok : mm_hi;
+            } else if (kept[i] && !plain) {
                 const uint32_t b = __float_as_uint(val[i]);
                 const uint32_t e = (b >> 23) & 255u;
                 const uint32_t m = e ? ((b & 0x7fffffu) | 0x800000u) : (b & 0x7fffffu);
@@ -1071,7 +1077,13 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
                 P.chunk_cnt[c.chunk] = t | (t << 16);    // kept | sent << 16
             }
         }
-        if (!plain) ++pending;
+        if (mm) {
+            mm_lo = __reduce_min_sync(0xffffffffu, mm_lo);
+            mm_hi = __reduce_max_sync(0xffffffffu, mm_hi);
+            if (lane == 0 && mm_lo <= mm_hi) { atomicMin(&P.units[c.u].emin, mm_lo); atomicMax(&P.units[c.u].emax, mm_hi); }
+        } else if (!plain) {
+            ++pending;
+        }
     }
     if (pending) flush();
 }
@@ -1216,7 +1228,7 @@ __device__ __forceinline__ void unit_rows(const Plan& P, size_t base, uint32_t c
             for (int j = 0; j < NB; ++j) {
                 const uint32_t off = (uint32_t)((b * NB + j) * BT) + threadIdx.x;
                 ix[j] = (AUX && off < c) ? P.cand_idx[base + off] : 0u;
-                vq[j] = (AUX && RANDK && off < c) ? __float_as_uint(P.cand_val[base + off]) : 0u;
+                vq[j] = (AUX && (RANDK || P.qz == QS_MINMAX) && off < c) ? __float_as_uint(P.cand_val[base + off]) : 0u;
             }
 #pragma unroll
             for (int j = 0; j < NB; ++j) {
@@ -1247,7 +1259,8 @@ template <bool RANDK>
 __device__ void unit_by_warp(const Plan& P, const Tab& tab, uint32_t u, uint32_t r, uint32_t seg, bool early, int lane) {
     const uint32_t c = tab.c[u], k = P.kseg[seg];
     const size_t base = (size_t)r * P.cap + tab.start[u];
-    const bool plain = P.qz == QS_NONE, l1 = P.qz == QS_SIGN_L1;
+    const bool mm = P.qz == QS_MINMAX;
+    const bool plain = P.qz == QS_NONE || mm, l1 = P.qz == QS_SIGN_L1;   // (no norm for the plain sparsifier and the min/max quantizer)
     uint32_t key[2], idx[2], vb[2];
     bool in[2];
 #pragma unroll
@@ -1256,7 +1269,7 @@ __device__ void unit_by_warp(const Plan& P, const Tab& tab, uint32_t u, uint32_t
         in[q] = j < c;
         key[q] = in[q] ? sort_key<RANDK>(P, base + j) : 0u;
         idx[q] = in[q] ? P.cand_idx[base + j] : 0u;
-        vb[q] = (RANDK && in[q]) ? __float_as_uint(P.cand_val[base + j]) : (key[q] >> 1);
+        vb[q] = ((RANDK || mm) && in[q]) ? __float_as_uint(P.cand_val[base + j]) : (key[q] >> 1);
     }
     // rank of each candidate: those before it have a larger key, or an equal one earlier in the list
     uint32_t rank[2] = {0u, 0u};
@@ -1335,14 +1348,27 @@ __device__ void unit_by_warp(const Plan& P, const Tab& tab, uint32_t u, uint32_t
     // the level-0 counts of the order stage are not needed on this path: leave them zero
 #pragma unroll
     for (int i = 0; i < 8; ++i) P.hist[(size_t)u * 256 + (uint32_t)lane + 32u * i] = 0u;
+    // min/max quantizer: ordered keys of the smallest and largest kept value
+    uint32_t mm_lo = 0xffffffffu, mm_hi = 0u;
+    if (mm) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+            if (kept[q]) {
+                const uint32_t ok = float_order(__uint_as_float(vb[q]));
+                mm_lo = ok < mm_lo ? ok : mm_lo;
+                mm_hi = ok > mm_hi ? ok : mm_hi;
+            }
+        mm_lo = __reduce_min_sync(0xffffffffu, mm_lo);
+        mm_hi = __reduce_max_sync(0xffffffffu, mm_hi);
+    }
     if (lane == 0) {
         Unit& out = P.units[u];
         out.tau = tau;
         out.tie_max = tie_max;
         out.tie_t = 0;
         out.n = 0;
-        out.emin = 255u;
-        out.emax = 0u;
+        out.emin = mm ? mm_lo : 255u;
+        out.emax = mm ? mm_hi : 0u;
         out.norm = norm;
         if (!RANDK) predict_floor(P, r, seg, tau, c, k);
     }
@@ -1352,7 +1378,8 @@ template <bool RANDK>
 __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, bool early, UnitSh& S, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t items = (uint32_t)P.nseg * (uint32_t)act.n;
-    const bool plain = P.qz == QS_NONE, l1 = P.qz == QS_SIGN_L1;
+    const bool mm = P.qz == QS_MINMAX;
+    const bool plain = P.qz == QS_NONE || mm, l1 = P.qz == QS_SIGN_L1;   // (no norm for the plain sparsifier and the min/max quantizer)
     const uint32_t lt = (1u << lane) - 1u;
     // the shortest lists first, a warp each: eight consecutive units of the list to a block
     for (uint32_t item = blockIdx.x * (BT / 32) + wid; item < items; item += gridDim.x * (BT / 32)) {
@@ -1384,7 +1411,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
         }
         *reinterpret_cast<uint4*>(S.acc[threadIdx.x]) = make_uint4(0u, 0u, 0u, 0u);
         if (threadIdx.x < 16) S.kept[threadIdx.x] = 0u;
-        if (threadIdx.x == 0) { S.ctl[4] = 0xffffffffu; S.ctl[5] = 0u; }
+        if (threadIdx.x == 0) { S.ctl[4] = 0xffffffffu; S.ctl[5] = 0u; S.ctl[6] = 0xffffffffu; S.ctl[7] = 0u; }   // (6, 7: smallest / largest kept value)
         uint32_t tau, tie_max;
         if (c <= (uint32_t)BT) {
             // ranks by direct counting: candidate j comes before this one if its key is larger, or
@@ -1455,6 +1482,12 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             const uint32_t live = __ballot_sync(0xffffffffu, kept);
             if (early && lane == 0 && live) atomicAdd(&S.kept[i / PER], __popc(live));
             if (early && kept) mem_ahead(P, r, idx);
+            if (mm) {                                // ordered keys of the smallest and largest kept value
+                const uint32_t ok = float_order(__uint_as_float(vb));
+                const uint32_t w_lo = __reduce_min_sync(0xffffffffu, kept ? ok : 0xffffffffu);
+                const uint32_t w_hi = __reduce_max_sync(0xffffffffu, kept ? ok : 0u);
+                if (lane == 0 && live) { atomicMin(&S.ctl[6], w_lo); atomicMax(&S.ctl[7], w_hi); }
+            }
             if (kept && !plain) {
                 const uint32_t b = RANDK ? vb : (kv >> 1);
                 const uint32_t e = (b >> 23) & 255u;
@@ -1467,8 +1500,9 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             return 0u;
         };
         auto none = [](uint32_t, uint32_t) {};
-        // the indices are needed for a tie cut and for the request above; Rand_k reads the values too
-        if (early || ties || RANDK) unit_rows<RANDK, 8, true>(P, base, c, key, take, none);
+        // the indices are needed for a tie cut and for the request above; Rand_k and the min/max
+        // quantizer read the values too
+        if (early || ties || RANDK || mm) unit_rows<RANDK, 8, true>(P, base, c, key, take, none);
         else unit_rows<RANDK, 8, false>(P, base, c, key, take, none);
         __syncthreads();
         if (wid == 0) {
@@ -1488,8 +1522,8 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
                 out.tie_max = tie_max;
                 out.tie_t = 0;
                 out.n = 0;
-                out.emin = 255u;
-                out.emax = 0u;
+                out.emin = mm ? S.ctl[6] : 255u;
+                out.emax = mm ? S.ctl[7] : 0u;
                 auto sums = [&](uint32_t e, unsigned long long* a0, unsigned long long* a1) {
                     *a0 = ((unsigned long long)S.acc[e][1] << 16) + S.acc[e][0];
                     *a1 = ((unsigned long long)S.acc[e][3] << 16) + S.acc[e][2];
@@ -1512,7 +1546,7 @@ template <bool RANDK>
 __device__ void stage_quant(const Plan& P, const Tab& tab, uint32_t* sh_u, uint32_t* sh_w) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t total = tab.total_chunks;
-    const bool sign_op = qz_is_sign(P.qz), plain = P.qz == QS_NONE;
+    const bool sign_op = qz_is_sign(P.qz), plain = P.qz == QS_NONE, mm = P.qz == QS_MINMAX;
     ChunkCtx c;
     const uint32_t share = (total + gridDim.x - 1) / gridDim.x;      // consecutive chunks: mostly one unit
     const uint32_t c_lo = blockIdx.x * share, c_hi = c_lo + share < total ? c_lo + share : total;
@@ -1538,13 +1572,21 @@ __device__ void stage_quant(const Plan& P, const Tab& tab, uint32_t* sh_u, uint3
             if (off >= c.c) continue;
             uint32_t q = 0;
             if (is_kept<RANDK>(c.un, key[i], idx[i])) {
-                const bool neg = val[i] < 0.0f;
+                const bool neg = !mm && val[i] < 0.0f;       // (the min/max quantizer has no sign stream)
                 int level = 1;
-                if (!sign_op && !plain) level = qsgd_level(val[i], N, P.s, philox_word(P, c.r, idx[i], 0u));
+                float g;
+                if (mm) {
+                    const float lo = order_float(c.un.emin), hi = order_float(c.un.emax);
+                    level = minmax_level(val[i], lo, hi, P.s, philox_word(P, c.r, idx[i], 0u));
+                    g = minmax_value(lo, hi, P.s, level);
+                } else {
+                    if (!sign_op && !plain) level = qsgd_level(val[i], N, P.s, philox_word(P, c.r, idx[i], 0u));
+                    g = plain ? val[i] : coord_value(P, N, level, neg, cs, k);
+                }
                 q = Q_SEL | (neg ? Q_NEG : 0u) | (uint32_t)level;
                 cnt += 1u;
                 if (level) {
-                    mem[idx[i]] = val[i] - (plain ? val[i] : coord_value(P, N, level, neg, cs, k));
+                    mem[idx[i]] = val[i] - g;
                     cnt += 1u << 16;
                 }
             }
@@ -1653,8 +1695,9 @@ __device__ void stage_pack_dir(const Plan& P, const Active& act, uint32_t* wire,
         const uint32_t g = i % P.nseg;
         const Unit& un = P.units[(size_t)r * P.nseg + g];
         uint32_t* row = wire + (size_t)r * stride;
-        row[2 * g] = un.n;
-        row[2 * g + 1] = __float_as_uint(un.norm);
+        const bool mm = P.qz == QS_MINMAX;           // (the pair carries (min, max), n = k)
+        row[2 * g] = mm ? __float_as_uint(order_float(un.emin)) : un.n;
+        row[2 * g + 1] = __float_as_uint(mm ? order_float(un.emax) : un.norm);
         if (g == 0 && bits_out) bits_out[r] = P.bits[r];
     }
 }
@@ -1684,7 +1727,7 @@ __device__ __forceinline__ void block_sum4(uint32_t v[4], uint32_t* sh) {
 template <bool RANDK>
 __device__ void pack_chunk(const Plan& P, const Tab& tab, uint32_t chunk, ChunkCtx& c, bool merge, uint32_t* wire,
                            long long stride, long long* bits_out, uint32_t* sh_u, uint32_t* sh) {
-    const bool plain = P.qz == QS_NONE, has_lvl = !qz_is_sign(P.qz) && !plain;
+    const bool plain = P.qz == QS_NONE, has_lvl = qz_has_levels(P.qz), mm = P.qz == QS_MINMAX;
     c = chunk_context(P, tab, chunk, sh_u, &c);
     // this thread's candidates first: their reads overlap the sums below
     uint32_t q[PER], e[PER];
@@ -1723,8 +1766,8 @@ __device__ void pack_chunk(const Plan& P, const Tab& tab, uint32_t chunk, ChunkC
             P.units[c.u].n = unit_n;
             if (sums[2] != P.kseg[c.seg]) set_status(P, QS_STATE);
             uint32_t* row = wire + (size_t)c.r * stride;
-            row[2 * c.seg] = unit_n;
-            row[2 * c.seg + 1] = __float_as_uint(c.un.norm);
+            row[2 * c.seg] = mm ? __float_as_uint(order_float(c.un.emin)) : unit_n;      // (min/max: the pair carries (min, max), n = k)
+            row[2 * c.seg + 1] = __float_as_uint(mm ? order_float(c.un.emax) : c.un.norm);
             if (P.nseg == 1) {
                 const long long bits = 64 + (long long)unit_n * entry_bits(bi, (uint32_t)P.bl, P.qz);
                 P.bits[c.r] = bits;
@@ -1741,7 +1784,7 @@ __device__ void pack_chunk(const Plan& P, const Tab& tab, uint32_t chunk, ChunkC
     }
     uint32_t* w_idx = wire + (size_t)c.r * stride + pay;
     uint32_t* w_sgn = w_idx + words_for(unit_n, bi);
-    uint32_t* w_lvl = w_sgn + words_for(unit_n, 1);
+    uint32_t* w_lvl = mm ? w_sgn : w_sgn + words_for(unit_n, 1);          // (no sign stream in front of the min/max levels)
     uint32_t* o_idx = P.sel_idx + (size_t)c.r * P.K + P.kprefix[c.seg];
     uint32_t* o_q = P.sel_q + (size_t)c.r * P.K + P.kprefix[c.seg];
     uint32_t mine = 0;                            // kept | sent << 16 among this thread's candidates
@@ -1889,7 +1932,7 @@ __device__ void stage_dec_prep(const Plan& P, const Active& act, const uint32_t*
             const uint32_t g = base + threadIdx.x;
             uint32_t n = 0, words = 0;
             if (g < (uint32_t)P.nseg) {
-                n = row[2 * g];
+                n = P.qz == QS_MINMAX ? P.kseg[g] : row[2 * g];                  // (min/max: every kept entry is sent)
                 if (n > P.kseg[g]) { n = 0; set_status(P, QS_INVALID_ARG); }     // not a record of this plan
                 words = streams_words(n, P.bidx[g], (uint32_t)P.bl, P.qz);
             }
@@ -1912,7 +1955,7 @@ struct Entry { uint32_t seg, j, n, coord; const uint32_t* w_idx; };
 __device__ __forceinline__ void record_segment(const Plan& P, const uint32_t* wire, long long stride, int r,
                                                uint32_t seg, uint32_t* n, uint32_t* pay) {
     if (P.nseg == 1) {                           // read straight from the record: no offsets to look up
-        const uint32_t v = wire[(size_t)r * stride];
+        const uint32_t v = P.qz == QS_MINMAX ? P.kseg[0] : wire[(size_t)r * stride];
         *n = v <= P.kseg[0] ? v : 0u;
         *pay = 2u;
     } else {
@@ -1954,6 +1997,9 @@ __device__ __forceinline__ float entry_value(const Plan& P, const uint32_t* row,
     const uint32_t* w_lvl = w_sgn + words_for(en.n, 1);
     const bool neg = (w_sgn[en.j >> 5] >> (en.j & 31u)) & 1u;
     if (P.qz == QS_NONE) return __uint_as_float(w_sgn[en.j]);       // the value stream sits where the signs would
+    if (P.qz == QS_MINMAX)                                          // so does the level stream; the header pair is (min, max)
+        return minmax_value(__uint_as_float(row[2 * en.seg]), __uint_as_float(row[2 * en.seg + 1]), P.s,
+                            (int)get_bits(w_sgn, (uint64_t)en.j * P.bl, P.bl) + 1);
     const int level = qz_is_sign(P.qz) ? 1 : (int)get_bits(w_lvl, (uint64_t)en.j * P.bl, P.bl) + 1;
     return coord_value(P, __uint_as_float(row[2 * en.seg + 1]), level, neg, P.cscale[en.seg], P.kseg[en.seg]);
 }
@@ -1963,7 +2009,7 @@ __device__ void stage_dec_mark(const Plan& P, const Active& act, const uint32_t*
     for (uint64_t id = (uint64_t)blockIdx.x * BT + threadIdx.x; id < total; id += (uint64_t)gridDim.x * BT) {
         const int r = act.r[id / P.K];
         Entry en;
-        if (P.nseg == 1 && id % P.K == 0 && wire[(size_t)r * stride] > P.kseg[0]) set_status(P, QS_INVALID_ARG);
+        if (P.nseg == 1 && P.qz != QS_MINMAX && id % P.K == 0 && wire[(size_t)r * stride] > P.kseg[0]) set_status(P, QS_INVALID_ARG);
         if (!locate_entry(P, wire, stride, r, (uint32_t)(id % P.K), &en)) continue;
         if (en.coord < P.d) atomicOr(&P.touch[en.coord], 1u << r);
         else set_status(P, QS_INVALID_ARG);
@@ -2076,7 +2122,7 @@ constexpr size_t MID_SCRATCH_BYTES = (ORDER_ITEMS_MAX + 8) * sizeof(uint32_t) + 
 constexpr size_t MID_POOL_BYTES = sizeof(BcBlock) > MID_SCRATCH_BYTES ? sizeof(BcBlock) : MID_SCRATCH_BYTES;
 
 // what a lane keeps about the unit (its worker, a segment) its candidates mostly belong to
-struct UnitLite { uint32_t tau, tie_max, k, end; float norm, c; };
+struct UnitLite { uint32_t tau, tie_max, k, end; float norm, c, lo; };   // (min/max quantizer: lo = smallest, norm = largest kept value)
 
 // Lanes to workers: the warp is cut into as many equal parts as the next power of two of the
 // active workers; part j of worker slot w (lane w + j * parts) walks entries j, j + J, .. of the
@@ -2102,10 +2148,11 @@ __device__ __forceinline__ LaneMap lane_map(const Active& act, int lane) {
 }
 
 __device__ __forceinline__ UnitLite unit_lite(const Plan& P, const LaneMap& L, uint32_t seg) {
-    UnitLite u = {0u, 0u, 0u, 0u, 0.0f, 0.0f};
+    UnitLite u = {0u, 0u, 0u, 0u, 0.0f, 0.0f, 0.0f};
     if (L.live) {
         const Unit& g = P.units[(size_t)L.my_r * P.nseg + seg];
         u.tau = g.tau; u.tie_max = g.tie_max; u.norm = g.norm;
+        if (P.qz == QS_MINMAX) { u.lo = order_float(g.emin); u.norm = order_float(g.emax); }
         u.k = P.kseg[seg]; u.c = P.cscale[seg]; u.end = P.seg_off[seg + 1];
     }
     return u;
@@ -2167,6 +2214,8 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
             if (sent) {
                 if (P.qz == QS_NONE) {
                     gv = val;
+                } else if (P.qz == QS_MINMAX) {
+                    gv = minmax_value(u.lo, u.norm, P.s, minmax_level(val, u.lo, u.norm, P.s, philox_word(P, my_r, idx, 0u)));
                 } else {
                     int level = 1;
                     if (!qz_is_sign(P.qz)) level = qsgd_level(val, u.norm, P.s, philox_word(P, my_r, idx, 0u));
@@ -2661,7 +2710,7 @@ __global__ void __launch_bounds__(256) export_kernel(const Plan P, long long* se
         if (sign) sign[i] = (q & Q_NEG) ? 1 : 0;
     }
     for (uint32_t u = blockIdx.x * 256u + threadIdx.x; u < P.U; u += gridDim.x * 256u) {
-        if (norm) norm[u] = P.units[u].norm;
+        if (norm) norm[u] = P.qz == QS_MINMAX ? order_float(P.units[u].emax) : P.units[u].norm;
         if (n) n[u] = P.units[u].n;
     }
 }

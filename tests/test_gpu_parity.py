@@ -150,7 +150,8 @@ def test_config1_single_round():
 @pytest.mark.parametrize("d,k", [(1, 1), (2, 1), (2, 2), (31, 4), (32, 32), (33, 7), (127, 9), (128, 1), (129, 129),
                                  (1000, 10), (4099, 41), (7850, 40)])
 @pytest.mark.parametrize("sp,qz", [(O.TOPK, O.QSGD), (O.TOPK, O.SIGN_L1), (O.RANDK, O.QSGD_SCALED), (O.RANDK, O.SIGN_L1),
-                                   (O.TOPK, O.NONE), (O.RANDK, O.NONE), (O.TOPK, O.SIGN_L2)])
+                                   (O.TOPK, O.NONE), (O.RANDK, O.NONE), (O.TOPK, O.SIGN_L2), (O.TOPK, O.MINMAX),
+                                   (O.RANDK, O.MINMAX)])
 def test_small_and_ragged_sizes(d, k, sp, qz):
     R = 3
     x, xw, mem = I.gaussian_round(R, d, seed=d)
@@ -173,7 +174,7 @@ def test_ties_zeros_and_equal_values(d):
     few = g.choice(np.array([0.0, 1.0, -1.0, 2.0, -0.0], np.float32), size=(R, d)).astype(np.float32)
     cases.append((np.zeros(d, np.float32), few, z.copy(), d * 6 // 25))               # five distinct values
     for x, xw, mem, k in cases:
-        for qz in (O.QSGD, O.SIGN_L1):
+        for qz in (O.QSGD, O.SIGN_L1, O.MINMAX):
             p = Pair(R, d, k=k, s=16, quantizer=qz, seed=1, x=x, xw=xw, mem=mem)
             p.round_split(0)
             p.round_fused(1)
@@ -181,7 +182,7 @@ def test_ties_zeros_and_equal_values(d):
 
 
 @pytest.mark.parametrize("d", [40, 200, 3000, 20000])
-@pytest.mark.parametrize("qz", [O.QSGD, O.SIGN_L1, O.SIGN_L2])
+@pytest.mark.parametrize("qz", [O.QSGD, O.SIGN_L1, O.SIGN_L2, O.MINMAX])
 def test_norm_over_wide_exponent_ranges(d, qz):
     # kept values spread over sixty binary orders of magnitude (and a few subnormals): the exact sum
     # cannot take the short 64/128-bit route and goes through the long accumulator, in each of the
@@ -229,7 +230,7 @@ def test_per_tensor_and_flat_over_rounds():
                 dict(offsets=off, kseg=I.k_per_tensor_ratio(sizes)),
                 dict(offsets=off, kseg=I.k_per_tensor_capped(sizes, 10))]
     for kw in variants:
-        for qz in (O.SIGN_L1, O.QSGD, O.NONE, O.SIGN_L2):
+        for qz in (O.SIGN_L1, O.QSGD, O.NONE, O.SIGN_L2, O.MINMAX):
             p = Pair(R, d, s=16, quantizer=qz, seed=3, x=x, xw=np.broadcast_to(x, (R, d)).copy(), mem=zeros, **kw)
             for rnd in range(6):
                 p.drift(I.laplace_drift(R, off, scales, 0, rnd))
@@ -294,7 +295,7 @@ def test_colliding_workers():
     x, xw, mem = I.gaussian_round(R, d, seed=13)
     xw[:] = xw[0]
     mem[:] = mem[0]
-    for qz in (O.QSGD, O.SIGN_L1, O.NONE, O.SIGN_L2):
+    for qz in (O.QSGD, O.SIGN_L1, O.NONE, O.SIGN_L2, O.MINMAX):
         p = Pair(R, d, k=k, s=16, quantizer=qz, seed=4, x=x, xw=xw, mem=mem)
         p.round_fused(0)
         p.close()
@@ -522,3 +523,20 @@ def test_bounded_wait_runs_out_and_the_context_recovers(monkeypatch):
     p.drift(I.gaussian_drift(R, d, 5, 1, std=1e-2))
     p.round_split(1)
     p.close()
+
+
+def test_minmax_quantizer_rounds_with_masks_and_long_lists():
+    """The stochastic quantizer between the smallest and largest kept entry over several rounds: long
+    candidate lists (the grid-wide stages), asynchronous masks with anchors, and two levels only."""
+    R, d, k = 4, 120000, 9000
+    x, xw, mem = I.gaussian_round(R, d, seed=43)
+    anchors = np.broadcast_to(x, (R, d)).copy()
+    for s, anc in ((2, None), (7, anchors)):
+        p = Pair(R, d, k=k, s=s, quantizer=O.MINMAX, seed=10, x=x, xw=xw, mem=mem, anchors=anc)
+        masks = [None, np.array([1, 0, 1, 1], np.uint8), None] if anc is not None else [None] * 3
+        for rnd, m in enumerate(masks):
+            p.drift(I.gaussian_drift(R, d, 6, rnd, std=1e-2))
+            (p.round_fused if rnd % 2 else p.round_split)(rnd, m)
+        p.close()
+    with pytest.raises(B.QsError):                   # one level is not a quantizer between two values
+        B.Context(2, 100, 10, 1, B.QS_TOPK, B.QS_MINMAX)
