@@ -1429,8 +1429,13 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
             tau = S.ctl[1];
             tie_max = S.ctl[4];
         } else {
-            if (threadIdx.x == 0) { S.ctl[1] = 0u; S.ctl[2] = k; }
-            for (int level = 0; level < 4; ++level) {
+            // level 0 (the top key byte) was counted per unit by the order stage
+            if (wid == 0) {
+                uint32_t bin, above;
+                find_bin(P.hist + (size_t)u * 256, k, lane, &bin, &above);
+                if (lane == 0) { S.ctl[1] = bin; S.ctl[2] = k - above; S.ctl[3] = P.hist[(size_t)u * 256 + bin]; }
+            }
+            for (int level = 1; level < 4; ++level) {
                 const int shift = 24 - 8 * level;
                 S.hist[threadIdx.x] = 0u;
                 __syncthreads();
