@@ -31,7 +31,8 @@
  *   - Status codes: QS_OK = 0, negative = error.  Nothing is printed, nothing aborts.
  *   - worker_mask: host array of R bytes, non-zero = worker takes part; NULL = all.
  *   - R <= 32, 1 <= k <= d <= 2^32 - 4096 (coordinates are counted in 32 bits, in tiles of
- *     2048), 1 <= s <= 65535, round < 2^56, R x nseg <= 2048.
+ *     2048), 1 <= s <= 65535, round < 2^56, R x nseg <= 16384 (up to 2048 (worker, segment)
+ *     units their table lives in shared memory; beyond that it is read from global memory).
  *
  * Arithmetic (identical, operation for operation, to the CPU checker under oracle/):
  *   fp32 with no fused multiply-add; u = mem + (x - xw); Top_k orders by the bit

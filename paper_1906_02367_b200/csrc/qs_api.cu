@@ -154,7 +154,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     const int64_t d = (int64_t)P.d;
     if (nseg < 1 || !offsets || !kseg || offsets[0] != 0 || offsets[nseg] != d)
         return fail(c, QS_INVALID_ARG, "segments must start at 0 and end at d");
-    if ((int64_t)P.R * nseg > UT_MAX) return fail(c, QS_INVALID_ARG, "R x nseg exceeds the unit table (2048)");
+    if ((int64_t)P.R * nseg > U_MAX) return fail(c, QS_INVALID_ARG, "R x nseg exceeds 16384 units");
     for (int g = 0; g < nseg; ++g) {
         const int64_t n = offsets[g + 1] - offsets[g];
         if (n < 1 || kseg[g] < 1 || kseg[g] > n) return fail(c, QS_INVALID_ARG, "need 1 <= k_seg <= segment length");
@@ -255,6 +255,7 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     AL(chunk_cnt, (size_t)P.maxchunks + 1, true);
     AL(chunk_dir, (size_t)P.maxchunks + 1, false);
     AL(unit_tab, P.U, false);
+    if (P.U > (uint32_t)UT_MAX) { AL(gtab, (size_t)4 * (P.U + 1) + 8, true); } else P.gtab = nullptr;
     AL(chunk_sel, (size_t)P.maxchunks + 1, true);
     AL(chunk_nz, (size_t)P.maxchunks + 1, true);
     AL(fb_hist, (size_t)P.U * FB_BINS, true);

@@ -18,6 +18,7 @@ constexpr int SUP_BLOCKS = 64;       // blocks per super-block of the two-level 
 #endif
 constexpr int CHUNK = QS_CHUNK;     // candidates per selection chunk (a multiple of the 256 threads)
 constexpr int UT_MAX = 2048;         // units whose table fits in the persistent kernel's shared memory
+constexpr int U_MAX = 16384;         // units in all: (worker, segment) pairs
 constexpr uint32_t ORDER_SUPS_MAX = 2048;   // (worker, super-block) sums the order stage can hold in shared memory
 constexpr int UNIT_CAP = 6144;       // candidates of a unit that one block may select from on its own (16 per thread)
 constexpr int FB_BINS = 2048;        // bins of the exact fallback histogram (top 11 key bits)
@@ -101,6 +102,7 @@ struct Plan {
     uint32_t* chunk_cnt;       // maxchunks + 1 (kept | sent << 16 per chunk)
     uint32_t* chunk_dir;       // maxchunks: unit of each chunk, for the packing warps of the closing stage
     uint4* unit_tab;           // U: (start, candidates, first chunk) of each unit, likewise
+    uint32_t* gtab;            // 4 (U + 1) + 8 words: the unit table of every block when U > UT_MAX (else null)
     uint32_t* chunk_sel;       // maxchunks + 1 exclusive sums of kept
     uint32_t* chunk_nz;        // maxchunks + 1 exclusive sums of sent
     uint32_t* fb_hist;         // U x FB_BINS, zero between rounds

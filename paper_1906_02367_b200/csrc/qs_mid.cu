@@ -454,6 +454,35 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
     return sh_flag[0];
 }
 
+// The unit table where every block can read it.  Up to UT_MAX units every block builds its own
+// copy in shared memory.  More units than that: block 0 builds the table in global memory, writes
+// the few numbers that go with it, and after a grid barrier every block reads it from there.
+// Returns false when that barrier gave up.
+__device__ bool table_step(const Plan& P, const Active& act, uint32_t* sh_tab, uint32_t* sh_scan, uint32_t* sh_flag, Tab* tab,
+                           uint32_t* missed, uint32_t& target, int* sh_abort) {
+    if (P.U <= (uint32_t)UT_MAX) {
+        *missed = build_table(P, act, sh_tab, sh_tab + UT_MAX, sh_tab + 2 * UT_MAX, sh_tab + 3 * UT_MAX + 4, sh_scan, sh_flag, tab);
+        return true;
+    }
+    uint32_t* g = P.gtab;
+    const uint32_t n = P.U + 1u;
+    if (blockIdx.x == 0) {
+        const uint32_t m = build_table(P, act, g, g + n, g + 2 * n, g + 3 * n, sh_scan, sh_flag, tab);
+        if (threadIdx.x == 0) {
+            uint32_t* info = g + 4 * n;
+            info[0] = tab->total_chunks; info[1] = tab->total_long; info[2] = tab->short_c;
+            info[3] = tab->any_short ? 1u : 0u; info[4] = tab->fast ? 1u : 0u; info[5] = m;
+        }
+    }
+    if (!grid_barrier(P, target, sh_abort)) return false;
+    const uint32_t* info = g + 4 * n;
+    tab->start = g; tab->c = g + n; tab->cb = g + 2 * n; tab->lb = g + 3 * n;
+    tab->total_chunks = info[0]; tab->total_long = info[1]; tab->short_c = info[2];
+    tab->any_short = info[3] != 0u; tab->fast = info[4] != 0u;
+    *missed = info[5];
+    return true;
+}
+
 // histogram of the top 11 key bits of one stretch of one segment, for missed workers
 template <bool RANDK>
 __device__ void stage_fb_hist(const Plan& P, const Active& act, uint32_t missed, uint32_t* sh_bins) {
@@ -2567,11 +2596,7 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
     uint32_t* sh_tab = reinterpret_cast<uint32_t*>(sh_pool);
     unsigned char* sh_big = sh_pool + (ORDER_ITEMS_MAX + 8) * sizeof(uint32_t);
     static_assert(MID_SCRATCH_BYTES <= MID_POOL_BYTES, "the stages' scratch must fit the pool");
-    uint32_t* t_start = sh_tab;
-    uint32_t* t_c = sh_tab + UT_MAX;
-    uint32_t* t_cb = sh_tab + 2 * UT_MAX;         // UT_MAX + 1 entries
-    uint32_t* t_lb = sh_tab + 3 * UT_MAX + 4;     // UT_MAX + 1 entries
-    static_assert(4 * UT_MAX + 5 <= ORDER_ITEMS_MAX + 8, "the unit table must fit");
+    static_assert(4 * UT_MAX + 5 <= ORDER_ITEMS_MAX + 8, "the unit table (four arrays of up to UT_MAX + 1 entries) must fit");
     static_assert(sizeof(UnitSh) <= FB_BINS * 4, "the unit stage's scratch must fit");
     const Plan& P = a.P;
     const Active& act = a.act;
@@ -2604,7 +2629,8 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         if (even) stage_order_even<RANDK>(P, act, 0u, bins, sh_tab, sh_scan);
         else stage_order<RANDK>(P, act, 0u, bins);
         QS_BARRIER();
-        const uint32_t missed = build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab);
+        uint32_t missed = 0;
+        if (!table_step(P, act, sh_tab, sh_scan, sh_flag, &tab, &missed, target, &sh_abort)) break;
         if (missed) {                              // the same value in every block
             stage_fb_hist<RANDK>(P, act, missed, bins);
             QS_BARRIER();
@@ -2615,7 +2641,9 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
             if (even) stage_order_even<RANDK>(P, act, missed, bins, sh_tab, sh_scan);
             else stage_order<RANDK>(P, act, missed, bins);
             QS_BARRIER();
-            if (build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab)) set_status(P, QS_STATE);   // the exact pass cannot miss
+            uint32_t again = 0;
+            if (!table_step(P, act, sh_tab, sh_scan, sh_flag, &tab, &again, target, &sh_abort)) break;
+            if (again) set_status(P, QS_STATE);    // the exact pass cannot miss
             if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd((unsigned long long*)&P.stats[0], (unsigned long long)__popc(missed));
         }
         if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -2650,7 +2678,8 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
             QS_BARRIER();
         }
     } else if (a.do_pack) {
-        build_table(P, act, t_start, t_c, t_cb, t_lb, sh_scan, sh_flag, &tab);
+        uint32_t unused = 0;
+        if (!table_step(P, act, sh_tab, sh_scan, sh_flag, &tab, &unused, target, &sh_abort)) break;
         QS_BARRIER();                              // the zeroed records
     }
     // Thresholds, tie cuts and norms are known.

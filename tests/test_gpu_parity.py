@@ -540,3 +540,20 @@ def test_minmax_quantizer_rounds_with_masks_and_long_lists():
         p.close()
     with pytest.raises(B.QsError):                   # one level is not a quantizer between two values
         B.Context(2, 100, 10, 1, B.QS_TOPK, B.QS_MINMAX)
+
+
+def test_more_units_than_the_shared_memory_table_holds():
+    """R x nseg above 2048: the ResNet-50-shaped table (161 segments, shrunk 64x) with sixteen workers makes
+    2576 (worker, segment) units, whose table the persistent kernel then keeps in global memory."""
+    sizes = I.scaled_sizes(I.resnet50_tensor_sizes(), 64)
+    off = I.segments_from_sizes(sizes)
+    d, R = int(off[-1]), 16
+    scales = I.tensor_scales(len(sizes), seed=0)
+    x = I.model_init(d, seed=0)
+    for qz in (O.SIGN_L1, O.QSGD):
+        p = Pair(R, d, s=16, quantizer=qz, seed=13, x=x, xw=np.broadcast_to(x, (R, d)).copy(), mem=np.zeros((R, d), np.float32),
+                 offsets=off, kseg=I.k_per_tensor_ratio(sizes))
+        for rnd in range(4):
+            p.drift(I.laplace_drift(R, off, scales, 1, rnd))
+            (p.round_fused if rnd % 2 else p.round_split)(rnd)
+        p.close()
