@@ -217,6 +217,36 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
             h_grp[g] = (uint32_t)sg;
         }
     }
+    // Tiles in which the workers together keep more entries than there are coordinates (small
+    // tensors kept whole, Section 5.1's k_t = min(d_t, 1000)) cost one warp of the closing stage
+    // many times an ordinary tile: they are handed out first, so that the rest of the stage hides them.
+    std::vector<uint32_t> h_tiles;
+    {
+        std::vector<double> crowd(P.ntile, 0.0);
+        bool any = false;
+        for (int g = 0; g < nseg; ++g) {
+            const int64_t n = offsets[g + 1] - offsets[g];
+            const double per = (double)R * (double)std::min<uint64_t>(h_target[g], (uint64_t)n) / (double)n;
+            if (per < 0.25) continue;                              // (ordinary ratios: never crowded)
+            for (int64_t t = offsets[g] / STILE; t * STILE < offsets[g + 1]; ++t) {
+                const int64_t a = std::max<int64_t>(offsets[g], t * STILE), b = std::min<int64_t>(offsets[g + 1], (t + 1) * STILE);
+                crowd[t] += per * (double)(b - a);
+            }
+        }
+        std::vector<uint32_t> heavy, rest;
+        for (uint32_t t = 0; t < P.ntile; ++t) (crowd[t] > 1024.0 ? heavy : rest).push_back(t);
+        any = !heavy.empty();
+        if (any) {
+            std::stable_sort(heavy.begin(), heavy.end(), [&](uint32_t a, uint32_t b) { return crowd[a] > crowd[b]; });
+            // every eighth place at the front: a block draws a handful of tiles when it starts, and
+            // should get one crowded tile among them, not all of them
+            const size_t gap = heavy.size() * 8 <= P.ntile ? 8 : 1;
+            size_t ih = 0, ir = 0;
+            h_tiles.resize(P.ntile);
+            for (size_t t = 0; t < P.ntile; ++t)
+                h_tiles[t] = (ih < heavy.size() && (t % gap == 0 || ir == rest.size())) ? heavy[ih++] : rest[ir++];
+        }
+    }
     // first prediction: none for Top_k (the first round takes the exact pass); for Rand_k the
     // hash is uniform, so the cut that lets `target` coordinates through is known in advance
     h_guess.assign((size_t)R * nseg, NO_GUESS);
@@ -233,11 +263,14 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
 #define UP(field, vec) if ((rc = dev_upload(c, &P.field, vec)) != QS_OK) return rc
     UP(seg_off, h_off); UP(kseg, h_k); UP(kprefix, h_kp); UP(grp_seg, h_grp); UP(target, h_target);
     UP(cscale, h_c); UP(bidx, h_bi); UP(fb_tab, h_fb); UP(seg_order, h_order);
+    P.tile_order = nullptr;
+    if (!h_tiles.empty()) UP(tile_order, h_tiles);
 #undef UP
     const uint32_t* g_up = nullptr;
     if ((rc = dev_upload(c, &g_up, h_guess)) != QS_OK) return rc;
     P.guess = const_cast<uint32_t*>(g_up);
 #define AL(field, count, zero) if ((rc = dev_alloc(c, &P.field, (size_t)(count), zero)) != QS_OK) return rc
+    AL(wary, P.U, true);
     AL(stage, (size_t)R * P.cap, false);
     AL(tile_cnt, (size_t)R * P.nblk * BLK_TILES, true);
     AL(blk_count, (size_t)R * P.nblk, true);
@@ -301,7 +334,7 @@ uint64_t take_round(qs_ctx* c, uint64_t round) {
 
 int run_mid(qs_ctx* c, const Active& act, int do_compress, int do_pack, int do_decode, int do_broadcast,
             uint32_t* wire, int64_t stride, int64_t* bits_out) {
-    const cudaError_t e = launch_mid(c->P, act, do_compress, do_pack, do_decode, 0, do_broadcast, c->aligned ? 1 : 0,
+    const cudaError_t e = launch_mid(c->P, act, do_compress, do_pack, do_decode, do_broadcast, c->aligned ? 1 : 0,
                                      wire, stride, (long long)c->wire_words, (long long*)bits_out, c->mid_grid, c->st);
     c->P.test_miss_barrier = 0;                    // the test of the bounded wait concerns one launch
     if (e != cudaSuccess) return cuda_fail(c, e, "persistent kernel");

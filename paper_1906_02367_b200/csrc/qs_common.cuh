@@ -78,6 +78,7 @@ struct Plan {
     const uint32_t* grp_seg;   // ngroups: segment of the group's first coordinate
     const uint32_t* target;    // nseg: candidates aimed for
     const uint32_t* seg_order; // nseg: segments by falling candidate target (largest units are dealt first)
+    const uint32_t* tile_order; // ntile, or null for 0, 1, 2, ..: the order in which the closing stage hands tiles out (crowded tiles first)
     const float* cscale;       // nseg: fl32(1 / (1 + beta_{k,s}))
     const uint8_t* bidx;       // nseg: bits per index field
     const FbBlock* fb_tab;     // nfb
@@ -85,6 +86,7 @@ struct Plan {
     float* x; float* xw; float* mem; float* anchors;
     // scratch
     uint32_t* guess;           // R x nseg, sort-key space
+    uint32_t* wary;            // R x nseg: rounds for which the unit's prediction still aims wide after a miss
     uint2* stage;              // R x cap (index, value bits): candidates as the dense pass left them, tile t at t * STILE
     uint32_t* tile_cnt;        // R x (nblk x BLK_TILES): rows padded to whole blocks, the padding stays zero
     uint32_t* blk_count;       // R x nblk, zero between rounds

@@ -15,7 +15,7 @@ bool pass_a_tma_usable(const Plan& P, bool aligned, int step);
 cudaError_t launch_pass_a_tma(const Plan& P, const Active& act, const StepArgs& sa, int step, int sms, cudaStream_t st);
 // qs_mid.cu: the persistent kernel that runs every stage after the dense pass
 int mid_blocks_per_sm(bool randk);
-cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode, int patch,
+cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode,
                        int do_broadcast, int aligned, uint32_t* wire, long long stride, long long wire_words,
                        long long* bits_out, int grid, cudaStream_t st);
 void launch_export(const Plan& P, long long* sel_idx, int* level, uint8_t* sign, float* norm, long long* n,

@@ -12,12 +12,14 @@
 //               the stored u)
 //   select      radix select over the 32-bit sort key (4 levels of 8 bits), tie cut by lower
 //               index, next round's prediction; units with short candidate lists are selected
-//               from by one block each, with block barriers only, beside the first level
-//   quantize    exact norm of the kept values, levels and signs (Philox stream 0), m <- u - g,
-//               ordered positions of kept and sent entries
-//   pack        directory and the three bit streams of every segment
-//   decode      senders of every index, then one owner per index adds the values in worker
-//               order, updates x and (fused round) patches the workers' copies
+//               from by one block (or warp) each, with block barriers only, beside the first level
+//   quantize    exact norm of the kept values (or their smallest and largest), levels and signs
+//               (Philox stream 0), m <- u - g, ordered positions of kept and sent entries
+//   pack        directory and the bit streams of every segment
+//   closing     whole round: the master's update and the broadcast in one pass over x (the kept
+//               entries are found again in the dense pass's runs), the records written beside it
+//   decode      separate master call: senders of every index from the record words, then one
+//               owner per index adds the values in worker order and updates x
 //
 // Order-dependent results come only from ordered scans, never from the order of atomics.
 #include "qs_bulk.cuh"
@@ -31,7 +33,7 @@ constexpr int PER = CHUNK / BT;            // candidates per thread and chunk
 struct MidArgs {
     Plan P;
     Active act;
-    int do_compress, do_pack, do_decode, patch, do_broadcast, aligned;
+    int do_compress, do_pack, do_decode, do_broadcast, aligned;
     uint32_t* wire;
     long long stride, wire_words;
     long long* bits_out;
@@ -542,7 +544,12 @@ __device__ void stage_fb_guess(const Plan& P, const Active& act, uint32_t missed
             }
         }
         __syncthreads();
-        if (threadIdx.x == 0) P.guess[(size_t)r * P.nseg + seg] = *sh_best << FB_SHIFT;
+        if (threadIdx.x == 0) {
+            // rounds of wider slack after a miss (predict_floor); the first round of a context has no
+            // prediction to miss
+            if (P.guess[(size_t)r * P.nseg + seg] != NO_GUESS) P.wary[(size_t)r * P.nseg + seg] = 16u;
+            P.guess[(size_t)r * P.nseg + seg] = *sh_best << FB_SHIFT;
+        }
         __syncthreads();
     }
     for (int w = 0; w < act.n; ++w) {
@@ -758,8 +765,20 @@ __device__ void stage_hist(const Plan& P, const Tab& tab, int level, uint32_t* s
 // coordinates pass it, assuming the tail keeps its shape (log-linear in the count).  One thread.
 __device__ void predict_floor(const Plan& P, uint32_t r, uint32_t seg, uint32_t tau, uint32_t uc, uint32_t k) {
     uint32_t* gp = &P.guess[(size_t)r * P.nseg + seg];
+    const uint32_t n = P.seg_off[seg + 1] - P.seg_off[seg];
+    uint32_t want = P.target[seg];
+    // A unit whose prediction missed lately aims for three times the usual slack for a while: a
+    // workload whose scale jumps from round to round (workers that synchronise at uneven gaps)
+    // then pays with longer lists instead of with exact passes.
+    uint32_t* wary = &P.wary[(size_t)r * P.nseg + seg];
+    if (*wary) {
+        *wary -= 1u;
+        const uint64_t wide = (uint64_t)k + 3ull * (want - k);
+        want = wide < n ? (uint32_t)wide : n;
+    }
+    if (want >= n) { *gp = 0u; return; }          // every coordinate is a candidate (k = n, or nearly)
     const float tk = __uint_as_float(tau >> 1), tg = __uint_as_float(*gp >> 1);
-    const float target = (float)P.target[seg];
+    const float target = (float)want;
     float tn = tg;
     if (uc > k && tk > tg) {
         float ratio = __logf(target / (float)k) / __logf((float)uc / (float)k);
@@ -1005,7 +1024,7 @@ __device__ void stage_norm_accum(const Plan& P, const Tab& tab, bool merge, uint
     const bool plain = P.qz == QS_NONE;            // the plain sparsifier sends the values: no norm
     const bool mm = P.qz == QS_MINMAX;             // smallest and largest kept value in place of a norm
     // merge: a whole round with a quantizer that sends every kept entry at level 1; the counts and
-    // the sender bits are known here, and the pack stage does the rest of the quantize stage's work
+    // the kept entries are known here; the packing warps and the closing stage do the rest of the quantize stage's work
     const bool early = merge;
     const bool l1 = P.qz == QS_SIGN_L1;
     // A block takes consecutive chunks.  While they lie in one unit their sums stay in shared memory
@@ -1227,7 +1246,7 @@ __device__ void unit_norm(const Plan& P, uint32_t u, uint32_t count, uint32_t (*
 // kept set comes from ranks counted directly (key descending, list position ascending: the list
 // is in index order); above that from a four-level radix select over a histogram in shared
 // memory.  Then the tie cut, the next prediction, the exact norm (per-exponent sums in shared
-// memory) and, for the quantizers that send every kept entry, the sender bits and the kept counts
+// memory) and, for the quantizers that send every kept entry at level 1, the kept counts
 // per chunk.  Units are handed out by a ticket counter, largest first.
 constexpr int UPT = UNIT_CAP / BT;
 static_assert(UNIT_CAP % CHUNK == 0 && UNIT_CAP / CHUNK <= 16, "kept counts per chunk: sixteen slots");
@@ -1509,7 +1528,7 @@ __device__ void stage_unit(const Plan& P, const Tab& tab, const Active& act, boo
         }
         // the level-0 counts of the order stage are not needed on this path: leave them zero
         P.hist[(size_t)u * 256 + threadIdx.x] = 0u;
-        // kept entries: exact sums per exponent, sender bits and kept counts per chunk
+        // kept entries: exact sums per exponent (or smallest / largest value) and kept counts per chunk
         const bool ties = tie_max != 0xffffffffu;
         auto take = [&](uint32_t i, uint32_t off, uint32_t kv, uint32_t idx, uint32_t vb) {
             const bool kept = off < c && kv >= tau && !(ties && kv == tau && idx > tie_max);
@@ -2051,8 +2070,8 @@ __device__ void stage_dec_mark(const Plan& P, const Active& act, const uint32_t*
 }
 
 // The lowest worker that sent an index owns it: it adds the values of all senders in increasing
-// worker order, updates x, and in the fused round patches the workers' copies.
-__device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t* wire, long long stride, int patch) {
+// worker order and updates x.
+__device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t* wire, long long stride) {
     const uint64_t total = (uint64_t)act.n * P.K;
     for (uint64_t id = (uint64_t)blockIdx.x * BT + threadIdx.x; id < total; id += (uint64_t)gridDim.x * BT) {
         const int r = act.r[id / P.K];
@@ -2084,12 +2103,6 @@ __device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t
         }
         const float xn = P.x[en.coord] - acc / (float)P.rdiv;
         P.x[en.coord] = xn;
-        if (patch) {
-            for (int w = 0; w < act.n; ++w) {
-                P.xw[(size_t)act.r[w] * P.d + en.coord] = xn;
-                if (P.anchors) P.anchors[(size_t)act.r[w] * P.d + en.coord] = xn;
-            }
-        }
         P.touch[en.coord] = 0u;
     }
 }
@@ -2224,6 +2237,7 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
     // Entry i of this lane's worker's run: sent?  position in the tile and value.  The first look
     // at an entry leaves the answer in its place (in shared memory, or in the run itself, which
     // nothing reads after this stage), so that the random draws and the division are made once.
+    UnitLite later = {0u, 0u, 0u, 0u, 0.0f, 0.0f, 0.0f};
     auto cand = [&](uint32_t i, bool first, uint32_t* pos, float* g) -> bool {
         uint2* home = staged ? &cb[pbefore + i] : &run[i];
         const uint2 ent = *home;
@@ -2238,9 +2252,12 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
         if (sent) {
             UnitLite u = un;
             if (idx >= un.end) {                      // a later segment of the tile: look its unit up
-                uint32_t seg = gseg[(idx - e0) >> 7];
-                while (seg + 1 < (uint32_t)P.nseg && idx >= P.seg_off[seg + 1]) ++seg;
-                u = unit_lite(P, L, seg);
+                if (idx >= later.end) {               // (a lane's entries come in rising order: the last one looked up serves until its end)
+                    uint32_t seg = gseg[(idx - e0) >> 7];
+                    while (seg + 1 < (uint32_t)P.nseg && idx >= P.seg_off[seg + 1]) ++seg;
+                    later = unit_lite(P, L, seg);
+                }
+                u = later;
             }
             const float val = __uint_as_float(ent.y);
             const uint32_t key = RANDK ? ~philox_word(P, my_r, idx, 1u) : topk_key(val);
@@ -2285,6 +2302,52 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
     __syncwarp();
     const uint32_t m_lo = W.bm2[lane], m_hi = W.bm2[lane + 32];
     const bool any_multi = __any_sync(0xffffffffu, (m_lo | m_hi) != 0u);
+    // rank of a coordinate among those with several senders: popcounts before its word
+    uint32_t npos = 0;
+    if (any_multi) {
+        const uint32_t c_lo = __popc(m_lo), c_hi = __popc(m_hi);
+        const uint32_t i_lo = warp_incl_scan(c_lo, lane), i_hi = warp_incl_scan(c_hi, lane);
+        const uint32_t n_lo = __shfl_sync(0xffffffffu, i_lo, 31);
+        npos = n_lo + __shfl_sync(0xffffffffu, i_hi, 31);
+        W.pref[lane] = i_lo - c_lo;
+        W.pref[lane + 32] = n_lo + i_hi - c_hi;
+        __syncwarp();
+    }
+    if (npos > wp) {
+        // Many coordinates with several senders (small tensors that every worker sends whole):
+        // the sums are formed in the tile's own buffer, worker after worker in their order, all
+        // lanes on one worker's entries at a time; x itself is read again from global memory, which
+        // still holds the round's model.  A worker sends a coordinate at most once, so its lanes
+        // never meet at one sum, and a coordinate with one sender gets 0 + g as everywhere else.
+        // Time is in proportion to the candidates.
+        for (uint32_t j = lane; j < nel; j += 32)
+            if ((W.bm1[j >> 5] >> (j & 31u)) & 1u) xs[j] = 0.0f;
+        __syncwarp();
+        for (int w = 0; w < L.nact; ++w) {
+            const uint32_t cnt_w = __shfl_sync(0xffffffffu, cnt, w);
+            const uint32_t pb_w = __shfl_sync(0xffffffffu, pbefore, w);
+            const uint32_t r_w = __shfl_sync(0xffffffffu, my_r, w);
+            const uint2* run_w = staged ? cb + pb_w : P.stage + (size_t)r_w * P.cap + (size_t)tile * STILE;
+            for (uint32_t i0 = 0; i0 < cnt_w; i0 += 128u) {
+                uint2 e[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t i = i0 + (uint32_t)q * 32u + (uint32_t)lane;
+                    e[q] = i < cnt_w ? run_w[i] : make_uint2(0u, 0u);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (e[q].x >> 31) {
+                        const uint32_t pos = e[q].x & (uint32_t)(STILE - 1);
+                        xs[pos] = xs[pos] + __uint_as_float(e[q].y);
+                    }
+            }
+            __syncwarp();
+        }
+        for (uint32_t j = lane; j < nel; j += 32)
+            if ((W.bm1[j >> 5] >> (j & 31u)) & 1u) xs[j] = P.x[e0 + j] - xs[j] / rdiv;
+        __syncwarp();
+    } else {
     // coordinates with one sender
     for (uint32_t i = my_j; i < cnt; i += J) {
         uint32_t pos = 0;
@@ -2296,14 +2359,6 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
         }
     }
     if (any_multi) {
-        // rank of a coordinate among those with several senders: popcounts before its word
-        const uint32_t c_lo = __popc(m_lo), c_hi = __popc(m_hi);
-        const uint32_t i_lo = warp_incl_scan(c_lo, lane), i_hi = warp_incl_scan(c_hi, lane);
-        const uint32_t n_lo = __shfl_sync(0xffffffffu, i_lo, 31);
-        const uint32_t npos = n_lo + __shfl_sync(0xffffffffu, i_hi, 31);
-        W.pref[lane] = i_lo - c_lo;
-        W.pref[lane + 32] = n_lo + i_hi - c_hi;
-        __syncwarp();
         for (uint32_t w0 = 0; w0 < npos; w0 += wp) {
             for (uint32_t i = my_j; i < cnt; i += J) {
                 uint32_t pos = 0;
@@ -2347,6 +2402,7 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
             if (lane == 0) W.nm = 0u;
             __syncwarp();
         }
+    }
     }
     __syncwarp();                                     // every lane is done with the tile and the bitmaps
     // x in global memory: every changed coordinate's 32-byte sector, whole and once (a sector
@@ -2431,7 +2487,11 @@ __device__ void stage_update_broadcast(const Plan& P, const Active& act, BcBlock
         // tickets are drawn two tiles ahead of the copies and counts read one tile ahead, so that
         // neither round trip is on the path
         uint32_t tA = 0, tB = 0;
-        if (lane == 0) { tA = atomicAdd(P.bar + 2, 1u); tB = atomicAdd(P.bar + 2, 1u); }
+        auto draw = [&]() -> uint32_t {                // the next tile in the order they are handed out
+            const uint32_t t = atomicAdd(P.bar + 2, 1u);
+            return (P.tile_order && t < ntile) ? P.tile_order[t] : t;
+        };
+        if (lane == 0) { tA = draw(); tB = draw(); }
         tA = __shfl_sync(0xffffffffu, tA, 0);
         tB = __shfl_sync(0xffffffffu, tB, 0);
         auto gseg_of = [&](uint32_t tile) -> uint32_t {
@@ -2443,7 +2503,7 @@ __device__ void stage_update_broadcast(const Plan& P, const Active& act, BcBlock
             BcSlot& S = B.slot[s];
             const uint32_t tile = tA;
             uint32_t tC = 0;
-            if (lane == 0) tC = atomicAdd(P.bar + 2, 1u);
+            if (lane == 0) tC = draw();
             const uint32_t cntB = tile_count(P, L, tB), gsB = gseg_of(tB);
             if (tile >= ntile) {
                 if (lane == 0) { S.tile = NO_TILE; mbar_expect(&B.full[s], 0u); }
@@ -2710,7 +2770,7 @@ __global__ void __launch_bounds__(BT, 4) mid_kernel(const MidArgs a) {
         }
         stage_dec_mark(P, act, a.wire, a.stride);
         QS_BARRIER();
-        stage_dec_apply(P, act, a.wire, a.stride, a.patch);
+        stage_dec_apply(P, act, a.wire, a.stride);
     }
     } while (0);
 #undef QS_BARRIER
@@ -2760,12 +2820,12 @@ int mid_blocks_per_sm(bool randk) {
     return e == cudaSuccess ? per_sm : 0;
 }
 
-cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode, int patch,
+cudaError_t launch_mid(const Plan& P, const Active& act, int do_compress, int do_pack, int do_decode,
                        int do_broadcast, int aligned, uint32_t* wire, long long stride, long long wire_words,
                        long long* bits_out, int grid, cudaStream_t st) {
     MidArgs a;
     a.P = P; a.act = act;
-    a.do_compress = do_compress; a.do_pack = do_pack; a.do_decode = do_decode; a.patch = patch;
+    a.do_compress = do_compress; a.do_pack = do_pack; a.do_decode = do_decode;
     a.do_broadcast = do_broadcast; a.aligned = aligned;
     a.wire = wire; a.stride = stride; a.wire_words = wire_words; a.bits_out = bits_out;
     void* params[] = {&a};
