@@ -2145,7 +2145,7 @@ struct BcSlot {
     uint32_t gseg[STILE / GROUP];  // segment of the first coordinate of each 128-coordinate group
     uint32_t tile, staged;
     uint32_t whole;                // the working warp asks for the whole tile to be stored to x (many coordinates changed)
-    uint32_t pad;
+    uint32_t crowded;              // so many candidates that the tile is walked worker by worker
 };
 
 struct BcScratch {                 // of one working warp
@@ -2194,15 +2194,68 @@ __device__ __forceinline__ LaneMap lane_map(const Active& act, int lane) {
     return L;
 }
 
-__device__ __forceinline__ UnitLite unit_lite(const Plan& P, const LaneMap& L, uint32_t seg) {
-    UnitLite u = {0u, 0u, 0u, 0u, 0.0f, 0.0f, 0.0f};
-    if (L.live) {
-        const Unit& g = P.units[(size_t)L.my_r * P.nseg + seg];
-        u.tau = g.tau; u.tie_max = g.tie_max; u.norm = g.norm;
-        if (P.qz == QS_MINMAX) { u.lo = order_float(g.emin); u.norm = order_float(g.emax); }
-        u.k = P.kseg[seg]; u.c = P.cscale[seg]; u.end = P.seg_off[seg + 1];
-    }
+__device__ __forceinline__ UnitLite unit_of(const Plan& P, uint32_t r, uint32_t seg) {
+    UnitLite u;
+    const Unit& g = P.units[(size_t)r * P.nseg + seg];
+    u.tau = g.tau; u.tie_max = g.tie_max; u.norm = g.norm; u.lo = 0.0f;
+    if (P.qz == QS_MINMAX) { u.lo = order_float(g.emin); u.norm = order_float(g.emax); }
+    u.k = P.kseg[seg]; u.c = P.cscale[seg]; u.end = P.seg_off[seg + 1];
     return u;
+}
+
+__device__ __forceinline__ UnitLite unit_lite(const Plan& P, const LaneMap& L, uint32_t seg) {
+    const UnitLite none = {0u, 0u, 0u, 0u, 0.0f, 0.0f, 0.0f};
+    return L.live ? unit_of(P, L.my_r, seg) : none;
+}
+
+// First look at one entry of worker r's run in the tile that starts at e0: was it sent, and with
+// what value?  un: the unit of the tile's first segment, later: the last unit looked up beyond it
+// (a walk's entries come in rising order, so it serves until its segment ends).  mem_update: the
+// worker's memory at a sent coordinate is written here (quantizers without a quantize stage).
+template <bool RANDK>
+__device__ __forceinline__ bool first_look(const Plan& P, uint32_t r, const UnitLite& un, UnitLite& later, const uint32_t* gseg,
+                                           uint32_t e0, uint32_t nel, uint2 ent, bool mem_update, uint32_t* pos, float* g) {
+    const uint32_t idx = ent.x;
+    bool sent = idx >= e0 && idx - e0 < nel;                        // (an entry outside its tile is never written by the dense pass)
+    float gv = 0.0f;
+    if (sent) {
+        UnitLite u = un;
+        if (idx >= un.end) {                          // a later segment of the tile: look its unit up
+            if (idx >= later.end) {
+                uint32_t seg = gseg[(idx - e0) >> 7];
+                while (seg + 1 < (uint32_t)P.nseg && idx >= P.seg_off[seg + 1]) ++seg;
+                later = unit_of(P, r, seg);
+            }
+            u = later;
+        }
+        const float val = __uint_as_float(ent.y);
+        const uint32_t key = RANDK ? ~philox_word(P, r, idx, 1u) : topk_key(val);
+        sent = key > u.tau || (key == u.tau && idx <= u.tie_max);
+        if (sent) {
+            if (P.qz == QS_NONE) {
+                gv = val;
+            } else if (P.qz == QS_MINMAX) {
+                gv = minmax_value(u.lo, u.norm, P.s, minmax_level(val, u.lo, u.norm, P.s, philox_word(P, r, idx, 0u)));
+            } else {
+                int level = 1;
+                if (!qz_is_sign(P.qz)) level = qsgd_level(val, u.norm, P.s, philox_word(P, r, idx, 0u));
+                sent = level != 0;                                 // (level 0: kept, not sent)
+                if (sent) {                                        // the value as coord_value forms it
+                    if (qz_is_sign(P.qz)) {
+                        gv = u.norm / (float)u.k;
+                    } else {
+                        gv = (u.norm * (float)level) / (float)P.s;
+                        if (P.qz == QS_QSGD_SCALED) gv = gv * u.c;
+                    }
+                    if (val < 0.0f) gv = -gv;
+                }
+            }
+        }
+        if (mem_update && sent) P.mem[(size_t)r * P.d + idx] = val - gv;
+    }
+    *pos = sent ? idx - e0 : 0u;
+    *g = gv;
+    return sent;
 }
 
 // The update of one tile by one warp.  xs: the tile in shared memory; cnt: candidates of this
@@ -2213,11 +2266,12 @@ __device__ __forceinline__ UnitLite unit_lite(const Plan& P, const LaneMap& L, u
 // store the whole tile; taken when so many coordinates changed that one sequential store is cheaper
 // than their scattered sectors).
 constexpr uint32_t WHOLE_TILE_MIN = 64;
+constexpr uint32_t CROWDED_MIN = 1024;               // candidates of all workers from which a tile is walked worker by worker
 
 template <bool RANDK>
 __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t tile, uint32_t cnt, bool staged, uint2* cb,
                            uint32_t pbefore, const uint32_t* gseg, float* xs, BcScratch& W, const UnitLite& un, bool mem_update,
-                           bool can_whole) {
+                           bool can_whole, bool crowded) {
     const uint32_t e0 = tile * (uint32_t)STILE;
     const uint32_t nel = P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE;
     const float rdiv = (float)P.rdiv;
@@ -2227,7 +2281,8 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
     // What will be read from global memory is asked for now, all of it at once (one round trip in
     // place of one per entry): the run itself when it is not in shared memory, and the units of
     // the next few segments when the tile may hold more than one.
-    if (!staged)
+    constexpr uint32_t AHEAD = 8;                     // lines asked for ahead of a crowded tile's walk without the ring
+    if (!staged && !crowded)
         for (uint32_t line = my_j; line * 16u < cnt; line += J) asm volatile("prefetch.global.L1 [%0];" ::"l"(run + line * 16u));
     if (un.end < e0 + nel && L.live) {
         const uint32_t s0 = gseg[0];
@@ -2246,50 +2301,113 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
             *g = __uint_as_float(ent.y);
             return (ent.x >> 31) != 0u;
         }
-        const uint32_t idx = ent.x;
-        bool sent = idx >= e0 && idx - e0 < nel;                    // (an entry outside its tile is never written by the dense pass)
-        float gv = 0.0f;
-        if (sent) {
-            UnitLite u = un;
-            if (idx >= un.end) {                      // a later segment of the tile: look its unit up
-                if (idx >= later.end) {               // (a lane's entries come in rising order: the last one looked up serves until its end)
-                    uint32_t seg = gseg[(idx - e0) >> 7];
-                    while (seg + 1 < (uint32_t)P.nseg && idx >= P.seg_off[seg + 1]) ++seg;
-                    later = unit_lite(P, L, seg);
-                }
-                u = later;
-            }
-            const float val = __uint_as_float(ent.y);
-            const uint32_t key = RANDK ? ~philox_word(P, my_r, idx, 1u) : topk_key(val);
-            sent = key > u.tau || (key == u.tau && idx <= u.tie_max);
-            if (sent) {
-                if (P.qz == QS_NONE) {
-                    gv = val;
-                } else if (P.qz == QS_MINMAX) {
-                    gv = minmax_value(u.lo, u.norm, P.s, minmax_level(val, u.lo, u.norm, P.s, philox_word(P, my_r, idx, 0u)));
-                } else {
-                    int level = 1;
-                    if (!qz_is_sign(P.qz)) level = qsgd_level(val, u.norm, P.s, philox_word(P, my_r, idx, 0u));
-                    sent = level != 0;                             // (level 0: kept, not sent)
-                    if (sent) {                                    // the value as coord_value forms it
-                        if (qz_is_sign(P.qz)) {
-                            gv = u.norm / (float)u.k;
-                        } else {
-                            gv = (u.norm * (float)level) / (float)P.s;
-                            if (P.qz == QS_QSGD_SCALED) gv = gv * u.c;
-                        }
-                        if (val < 0.0f) gv = -gv;
-                    }
-                }
-            }
-        }
-        *pos = sent ? idx - e0 : 0u;
-        *g = gv;
-        // the worker's memory at a sent coordinate (quantizers that have no quantize stage of their own)
-        if (mem_update && sent && first) P.mem[(size_t)my_r * P.d + idx] = __uint_as_float(ent.y) - gv;
-        *home = make_uint2(*pos | (sent ? 0x80000000u : 0u), __float_as_uint(gv));
+        const bool sent = first_look<RANDK>(P, my_r, un, later, gseg, e0, nel, ent, mem_update, pos, g);
+        *home = make_uint2(*pos | (sent ? 0x80000000u : 0u), __float_as_uint(*g));
         return sent;
     };
+    // A crowded tile (small tensors that every worker sends whole, so that most coordinates have
+    // several senders): one walk, worker after worker in their order with all lanes on one
+    // worker's entries, the sums formed in the tile's own buffer.  A worker sends a coordinate at
+    // most once, so its lanes never meet at one sum; a coordinate with one sender gets 0 + g as
+    // everywhere else; x itself is read again from global memory, which still holds the round's
+    // model; a sum of zero leaves x as it is, as x - 0 / R would.  No bitmaps of senders: with all
+    // workers at the same coordinates their words would be fought over.
+    if (crowded) {
+        // x again at the end: asked for now, so that it waits in the L1 by then
+        for (uint32_t line = lane; line * 32u < nel; line += 32) asm volatile("prefetch.global.L1 [%0];" ::"l"(P.x + e0 + line * 32u));
+        for (uint32_t j = lane; j < (uint32_t)STILE; j += 32) xs[j] = 0.0f;
+        __syncwarp();
+        // The runs come through a ring of RING_N pieces of RING_E entries in the slot's candidate
+        // buffer (free: a crowded tile is never staged), filled by asynchronous 16-byte copies that
+        // run RING_N - 1 pieces ahead of the walk and across the change from one worker to the next:
+        // a load from the L2 or from HBM takes microseconds while the broadcast's stores fill the
+        // memory system, and one load per 32 entries would wait that long every time.
+        constexpr uint32_t RING_E = 64, RING_N = 6;
+        static_assert(RING_E * RING_N <= (uint32_t)CB, "the ring lives in the candidate buffer");
+        const bool ring = cb != nullptr && !staged && (P.cap & 1ull) == 0ull && (reinterpret_cast<uintptr_t>(P.stage) & 15u) == 0u;
+        uint32_t iw = 0, ic = 0, islot = 0;            // filling: worker slot, piece of its run, ring place
+        auto fill = [&]() {
+            uint32_t cnt_i = 0;
+            while (iw < (uint32_t)L.nact && ic * RING_E >= (cnt_i = __shfl_sync(0xffffffffu, cnt, iw))) { ++iw; ic = 0; }
+            if (iw < (uint32_t)L.nact) {
+                const uint32_t r_i = __shfl_sync(0xffffffffu, my_r, iw);
+                const uint32_t at = ic * RING_E + 2u * (uint32_t)lane;        // this lane's pair of entries (rows are even: a pair never crosses a row's end)
+                const uint2* src = P.stage + (size_t)r_i * P.cap + (size_t)tile * STILE + at;
+                if (at < cnt_i)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(cb + (islot % RING_N) * RING_E + 2u * (uint32_t)lane)), "l"(src) : "memory");
+                ++ic;
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");     // (an empty group keeps the count in step)
+            ++islot;
+        };
+        if (ring)
+            for (uint32_t q = 0; q + 1 < RING_N; ++q) fill();
+        uint32_t cslot = 0;
+        for (int w = 0; w < L.nact; ++w) {
+            const uint32_t cnt_w = __shfl_sync(0xffffffffu, cnt, w);
+            const uint32_t r_w = __shfl_sync(0xffffffffu, my_r, w);
+            // the unit of the tile's first segment, from the lane that holds this worker's
+            UnitLite uw;
+            uw.tau = __shfl_sync(0xffffffffu, un.tau, w); uw.tie_max = __shfl_sync(0xffffffffu, un.tie_max, w);
+            uw.k = __shfl_sync(0xffffffffu, un.k, w); uw.end = __shfl_sync(0xffffffffu, un.end, w);
+            uw.norm = __shfl_sync(0xffffffffu, un.norm, w); uw.c = __shfl_sync(0xffffffffu, un.c, w);
+            uw.lo = __shfl_sync(0xffffffffu, un.lo, w);
+            UnitLite lw = {0u, 0u, 0u, 0u, 0.0f, 0.0f, 0.0f};
+            if (ring) {
+                for (uint32_t c0 = 0; c0 < cnt_w; c0 += RING_E) {
+                    fill();
+                    asm volatile("cp.async.wait_group %0;" ::"n"(RING_N - 1) : "memory");
+                    __syncwarp();                     // every lane's part of the piece has landed
+                    const uint2* piece = cb + (cslot % RING_N) * RING_E;
+#pragma unroll
+                    for (uint32_t h = 0; h < RING_E; h += 32) {
+                        const uint32_t i = c0 + h + (uint32_t)lane;
+                        uint32_t pos = 0;
+                        float g = 0.0f;
+                        if (i < cnt_w && first_look<RANDK>(P, r_w, uw, lw, gseg, e0, nel, piece[h + lane], mem_update, &pos, &g))
+                            xs[pos] = xs[pos] + g;
+                    }
+                    __syncwarp();                     // the piece may be filled again
+                    ++cslot;
+                }
+            } else {
+                const uint2* run_w = staged ? cb + __shfl_sync(0xffffffffu, pbefore, w) : P.stage + (size_t)r_w * P.cap + (size_t)tile * STILE;
+                uint2 nxt = make_uint2(0u, 0u);
+                if ((uint32_t)lane < cnt_w) nxt = run_w[lane];
+                for (uint32_t i = lane; i < cnt_w; i += 32) {
+                    const uint2 ent = nxt;
+                    if (i + 32u < cnt_w) nxt = run_w[i + 32u];
+                    if (!staged && (lane & 15) == 0 && i + AHEAD * 16u < cnt_w) asm volatile("prefetch.global.L1 [%0];" ::"l"(run_w + i + AHEAD * 16u));
+                    uint32_t pos = 0;
+                    float g = 0.0f;
+                    if (first_look<RANDK>(P, r_w, uw, lw, gseg, e0, nel, ent, mem_update, &pos, &g)) xs[pos] = xs[pos] + g;
+                }
+            }
+            __syncwarp();
+        }
+        if (ring) asm volatile("cp.async.wait_group 0;" ::: "memory");
+        for (uint32_t m0 = 0; m0 < (uint32_t)(STILE / 32); m0 += 4) {
+            float xv[4];
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q) {
+                const uint32_t j = (m0 + q) * 32u + (uint32_t)lane;
+                xv[q] = j < nel ? P.x[e0 + j] : 0.0f;
+            }
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q) {
+                const uint32_t j = (m0 + q) * 32u + (uint32_t)lane;
+                bool ch = false;
+                if (j < nel) {
+                    const float sum = xs[j];
+                    ch = sum != 0.0f;
+                    xs[j] = ch ? xv[q] - sum / rdiv : xv[q];
+                }
+                const uint32_t bits = __ballot_sync(0xffffffffu, ch);
+                if (lane == 0) W.bm1[m0 + q] = bits;
+            }
+        }
+        __syncwarp();
+    } else {
     // senders per coordinate
     for (uint32_t i = my_j; i < cnt; i += J) {
         uint32_t pos = 0;
@@ -2330,6 +2448,8 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
             const uint2* run_w = staged ? cb + pb_w : P.stage + (size_t)r_w * P.cap + (size_t)tile * STILE;
             for (uint32_t i0 = 0; i0 < cnt_w; i0 += 128u) {
                 uint2 e[4];
+                if (!staged && i0 + 256u + (uint32_t)lane * 16u < cnt_w)            // the batch after the next, by lines
+                    asm volatile("prefetch.global.L1 [%0];" ::"l"(run_w + i0 + 256u + (uint32_t)lane * 16u));
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const uint32_t i = i0 + (uint32_t)q * 32u + (uint32_t)lane;
@@ -2402,6 +2522,7 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
             if (lane == 0) W.nm = 0u;
             __syncwarp();
         }
+    }
     }
     }
     __syncwarp();                                     // every lane is done with the tile and the bitmaps
@@ -2519,6 +2640,7 @@ __device__ void stage_update_broadcast(const Plan& P, const Active& act, BcBlock
                 if (lane == 0) {
                     S.tile = tile;
                     S.staged = staged ? 1u : 0u;
+                    S.crowded = ptotal >= CROWDED_MIN ? 1u : 0u;
                     mbar_expect(&B.full[s], nel * 4u + (staged ? ptotal * 8u : 0u));
                     bulk_load(S.xs, P.x + e0, nel * 4u, &B.full[s]);
                 }
@@ -2581,7 +2703,7 @@ __device__ void stage_update_broadcast(const Plan& P, const Active& act, BcBlock
             if (!one_seg) un = unit_lite(P, L, S.gseg[0]);
             const uint32_t cnt = L.live ? S.cnt[L.my_w] : 0u;
             const bool whole = apply_tile<RANDK>(P, L, lane, tile, cnt, S.staged != 0u, S.cb, L.live ? S.pbefore[L.my_w] : 0u, S.gseg, S.xs,
-                                                 W, un, mem_update, true);
+                                                 W, un, mem_update, true, S.crowded != 0u);
             if (lane == 0) S.whole = whole ? 1u : 0u;
             fence_async_smem();                       // the tile as updated must be what the bulk stores read
             __syncwarp();
@@ -2619,7 +2741,7 @@ __device__ void stage_update_broadcast_plain(const Plan& P, const Active& act, B
         if (lane < STILE / GROUP) gseg[lane] = one_seg ? 0u : P.grp_seg[(size_t)tile * (STILE / GROUP) + lane];
         __syncwarp();
         if (!one_seg) un = unit_lite(P, L, gseg[0]);
-        apply_tile<RANDK>(P, L, lane, tile, tile_count(P, L, tile), false, nullptr, 0u, gseg, xs, W, un, mem_update, false);
+        apply_tile<RANDK>(P, L, lane, tile, tile_count(P, L, tile), false, nullptr, 0u, gseg, xs, W, un, mem_update, false, false);
         __syncwarp();
         for (int w = 0; w < act.n; ++w)
             for (uint32_t i = lane; i < nel; i += 32) {
