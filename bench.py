@@ -325,9 +325,9 @@ def time_large(torch, B, dev, peak, R_, d, k, s, sparsifier, drift_rows, x, xw, 
             "fallback_worker_rounds": st["fallback_worker_rounds"], "steps": steps, "warmup": warmup}
 
 
-def time_config3(torch, B, dev, peak):
-    """R = 16, d = 2^26, Gaussian drift N(0, 1e-3), Rand_k k = 1% by keyed-hash rank, QSGD s = 4."""
-    R3, d = 16, 1 << 26
+def time_config3(torch, B, dev, peak, shrink=1, steps=5, warmup=4):
+    """R = 16, d = 2^26 (divided by shrink), Gaussian drift N(0, 1e-3), Rand_k k = 1% by keyed-hash rank, QSGD s = 4."""
+    R3, d = 16, (1 << 26) // shrink
     gen = torch.Generator(device=dev)
     gen.manual_seed(3)
     x = torch.from_numpy(I.model_init(d, seed=1)).to(dev)
@@ -339,14 +339,15 @@ def time_config3(torch, B, dev, peak):
         for r in range(R3):
             e1.normal_(0.0, 1e-3, generator=gen)
             xw[r].add_(e1)
-    out = time_large(torch, B, dev, peak, R3, d, I.k_from_ratio(d, 1, 100), 4, B.QS_RANDK, drift, x, xw, mem, seed=3)
-    out["workload"] = "Rand_k round: R=16, d=2^26, drift N(0,1e-3), Rand_k k=1% by keyed-hash rank, QSGD s=4"
+    out = time_large(torch, B, dev, peak, R3, d, I.k_from_ratio(d, 1, 100), 4, B.QS_RANDK, drift, x, xw, mem, seed=3,
+                     steps=steps, warmup=warmup)
+    out["workload"] = "Rand_k round: R=16, d=%d, drift N(0,1e-3), Rand_k k=1%% by keyed-hash rank, QSGD s=4" % d
     del x, xw, mem, e1
     torch.cuda.empty_cache()
     return out
 
 
-def time_config5(torch, B, dev, peak, steps=4, warmup=3):
+def time_config5(torch, B, dev, peak, steps=4, warmup=20):
     """R = 4, d = 2^28, drift N(0, 1e-3) with 0.1% outliers x100, Top_k ratio in {1e-4, 1e-3, 1e-2, 1e-1} x QSGD
     s in {2, 16, 256}: the twelve points."""
     R5, d = 4, 1 << 28
@@ -489,6 +490,18 @@ def run_reference(args):
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
+
+
+def run_config3(args):
+    """The Rand_k round of config 3 alone (R = 16, d = 2^26 / --shrink): one JSON line."""
+    import torch
+    from paper_1906_02367_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peak, peak_src = peak_hbm()
+    out = time_config3(torch, B, dev, peak, shrink=args.shrink, steps=max(2, min(args.steps, 20)), warmup=max(3, min(args.warmup, 6)))
+    out["peak_source"] = peak_src
+    print(json.dumps({"metric": "config3_randk_round", "unit": "ms", **out}))
 
 
 def run_sweep5(args):
@@ -772,7 +785,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor", "paper_table", "async", "step", "sharded"])
+    ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor", "paper_table", "async", "step", "sharded", "config3"])
     ap.add_argument("--shrink", type=int, default=1, help="divide every tensor size (profiling on a small case)")
     ap.add_argument("--sweep5", action="store_true", help="run the d = 2^28 ratio x s sweep instead of the headline workload")
     ap.add_argument("--no-e2e", action="store_true")
@@ -796,6 +809,8 @@ def main():
         run_step(args)
     elif args.variant == "sharded":
         run_sharded(args)
+    elif args.variant == "config3":
+        run_config3(args)
     else:
         run_ours(args)
 
