@@ -415,7 +415,8 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
                 c = ss[seg + 1] - start;
                 if (c < P.kseg[seg]) atomicOr(sh_flag, 1u << r);
                 atomicMax(sh_flag + 1, c);
-                if (c > (uint32_t)BT && c <= P.unit_cap) atomicAdd(sh_flag + 2, 1u);   // lists that would keep a block busy for a while
+                // lists that would keep a block busy for a while: weight 2, or 1 up to half the cap
+                if (c > (uint32_t)BT && c <= P.unit_cap) atomicAdd(sh_flag + 2, c > P.unit_cap / 2u ? 2u : 1u);
             }
         }
         uint32_t total;
@@ -431,11 +432,11 @@ __device__ uint32_t build_table(const Plan& P, const Active& act, uint32_t* t_st
     tab->fast = (P.nseg == 1 || qz_sends_all(P.qz)) && (longest + CHUNK - 1) / CHUNK <= 1024u;
     // Which units one block selects from on its own (block barriers only), and which take the
     // grid-wide radix levels: every list up to the cap when there is a block for each list that
-    // would keep one busy for a while (lists are dealt largest first); otherwise only the lists of
-    // at most one candidate per thread.
+    // would keep one busy for a while, two lists of up to half the cap counting as one (lists are
+    // dealt largest first); otherwise only the lists of at most one candidate per thread.
     uint32_t short_c = 0;
     if (P.unit_cap) {
-        const bool all = sh_flag[2] <= gridDim.x;
+        const bool all = sh_flag[2] <= 2u * gridDim.x;
         short_c = all ? P.unit_cap : (P.unit_cap < (uint32_t)BT ? P.unit_cap : (uint32_t)BT);
     }
     tab->short_c = short_c;
