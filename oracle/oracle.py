@@ -34,6 +34,7 @@ def lib():
         _lib.qso_beta_qsgd.restype = C.c_double
         _lib.qso_beta_qsgd.argtypes = [C.c_int64, C.c_int]
         _lib.qso_wire_words.restype = C.c_int64
+        _lib.qso_gap_words.restype = C.c_int64
     return _lib
 
 
@@ -181,6 +182,32 @@ def unpack_accumulate(plan, x, wire, mask=None):
     return lib().qso_unpack_accumulate(*plan._head(), C.c_int(plan.quantizer), _f32(x),
                                        _p(wire, C.c_uint32), C.c_int64(wire.shape[1]),
                                        _p(m, C.c_uint8))
+
+
+def gap_words(plan):
+    return int(lib().qso_gap_words(*plan._head(), C.c_int(plan.quantizer)))
+
+
+def recode_gaps(plan, wire, mask=None):
+    """Plain records -> gap-coded records (first index + gaps in fields of the widest gap's length)."""
+    m = _mask(mask)
+    wire = np.ascontiguousarray(wire, dtype=np.uint32)
+    stride = gap_words(plan)
+    out = np.zeros((plan.R, stride), dtype=np.uint32)
+    bits = np.zeros(plan.R, dtype=np.int64)
+    rc = lib().qso_recode_gaps(*plan._head(), C.c_int(plan.quantizer), _p(wire, C.c_uint32), C.c_int64(wire.shape[1]),
+                               _p(m, C.c_uint8), _p(out, C.c_uint32), C.c_int64(stride), _p(bits, C.c_int64))
+    return {"rc": rc, "packed": out, "bits": bits, "stride": stride}
+
+
+def decode_gaps(plan, packed, mask=None):
+    m = _mask(mask)
+    packed = np.ascontiguousarray(packed, dtype=np.uint32)
+    stride = plan.wire_words()
+    wire = np.zeros((plan.R, stride), dtype=np.uint32)
+    rc = lib().qso_decode_gaps(*plan._head(), C.c_int(plan.quantizer), _p(packed, C.c_uint32), C.c_int64(packed.shape[1]),
+                               _p(m, C.c_uint8), _p(wire, C.c_uint32), C.c_int64(stride))
+    return {"rc": rc, "wire": wire}
 
 
 def broadcast(plan, x, xw, anchors=None, mask=None):

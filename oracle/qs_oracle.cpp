@@ -71,6 +71,10 @@
 //             bits, and for QSGD n fields (level-1) of b_lvl = max(1,
 //             ceil(log2 s)) bits.  QSGD drops level-0 entries; Sign sends all
 //             k.  bits = sum_seg 64 + n (b_idx + 1 + b_lvl).
+//   [gap coding] the paper counts transmitted bits and leaves the coding of the k
+//             indices open: a second form of the record sends the first index of a
+//             segment and then the gaps between successive indices in fields as
+//             wide as the segment's largest gap needs (format above recode_gaps_row).
 //   [philox]  key = (seed_lo, seed_hi); counter = (element >> 2, worker,
 //             round_lo, (round_hi << 8) | stream); word = out[element & 3];
 //             element is the global coordinate index.
@@ -81,7 +85,9 @@
 // (level = s, g = u, m = 0); unbiasedness and the second-moment bound of
 // Definition 1; the closed form of Lemma 3's proof for m = 1; inclusion
 // probability k/d of Rand_k; an independent Python bit reader for the wire;
-// the memory-maintenance identity of Lemma 6; the async divisor R.
+// the memory-maintenance identity of Lemma 6; the async divisor R; for the
+// gap-coded record a hand-worked example, an independent Python reader, the round
+// trip and the saving on uniformly spread indices.
 //
 // Build: g++ -O2 -ffp-contract=off -shared -fPIC (see oracle/build.py).
 
@@ -487,6 +493,88 @@ void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
     }
 }
 
+// ---------------------------------------------------------------- gap-coded record
+// The paper counts what the workers transmit in bits (Section 5, the x-axes of the figures) and
+// leaves the coding of the k indices open.  [gap coding] A second form of the record sends, per
+// segment, the first index and then the gaps between successive indices (ascending, so every gap
+// g_j = i_j - i_(j-1) - 1 >= 0) in fields of w bits, w the bit length of the largest gap of that
+// segment (0 when all indices are consecutive or n <= 1).  Row of one worker:
+//   directory: nseg entries of four words (n, norm bits, w, first index); the min/max quantizer
+//              keeps (min, max) in the first two, n = k;
+//   per segment: n - 1 gap fields of w bits, LSB first, padded to a word; then the streams that
+//              follow the indices in the plain record (signs, levels or values), word for word.
+// bits per segment: 64 + 6 + [n >= 1] (b_idx + (n - 1) w) + n (entry bits - b_idx).
+int bit_length(uint32_t v) { int b = 0; while (v) { ++b; v >>= 1; } return b; }
+
+int64_t gap_words(const Plan& P) {
+    int64_t w = 4 * (int64_t)P.nseg;
+    const int bl = bits_lvl(P.s);
+    for (int g = 0; g < P.nseg; ++g) {
+        const int bi = bits_idx(P.off[g + 1] - P.off[g]);
+        const int64_t k = P.kseg[g];
+        w += words_for(k - 1, bi) + payload_words(k, bi, bl, P.quantizer) - words_for(k, bi);
+    }
+    return w;
+}
+
+// plain record -> gap-coded record; returns its size in bits
+int64_t recode_gaps_row(const Plan& P, const uint32_t* wire, uint32_t* out) {
+    const int bl = bits_lvl(P.s);
+    const int minmax = P.quantizer == QZ_MINMAX;
+    int64_t in_at = 2 * (int64_t)P.nseg, out_at = 4 * (int64_t)P.nseg, bits = 0;
+    for (int g = 0; g < P.nseg; ++g) {
+        const int64_t n_el = P.off[g + 1] - P.off[g];
+        const int64_t n = minmax ? P.kseg[g] : (int64_t)wire[2 * g];
+        const int bi = bits_idx(n_el);
+        const uint32_t* w_idx = wire + in_at;
+        std::vector<uint32_t> idx(n);
+        for (int64_t j = 0; j < n; ++j) idx[j] = get_bits(w_idx, j * bi, bi);
+        uint32_t widest = 0;
+        for (int64_t j = 1; j < n; ++j) {
+            const uint32_t gap = idx[j] - idx[j - 1] - 1u;
+            if (gap > widest) widest = gap;
+        }
+        const int w = bit_length(widest);
+        out[4 * g] = wire[2 * g];
+        out[4 * g + 1] = wire[2 * g + 1];
+        out[4 * g + 2] = (uint32_t)w;
+        out[4 * g + 3] = n ? idx[0] : 0u;
+        for (int64_t j = 1; j < n; ++j) put_bits(out + out_at, (j - 1) * w, w, idx[j] - idx[j - 1] - 1u);
+        const int64_t gw = n ? words_for(n - 1, w) : 0, iw = words_for(n, bi);
+        const int64_t rest = payload_words(n, bi, bl, P.quantizer) - iw;
+        for (int64_t q = 0; q < rest; ++q) out[out_at + gw + q] = wire[in_at + iw + q];
+        bits += 64 + 6 + (n ? bi + (n - 1) * w : 0) + n * (entry_bits(bi, bl, P.quantizer) - bi);
+        in_at += iw + rest;
+        out_at += gw + rest;
+    }
+    return bits;
+}
+
+// gap-coded record -> plain record (the words of `wire` must be zero on entry)
+void decode_gaps_row(const Plan& P, const uint32_t* packed, uint32_t* wire) {
+    const int bl = bits_lvl(P.s);
+    const int minmax = P.quantizer == QZ_MINMAX;
+    int64_t in_at = 4 * (int64_t)P.nseg, out_at = 2 * (int64_t)P.nseg;
+    for (int g = 0; g < P.nseg; ++g) {
+        const int64_t n_el = P.off[g + 1] - P.off[g];
+        const int64_t n = minmax ? P.kseg[g] : (int64_t)packed[4 * g];
+        const int bi = bits_idx(n_el);
+        const int w = (int)packed[4 * g + 2];
+        wire[2 * g] = packed[4 * g];
+        wire[2 * g + 1] = packed[4 * g + 1];
+        uint32_t at = packed[4 * g + 3];
+        for (int64_t j = 0; j < n; ++j) {
+            if (j) at = at + get_bits(packed + in_at, (j - 1) * w, w) + 1u;
+            put_bits(wire + out_at, j * bi, bi, at);
+        }
+        const int64_t gw = n ? words_for(n - 1, w) : 0, iw = words_for(n, bi);
+        const int64_t rest = payload_words(n, bi, bl, P.quantizer) - iw;
+        for (int64_t q = 0; q < rest; ++q) wire[out_at + iw + q] = packed[in_at + gw + q];
+        in_at += gw + rest;
+        out_at += iw + rest;
+    }
+}
+
 bool valid_plan(const Plan& P) {
     if (P.R < 1 || P.d < 1 || P.nseg < 1 || P.s < 1 || P.s > 65535) return false;
     if (P.quantizer == QZ_MINMAX && P.s < 2) return false;
@@ -625,6 +713,41 @@ int qso_unpack_accumulate(int R, int64_t d, int nseg, const int64_t* off, const 
         master_add_record(P, wire + (int64_t)r * stride_words, acc.data());
     }
     for (int64_t i = 0; i < d; ++i) x[i] = x[i] - acc[i] / (float)R;
+    return ERR_OK;
+}
+
+int64_t qso_gap_words(int R, int64_t d, int nseg, const int64_t* off, const int64_t* kseg, int s,
+                      int quantizer) {
+    Plan P = {R, d, nseg, off, kseg, s, SP_TOPK, quantizer, 0};
+    return valid_plan(P) ? gap_words(P) : (int64_t)ERR_ARG;
+}
+
+// Plain records -> gap-coded records for the workers in mask; rows of `out` must be zero.
+int qso_recode_gaps(int R, int64_t d, int nseg, const int64_t* off, const int64_t* kseg, int s,
+                    int quantizer, const uint32_t* wire, int64_t stride_words, const uint8_t* mask,
+                    uint32_t* out, int64_t out_stride, int64_t* bits_out) {
+    Plan P = {R, d, nseg, off, kseg, s, SP_TOPK, quantizer, 0};
+    if (!valid_plan(P)) return ERR_ARG;
+    if (stride_words < wire_words(P) || out_stride < gap_words(P)) return ERR_CAPACITY;
+    for (int r = 0; r < R; ++r) {
+        if (mask && !mask[r]) continue;
+        const int64_t bits = recode_gaps_row(P, wire + (int64_t)r * stride_words, out + (int64_t)r * out_stride);
+        if (bits_out) bits_out[r] = bits;
+    }
+    return ERR_OK;
+}
+
+// Gap-coded records -> plain records; rows of `wire` must be zero.
+int qso_decode_gaps(int R, int64_t d, int nseg, const int64_t* off, const int64_t* kseg, int s,
+                    int quantizer, const uint32_t* packed, int64_t packed_stride, const uint8_t* mask,
+                    uint32_t* wire, int64_t stride_words) {
+    Plan P = {R, d, nseg, off, kseg, s, SP_TOPK, quantizer, 0};
+    if (!valid_plan(P)) return ERR_ARG;
+    if (stride_words < wire_words(P) || packed_stride < gap_words(P)) return ERR_CAPACITY;
+    for (int r = 0; r < R; ++r) {
+        if (mask && !mask[r]) continue;
+        decode_gaps_row(P, packed + (int64_t)r * packed_stride, wire + (int64_t)r * stride_words);
+    }
     return ERR_OK;
 }
 
