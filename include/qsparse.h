@@ -266,6 +266,35 @@ int64_t qs_record_bits(const qs_ctx* ctx, const int64_t* n);
 /* Sum of k_seg. */
 int64_t qs_total_k(const qs_ctx* ctx);
 
+/*
+ * Gap-coded records.  The paper measures what the workers send in bits (Section 5, the x-axes
+ * of its figures) and leaves the coding of the k indices open.  qs_recode_gaps turns the
+ * records of qs_pack / qs_sync_round into a second form in which a segment's ascending indices
+ * travel as the first index and the gaps i_j - i_(j-1) - 1, in fields of w bits, w the bit
+ * length of the segment's largest gap (0 when n <= 1 or all indices are consecutive);
+ * qs_decode_gaps turns them back, word for word, for qs_unpack_accumulate.  Row of a worker:
+ *   directory: nseg entries of four words (n, norm bits, w, first index) (the min/max
+ *              quantizer keeps (min, max) in the first two, n = k);
+ *   per segment: n - 1 gap fields of w bits, LSB first, padded to a word; then the streams
+ *              that follow the indices in the plain record (signs, levels or values), unchanged.
+ * Words after a record, up to qs_gap_words, are zero.
+ *   wire / stride_words     device, rows in the format of qs_pack (stride >= qs_wire_words)
+ *   packed / packed_stride  device, rows of packed_stride >= qs_gap_words(ctx) words
+ *   worker_mask             host, one byte per worker of the job, or NULL for all; rows of
+ *                           workers outside it are neither read nor written
+ *   bits_out                device, one int64 per worker, or NULL: exact size in bits,
+ *                           sum over segments of 64 + 6 + [n >= 1] (b_idx + (n - 1) w) + n (entry bits - b_idx)
+ * Both calls are asynchronous on the context's stream, allocate nothing and keep no state; a
+ * count above k_seg, a width above b_idx or a first index outside the segment in the input is
+ * clipped (the words read and written stay inside the rows).  QS_CAPACITY (nothing written) when
+ * a stride is too small.
+ */
+int64_t qs_gap_words(const qs_ctx* ctx);
+int qs_recode_gaps(qs_ctx* ctx, const uint32_t* wire, int64_t stride_words, const uint8_t* worker_mask,
+                   uint32_t* packed, int64_t packed_stride, int64_t* bits_out);
+int qs_decode_gaps(qs_ctx* ctx, const uint32_t* packed, int64_t packed_stride, const uint8_t* worker_mask,
+                   uint32_t* wire, int64_t stride_words);
+
 /* Synchronises the stream and returns the first error recorded on the device since the
  * last call (QS_OK if none), clearing it.  After a device-side error (QS_NONFINITE,
  * QS_TIMEOUT, QS_STATE) the round that hit it is void: its outputs are undefined, and this call

@@ -26,7 +26,7 @@ EXPORTS = [
     "qs_unpack_accumulate", "qs_broadcast", "qs_sync_round", "qs_export_selection", "qs_wire_words",
     "qs_record_bits", "qs_total_k", "qs_sync_status", "qs_last_error", "qs_get_round", "qs_set_round",
     "qs_get_stats", "qs_enable_phase_timing", "qs_get_phase_timing", "qs_get_stage_trace", "qs_unpack_accumulate_static",
-    "qs_destroy",
+    "qs_gap_words", "qs_recode_gaps", "qs_decode_gaps", "qs_destroy",
 ]
 
 _lib = None
@@ -64,6 +64,10 @@ def lib():
         L.qs_record_bits.restype = i64
         L.qs_total_k.argtypes = [vp]
         L.qs_total_k.restype = i64
+        L.qs_gap_words.argtypes = [vp]
+        L.qs_gap_words.restype = i64
+        L.qs_recode_gaps.argtypes = [vp, vp, i64, vp, vp, i64, vp]
+        L.qs_decode_gaps.argtypes = [vp, vp, i64, vp, vp, i64]
         L.qs_sync_status.argtypes = [vp]
         L.qs_last_error.argtypes = [vp]
         L.qs_last_error.restype = C.c_char_p
@@ -176,6 +180,18 @@ class Context:
     def unpack_accumulate(self, wire, mask=None):
         m, mp = _mask(mask, self.R_total)        # the records of the whole job
         self._check(lib().qs_unpack_accumulate(self._h, _ptr(wire), int(wire.shape[1]), mp))
+
+    def gap_words(self):
+        return int(lib().qs_gap_words(self._h))
+
+    def recode_gaps(self, wire, packed, mask=None, bits_out=None):
+        m, mp = _mask(mask, self.R_total)
+        self._check(lib().qs_recode_gaps(self._h, _ptr(wire), int(wire.shape[1]), mp, _ptr(packed), int(packed.shape[1]),
+                                         _ptr(bits_out)))
+
+    def decode_gaps(self, packed, wire, mask=None):
+        m, mp = _mask(mask, self.R_total)
+        self._check(lib().qs_decode_gaps(self._h, _ptr(packed), int(packed.shape[1]), mp, _ptr(wire), int(wire.shape[1])))
 
     def broadcast(self, mask=None):
         m, mp = _mask(mask, self.R)

@@ -18,7 +18,8 @@ struct qs_ctx {
     bool bound, aligned, compressed, use_tma;
     Active last;                       // workers of the last compression
     std::vector<int64_t> off, kseg;    // host copies of the segment table
-    int64_t wire_words;
+    int64_t wire_words, gap_words;
+    uint32_t longest_k, most_words, row_chunks;   // of the gap-coded record: largest k_seg, most stream words of a segment, chunk sums per worker
     uint64_t round;
     int64_t launches, rounds;
     std::string err;
@@ -208,6 +209,21 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.K = h_kp[nseg];
     P.nfb = (uint32_t)h_fb.size();
     c->wire_words = words;
+    {
+        int64_t gw = 4 * (int64_t)nseg;
+        uint64_t longest = 0, most = 0;
+        for (int g = 0; g < nseg; ++g) {
+            const uint32_t k = (uint32_t)kseg[g];
+            const uint64_t all = streams_words(k, h_bi[g], (uint32_t)P.bl, P.qz);
+            gw += (int64_t)words_for(k - 1, h_bi[g]) + (int64_t)all - (int64_t)words_for(k, h_bi[g]);
+            longest = std::max<uint64_t>(longest, k);
+            most = std::max<uint64_t>(most, all);
+        }
+        c->gap_words = gw;
+        c->longest_k = (uint32_t)longest;
+        c->most_words = (uint32_t)most;
+        c->row_chunks = (uint32_t)(P.K / gap_chunk()) + (uint32_t)nseg + 1u;
+    }
     if (nseg > 1) {
         h_grp.resize((size_t)P.ntile * (STILE / GROUP));     // whole tiles: the dense pass copies a tile's entries at once
         int sg = 0;
@@ -271,6 +287,8 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.guess = const_cast<uint32_t*>(g_up);
 #define AL(field, count, zero) if ((rc = dev_alloc(c, &P.field, (size_t)(count), zero)) != QS_OK) return rc
     AL(wary, P.U, true);
+    AL(gap_unit, (size_t)6 * MAX_R * nseg, true);
+    AL(gap_csum, (size_t)MAX_R * c->row_chunks, true);
     AL(stage, (size_t)R * P.cap, false);
     AL(tile_cnt, (size_t)R * P.nblk * BLK_TILES, true);
     AL(blk_count, (size_t)R * P.nblk, true);
@@ -580,6 +598,38 @@ int64_t qs_record_bits(const qs_ctx* c, const int64_t* n) {
         bits += 64 + n[g] * (int64_t)entry_bits((uint32_t)bi, (uint32_t)c->P.bl, c->P.qz);
     }
     return bits;
+}
+
+int64_t qs_gap_words(const qs_ctx* c) { return c ? c->gap_words : (int64_t)QS_INVALID_ARG; }
+
+int qs_recode_gaps(qs_ctx* c, const uint32_t* wire, int64_t stride_words, const uint8_t* worker_mask, uint32_t* packed,
+                   int64_t packed_stride, int64_t* bits_out) {
+    if (!c || !wire || !packed) return fail(c, QS_INVALID_ARG, "wire and packed are required");
+    if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
+    if (packed_stride < c->gap_words) return fail(c, QS_CAPACITY, "packed_stride is below qs_gap_words");
+    Active act;
+    if (!make_active_job(c, worker_mask, &act)) return QS_OK;
+    for (int i = 0; i < act.n; ++i)       // words after a record are zero
+        QS_CUDA_TRY(c, cudaMemsetAsync(packed + (size_t)act.r[i] * packed_stride, 0, (size_t)c->gap_words * 4, c->st));
+    const cudaError_t e = launch_recode_gaps(c->P, act, wire, stride_words, packed, packed_stride,
+                                             reinterpret_cast<long long*>(bits_out), c->longest_k, c->most_words, c->st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "gap-coded records");
+    return after_launch(c, 4, "gap-coded records");
+}
+
+int qs_decode_gaps(qs_ctx* c, const uint32_t* packed, int64_t packed_stride, const uint8_t* worker_mask, uint32_t* wire,
+                   int64_t stride_words) {
+    if (!c || !wire || !packed) return fail(c, QS_INVALID_ARG, "wire and packed are required");
+    if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
+    if (packed_stride < c->gap_words) return fail(c, QS_CAPACITY, "packed_stride is below qs_gap_words");
+    Active act;
+    if (!make_active_job(c, worker_mask, &act)) return QS_OK;
+    for (int i = 0; i < act.n; ++i)       // the index fields are or-ed into zeroed words
+        QS_CUDA_TRY(c, cudaMemsetAsync(wire + (size_t)act.r[i] * stride_words, 0, (size_t)c->wire_words * 4, c->st));
+    const cudaError_t e = launch_decode_gaps(c->P, act, packed, packed_stride, wire, stride_words, c->longest_k,
+                                             c->most_words, c->row_chunks, c->st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "plain records from gap-coded ones");
+    return after_launch(c, 4, "plain records from gap-coded ones");
 }
 
 int64_t qs_total_k(const qs_ctx* c) { return c ? (int64_t)c->P.K : (int64_t)QS_INVALID_ARG; }
