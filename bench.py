@@ -234,12 +234,29 @@ def run_ours(args):
         ctx.enable_phase_timing(False)
         st1 = ctx.stats()
         wire_bytes = int(bits.sum().item() + 7) // 8
+        # the last round's records once more in the gap-coded form (outside the timed region): what
+        # would travel with the indices sent as gaps, and what the two conversions cost
+        packed = torch.zeros((R, ctx.gap_words()), dtype=torch.int32, device=dev)
+        gap_bits = torch.zeros(R, dtype=torch.int64, device=dev)
+        back = torch.zeros_like(wire)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        for _ in range(2):
+            ev[0].record()
+            ctx.recode_gaps(wire, packed, None, gap_bits)
+            ev[1].record()
+            ctx.decode_gaps(packed, back)
+            ev[2].record()
+        torch.cuda.synchronize()
+        assert ctx.sync_status() == 0 and torch.equal(back, wire), "gap-coded records do not decode to the plain ones"
+        gap = {"wire_bytes_per_round": int(gap_bits.sum().item() + 7) // 8, "recode_ms": ev[0].elapsed_time(ev[1]),
+               "decode_ms": ev[1].elapsed_time(ev[2])}
+        del packed, back
         total_ms = max_over_ranks(float(sum(per_step)), dev)
         bmin = min_bytes(d, wire_bytes)
         value = aggregate_value(bmin, steps, total_ms, world)
         out = {"value": value, "ms_per_step": total_ms / steps, "ms_per_step_spread": spread(per_step),
                "pct_of_nominal_8TBps": 100.0 * value / world / NOMINAL_HBM_GBS, "pct_of_measured_copy": 100.0 * value / world / peak,
-               "min_bytes_per_round": bmin, "wire_bytes_per_round": wire_bytes, "k_total": int(kseg.sum()),
+               "min_bytes_per_round": bmin, "wire_bytes_per_round": wire_bytes, "gap_coded": gap, "k_total": int(kseg.sum()),
                "gpu_launches": st1["launches"] - st0["launches"],
                "fallback_worker_rounds": st1["fallback_worker_rounds"] - st0["fallback_worker_rounds"],
                "phases_ms_per_round": {k: v / max(1, phases["rounds"]) for k, v in phases.items() if k != "rounds"},
@@ -255,6 +272,7 @@ def run_ours(args):
         "worker_elements_per_s": world * R * d / (m["ms_per_step"] * 1e-3),
         "pct_of_nominal_8TBps": m["pct_of_nominal_8TBps"], "pct_of_measured_copy": m["pct_of_measured_copy"],
         "min_bytes_per_round": m["min_bytes_per_round"], "wire_bytes_per_round": m["wire_bytes_per_round"],
+        "gap_coded": m["gap_coded"],
         "ms_per_step_median": m["ms_per_step_spread"]["median"], "ms_per_step_spread": m["ms_per_step_spread"],
         "gpu_launches": m["gpu_launches"], "fallback_worker_rounds": m["fallback_worker_rounds"],
         "phases_ms_per_round": m["phases_ms_per_round"], "kernels_per_round": m["gpu_launches"] / max(1, args.steps),
