@@ -280,8 +280,10 @@ int64_t qs_total_k(const qs_ctx* ctx);
  * Words after a record, up to qs_gap_words, are zero.
  *   wire / stride_words     device, rows in the format of qs_pack (stride >= qs_wire_words)
  *   packed / packed_stride  device, rows of packed_stride >= qs_gap_words(ctx) words
- *   worker_mask             host, one byte per worker of the job, or NULL for all; rows of
- *                           workers outside it are neither read nor written
+ *   worker_mask             host, or NULL for all: one byte per worker of this context for
+ *                           qs_recode_gaps (the senders' side: the rows of qs_pack), one per
+ *                           worker of the job for qs_decode_gaps (the master's side, see
+ *                           qs_set_sharding); rows of workers outside it are neither read nor written
  *   bits_out                device, one int64 per worker, or NULL: exact size in bits,
  *                           sum over segments of 64 + 6 + [n >= 1] (b_idx + (n - 1) w) + n (entry bits - b_idx)
  * Both calls are asynchronous on the context's stream, allocate nothing and keep no state; a

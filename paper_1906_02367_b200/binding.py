@@ -185,7 +185,7 @@ class Context:
         return int(lib().qs_gap_words(self._h))
 
     def recode_gaps(self, wire, packed, mask=None, bits_out=None):
-        m, mp = _mask(mask, self.R_total)
+        m, mp = _mask(mask, self.R)              # this context's workers; decode_gaps takes the whole job's
         self._check(lib().qs_recode_gaps(self._h, _ptr(wire), int(wire.shape[1]), mp, _ptr(packed), int(packed.shape[1]),
                                          _ptr(bits_out)))
 

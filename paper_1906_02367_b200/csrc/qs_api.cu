@@ -608,7 +608,7 @@ int qs_recode_gaps(qs_ctx* c, const uint32_t* wire, int64_t stride_words, const 
     if (stride_words < c->wire_words) return fail(c, QS_CAPACITY, "stride_words is below qs_wire_words");
     if (packed_stride < c->gap_words) return fail(c, QS_CAPACITY, "packed_stride is below qs_gap_words");
     Active act;
-    if (!make_active_job(c, worker_mask, &act)) return QS_OK;
+    if (!make_active(c, worker_mask, &act)) return QS_OK;   // the sender's side: this context's workers
     for (int i = 0; i < act.n; ++i)       // words after a record are zero
         QS_CUDA_TRY(c, cudaMemsetAsync(packed + (size_t)act.r[i] * packed_stride, 0, (size_t)c->gap_words * 4, c->st));
     const cudaError_t e = launch_recode_gaps(c->P, act, wire, stride_words, packed, packed_stride,

@@ -4,7 +4,7 @@ The masterless form the paper mentions in Section 1: every worker's record goes 
 and each aggregates for itself.  Worker r lives on rank r // (R / G); a rank compresses and packs its
 own workers (qs_compress_feedback, qs_pack on a context that qs_set_sharding told its place in the
 job), the packed records are exchanged with ONE all-gather (the only data-path collective: a few
-tens of KB per worker), then every rank decodes the same R records in worker order
+tens of KB per worker; optionally in their gap-coded form, qs_recode_gaps / qs_decode_gaps), then every rank decodes the same R records in worker order
 (qs_unpack_accumulate), so the replicas of x stay bit-identical, and broadcasts to its own workers
 locally.  The gathered records land in this rank's memory before any kernel reads them.
 
@@ -47,7 +47,13 @@ class ShardedRound:
     """One rank's share of a job of R workers.  x is this rank's replica of the global model; xw, mem
     (and anchors) hold this rank's workers only."""
 
-    def __init__(self, R, engine, wire_local, rank=None, world=None, group=None):
+    def __init__(self, R, engine, wire_local, rank=None, world=None, group=None, packed_local=None, records=None):
+        """packed_local (R / G rows of qs_gap_words) and records (R rows of qs_wire_words) given: the
+        records travel in their gap-coded form (qs_recode_gaps before the all-gather, qs_decode_gaps
+        after it), which is what shrinks the one collective of the round."""
+        self.packed_local, self.records = packed_local, records
+        if (packed_local is None) != (records is None):
+            raise ValueError("gap-coded exchange needs both packed_local and records")
         self.group = group
         self.world = world if world is not None else (dist.get_world_size(group) if dist.is_initialized() else 1)
         self.rank = rank if rank is not None else (dist.get_rank(group) if dist.is_initialized() else 0)
@@ -63,7 +69,14 @@ class ShardedRound:
         if mine is None or mine.any():
             self.engine.compress_feedback(rnd, mine)
             self.engine.pack(self.wire_local, bits_out)
-        records = gather_records(self.wire_local, self.R, self.group)
+            if self.packed_local is not None:
+                self.engine.recode_gaps(self.wire_local, self.packed_local, mine)
+        if self.packed_local is not None:
+            packed = gather_records(self.packed_local, self.R, self.group)
+            self.engine.decode_gaps(packed, self.records, mask)
+            records = self.records
+        else:
+            records = gather_records(self.wire_local, self.R, self.group)
         self.engine.unpack_accumulate(records, mask)
         if mine is None or mine.any():
             self.engine.broadcast(mine)

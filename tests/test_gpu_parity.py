@@ -416,6 +416,20 @@ def test_sharded_contexts_reproduce_the_whole_job(sp, qz):
         for r in range(R):
             if mask is None or mask[r]:
                 assert np.array_equal(w[r], out["wire"][r]), f"record of worker {r}"
+        # the same exchange with the records gap-coded: packed by each shard, decoded from the gathered rows
+        packs = []
+        for base, count, ctx, gx, gxw, gmem, wire in shards:
+            packs.append(torch.zeros((count, ctx.gap_words()), dtype=torch.int32, device=dev))
+            mine = sharded.local_mask(mask, base, count)
+            if mine is None or mine.any():
+                ctx.recode_gaps(wire, packs[-1], mine)
+        for base, count, ctx, gx, gxw, gmem, wire in shards:
+            back = torch.zeros_like(records)
+            ctx.decode_gaps(torch.cat(packs, dim=0), back, mask)
+            b = back.cpu().numpy().view(np.uint32)
+            for r in range(R):
+                if mask is None or mask[r]:
+                    assert np.array_equal(b[r], out["wire"][r]), f"gap-coded record of worker {r}, shard at {base}"
         for base, count, ctx, gx, gxw, gmem, wire in shards:
             ctx.unpack_accumulate(records, mask)
             ctx.broadcast(sharded.local_mask(mask, base, count))

@@ -3,6 +3,8 @@ maximum of the ranks' times (gloo, world size 2)."""
 import os
 import sys
 
+import pytest
+
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -91,6 +93,20 @@ class _OracleEngine:
         for r, w in self.records.items():
             wire_local[r] = torch.from_numpy(w.view("int32"))
 
+    def recode_gaps(self, wire_local, packed_local, mask):
+        local = self.O.Plan(self.xw.shape[0], self.plan.d, s=self.plan.s, sparsifier=self.plan.sparsifier,
+                            quantizer=self.plan.quantizer, seed=self.plan.seed, offsets=self.plan.offsets, kseg=self.plan.kseg)
+        out = self.O.recode_gaps(local, wire_local.numpy().view("uint32"), mask)
+        assert out["rc"] == 0
+        for r in range(self.xw.shape[0]):
+            if mask is None or mask[r]:
+                packed_local[r] = torch.from_numpy(out["packed"][r].view("int32"))
+
+    def decode_gaps(self, packed, records, mask):
+        out = self.O.decode_gaps(self.plan, packed.numpy().view("uint32"), mask)
+        assert out["rc"] == 0
+        records.copy_(torch.from_numpy(out["wire"].view("int32")))
+
     def unpack_accumulate(self, records, mask):
         assert self.O.unpack_accumulate(self.plan, self.x, records.numpy().view("uint32"), mask) == 0
 
@@ -103,7 +119,7 @@ class _OracleEngine:
                     self.anchors[r] = self.x
 
 
-def _sharded_main(rank, world, port, out):
+def _sharded_main(rank, world, port, out, gap_coded):
     sys.path.insert(0, ROOT)
     import numpy as np
     from oracle import oracle as O
@@ -118,7 +134,9 @@ def _sharded_main(rank, world, port, out):
     eng = _OracleEngine(O, plan, x.copy(), xw[base:base + count].copy(), mem[base:base + count].copy(),
                         anchors[base:base + count].copy())
     wire_local = torch.zeros((count, plan.wire_words()), dtype=torch.int32)
-    job = sharded.ShardedRound(R, eng, wire_local)
+    gap = dict(packed_local=torch.zeros((count, O.gap_words(plan)), dtype=torch.int32),
+               records=torch.zeros((R, plan.wire_words()), dtype=torch.int32)) if gap_coded else {}
+    job = sharded.ShardedRound(R, eng, wire_local, **gap)
     masks = [None, np.array([1, 0, 0, 1], np.uint8), np.array([0, 0, 1, 1], np.uint8)]   # the last leaves rank 0 idle
     for rnd, mask in enumerate(masks):
         eng.xw += I.gaussian_drift(R, d, 8, rnd, std=1e-2)[base:base + count]
@@ -127,7 +145,8 @@ def _sharded_main(rank, world, port, out):
     dist.destroy_process_group()
 
 
-def test_sharded_round_equals_the_single_process_round():
+@pytest.mark.parametrize("gap_coded", [False, True])
+def test_sharded_round_equals_the_single_process_round(gap_coded):
     import numpy as np
     sys.path.insert(0, ROOT)
     from oracle import oracle as O
@@ -135,7 +154,7 @@ def test_sharded_round_equals_the_single_process_round():
     world, port = 2, 31500 + os.getpid() % 2000
     with mp.Manager() as m:
         out = m.dict()
-        mp.spawn(_sharded_main, args=(world, port, out), nprocs=world, join=True)
+        mp.spawn(_sharded_main, args=(world, port, out, gap_coded), nprocs=world, join=True)
         got = {r: out[r] for r in range(world)}
     R, d, k = 4, 3000, 40
     plan = O.Plan(R, d, k=k, s=16, sparsifier=O.TOPK, quantizer=O.QSGD, seed=3)
