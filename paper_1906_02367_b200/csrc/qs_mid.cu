@@ -2123,8 +2123,12 @@ __device__ void stage_dec_apply(const Plan& P, const Active& act, const uint32_t
 //   - a coordinate with one sender: x - (0 + g) / R, on the spot;
 //   - a coordinate with several senders (found with two bitmaps of the tile in shared memory):
 //     the entries are listed, and the entry of the lowest worker adds the values in increasing
-//     worker order before it updates x.  The list is bounded: positions are taken in windows of
-//     as many as fit.
+//     worker order before it updates x.  The list is bounded; when a tile has more such
+//     coordinates than it holds, the sums are formed in the tile's own buffer worker after worker
+//     and x is read again;
+//   - a crowded tile (1024 candidates or more: tensors every worker keeps whole) skips the
+//     bitmaps and is walked worker after worker from the start, its runs coming through a ring
+//     of asynchronous copies; such tiles are handed out first (Plan::tile_order).
 // Updated coordinates are also written to x in global memory.  No sender bitmaps over d, no
 // scattered reads of x, no stage for shared indices: everything the update needs is in the
 // tile's runs, and the copies never wait for the arithmetic as long as the working warps keep up.
@@ -2276,7 +2280,7 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
     const uint32_t e0 = tile * (uint32_t)STILE;
     const uint32_t nel = P.d - e0 < (uint32_t)STILE ? P.d - e0 : (uint32_t)STILE;
     const float rdiv = (float)P.rdiv;
-    const uint32_t wp = (uint32_t)(ML_CAP / (L.nact > 0 ? L.nact : 1));   // positions with several senders per window
+    const uint32_t wp = (uint32_t)(ML_CAP / (L.nact > 0 ? L.nact : 1));   // coordinates with several senders the list can take
     const uint32_t J = L.J, my_j = L.my_j, my_r = L.my_r;
     uint2* run = P.stage + (size_t)my_r * P.cap + (size_t)tile * STILE;
     // What will be read from global memory is asked for now, all of it at once (one round trip in
@@ -2494,7 +2498,7 @@ __device__ bool apply_tile(const Plan& P, const LaneMap& L, int lane, uint32_t t
             }
             __syncwarp();
             const uint32_t n = W.nm < (uint32_t)ML_CAP ? W.nm : (uint32_t)ML_CAP;
-            if (W.nm > (uint32_t)ML_CAP) set_status(P, QS_STATE);          // a window holds at most wp x nact entries
+            if (W.nm > (uint32_t)ML_CAP) set_status(P, QS_STATE);          // (at most wp x nact entries are listed)
             for (uint32_t j = lane; j < n; j += 32) {
                 const uint32_t me = W.mpos[j], pos = me & 0xffffu, slot = me >> 16;
                 bool owner = true;

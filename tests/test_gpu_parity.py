@@ -301,6 +301,28 @@ def test_colliding_workers():
         p.close()
 
 
+@pytest.mark.parametrize("R,d_tail", [(8, 5000), (32, 5000), (8, 5001), (3, 4998)])
+def test_tiles_where_every_worker_keeps_whole_tensors(R, d_tail):
+    # small tensors kept whole by every worker (the paper's k_t = min(d_t, 1000) rule): tiles with a
+    # thousand and more candidates, every coordinate with R senders, several segments inside a tile,
+    # a crowded last tile; rows aligned and not; whole rounds with masks and anchors
+    sizes = [3000, 512, 512, 1024, 700, d_tail]
+    off = I.segments_from_sizes(sizes)
+    kseg = np.array([30, 512, 512, 1000, 700, d_tail - 3 if R == 3 else 40], np.int64)
+    d = int(off[-1])
+    x, xw, mem = I.gaussian_round(R, d, seed=23)
+    anchors = np.broadcast_to(x, (R, d)).copy()
+    masks = [None, np.array([(r * 7 + 1) % 3 != 0 for r in range(R)], np.uint8), None]
+    for qz, s in ((O.SIGN_L1, 1), (O.QSGD, 4), (O.NONE, 1), (O.MINMAX, 8), (O.QSGD_SCALED, 16)):
+        for sp in (O.TOPK, O.RANDK):
+            p = Pair(R, d, s=s, sparsifier=sp, quantizer=qz, seed=8, offsets=off, kseg=kseg, x=x, xw=xw, mem=mem,
+                     anchors=anchors if qz in (O.SIGN_L1, O.QSGD) else None)
+            for rnd, m in enumerate(masks):
+                p.drift(I.gaussian_drift(R, d, 3, rnd, std=1e-2))
+                p.round_fused(rnd, m)
+            p.close()
+
+
 def test_async_rounds_with_masks_and_anchors():
     R, d, k = 4, 30000, 300
     x, xw, mem = I.gaussian_round(R, d, seed=17)
