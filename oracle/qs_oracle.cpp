@@ -73,8 +73,9 @@
 //             k.  bits = sum_seg 64 + n (b_idx + 1 + b_lvl).
 //   [gap coding] the paper counts transmitted bits and leaves the coding of the k
 //             indices open: a second form of the record sends the first index of a
-//             segment and then the gaps between successive indices in fields as
-//             wide as the segment's largest gap needs (format above recode_gaps_row).
+//             segment and then the gaps between successive indices in short fields,
+//             the few gaps too large for a field in a stream of exceptions; the width
+//             is the one that makes the record smallest (format above gap_words).
 //   [philox]  key = (seed_lo, seed_hi); counter = (element >> 2, worker,
 //             round_lo, (round_hi << 8) | stream); word = out[element & 3];
 //             element is the global coordinate index.
@@ -497,55 +498,93 @@ void master_add_record(const Plan& P, const uint32_t* wire, float* acc) {
 // The paper counts what the workers transmit in bits (Section 5, the x-axes of the figures) and
 // leaves the coding of the k indices open.  [gap coding] A second form of the record sends, per
 // segment, the first index and then the gaps between successive indices (ascending, so every gap
-// g_j = i_j - i_(j-1) - 1 >= 0) in fields of w bits, w the bit length of the largest gap of that
-// segment (0 when all indices are consecutive or n <= 1).  Row of one worker:
-//   directory: nseg entries of four words (n, norm bits, w, first index); the min/max quantizer
-//              keeps (min, max) in the first two, n = k;
-//   per segment: n - 1 gap fields of w bits, LSB first, padded to a word; then the streams that
-//              follow the indices in the plain record (signs, levels or values), word for word.
-// bits per segment: 64 + 6 + [n >= 1] (b_idx + (n - 1) w) + n (entry bits - b_idx).
+// g_j = i_j - i_(j-1) - 1 >= 0) in fields of w bits.  For w >= 1 the field value E = 2^w - 1 is an
+// escape: a gap >= E is sent as E and the gap itself follows, in order, in a stream of exceptions
+// of b_idx bits each.  w = 0 means no fields at all and needs every gap to be 0.  The sender takes
+// the w in 0 .. b_idx that makes (n - 1) w + x(w) b_idx smallest (x(w): gaps >= 2^w - 1), the
+// smallest such w on a tie; w = b_idx has no exceptions, so the code is never longer than the
+// plain one.  Row of one worker:
+//   directory: nseg entries of five words (n, norm bits, w, first index, x); the min/max
+//              quantizer keeps (min, max) in the first two, n = k.  x could be recounted from the
+//              fields; it is kept as a word so that the streams' places are known at once, and is
+//              not counted as transmitted;
+//   per segment: n - 1 gap fields of w bits, LSB first, padded to a word; x exception fields of
+//              b_idx bits, padded to a word; then the streams that follow the indices in the
+//              plain record (signs, levels or values), word for word.
+// bits per segment: 64 + 6 + [n >= 1] (b_idx + (n - 1) w + x b_idx) + n (entry bits - b_idx).
 int bit_length(uint32_t v) { int b = 0; while (v) { ++b; v >>= 1; } return b; }
 
 int64_t gap_words(const Plan& P) {
-    int64_t w = 4 * (int64_t)P.nseg;
+    int64_t w = 5 * (int64_t)P.nseg;
     const int bl = bits_lvl(P.s);
     for (int g = 0; g < P.nseg; ++g) {
         const int bi = bits_idx(P.off[g + 1] - P.off[g]);
         const int64_t k = P.kseg[g];
-        w += words_for(k - 1, bi) + payload_words(k, bi, bl, P.quantizer) - words_for(k, bi);
+        // fields and exceptions together never exceed (k - 1) b_idx bits; two streams, each padded
+        w += words_for(k - 1, bi) + 1 + payload_words(k, bi, bl, P.quantizer) - words_for(k, bi);
     }
     return w;
+}
+
+// the field width a segment's gaps are sent with, and the exceptions it leaves
+void choose_width(const std::vector<uint32_t>& gaps, int bi, int* w_out, int64_t* x_out) {
+    const int64_t m = (int64_t)gaps.size();
+    int best_w = bi;
+    int64_t best_x = 0, best_cost = m * bi;
+    for (int w = bi - 1; w >= 0; --w) {
+        int64_t x = 0;
+        bool all_zero = true;
+        for (int64_t j = 0; j < m; ++j) {
+            if (gaps[j]) all_zero = false;
+            if (w >= 1 && (uint64_t)gaps[j] >= (1ull << w) - 1ull) ++x;
+        }
+        if (w == 0 && !all_zero) continue;
+        const int64_t cost = m * w + x * bi;
+        if (cost <= best_cost) { best_cost = cost; best_w = w; best_x = x; }
+    }
+    *w_out = best_w;
+    *x_out = best_x;
 }
 
 // plain record -> gap-coded record; returns its size in bits
 int64_t recode_gaps_row(const Plan& P, const uint32_t* wire, uint32_t* out) {
     const int bl = bits_lvl(P.s);
     const int minmax = P.quantizer == QZ_MINMAX;
-    int64_t in_at = 2 * (int64_t)P.nseg, out_at = 4 * (int64_t)P.nseg, bits = 0;
+    int64_t in_at = 2 * (int64_t)P.nseg, out_at = 5 * (int64_t)P.nseg, bits = 0;
     for (int g = 0; g < P.nseg; ++g) {
         const int64_t n_el = P.off[g + 1] - P.off[g];
         const int64_t n = minmax ? P.kseg[g] : (int64_t)wire[2 * g];
         const int bi = bits_idx(n_el);
         const uint32_t* w_idx = wire + in_at;
-        std::vector<uint32_t> idx(n);
+        std::vector<uint32_t> idx(n), gaps;
         for (int64_t j = 0; j < n; ++j) idx[j] = get_bits(w_idx, j * bi, bi);
-        uint32_t widest = 0;
-        for (int64_t j = 1; j < n; ++j) {
-            const uint32_t gap = idx[j] - idx[j - 1] - 1u;
-            if (gap > widest) widest = gap;
+        for (int64_t j = 1; j < n; ++j) gaps.push_back(idx[j] - idx[j - 1] - 1u);
+        int w = 0;
+        int64_t x = 0;
+        if (n >= 2) choose_width(gaps, bi, &w, &x);
+        const uint32_t escape = w ? (uint32_t)((1ull << w) - 1ull) : 0u;
+        out[5 * g] = wire[2 * g];
+        out[5 * g + 1] = wire[2 * g + 1];
+        out[5 * g + 2] = (uint32_t)w;
+        out[5 * g + 3] = n ? idx[0] : 0u;
+        out[5 * g + 4] = (uint32_t)x;
+        const int64_t gw = n ? words_for(n - 1, w) : 0, ew = words_for(x, bi), iw = words_for(n, bi);
+        int64_t e = 0;
+        for (int64_t j = 0; j + 1 < n; ++j) {
+            if (w == 0) continue;
+            if (gaps[j] >= escape) {
+                put_bits(out + out_at, j * w, w, escape);
+                put_bits(out + out_at + gw, e * bi, bi, gaps[j]);
+                ++e;
+            } else {
+                put_bits(out + out_at, j * w, w, gaps[j]);
+            }
         }
-        const int w = bit_length(widest);
-        out[4 * g] = wire[2 * g];
-        out[4 * g + 1] = wire[2 * g + 1];
-        out[4 * g + 2] = (uint32_t)w;
-        out[4 * g + 3] = n ? idx[0] : 0u;
-        for (int64_t j = 1; j < n; ++j) put_bits(out + out_at, (j - 1) * w, w, idx[j] - idx[j - 1] - 1u);
-        const int64_t gw = n ? words_for(n - 1, w) : 0, iw = words_for(n, bi);
         const int64_t rest = payload_words(n, bi, bl, P.quantizer) - iw;
-        for (int64_t q = 0; q < rest; ++q) out[out_at + gw + q] = wire[in_at + iw + q];
-        bits += 64 + 6 + (n ? bi + (n - 1) * w : 0) + n * (entry_bits(bi, bl, P.quantizer) - bi);
+        for (int64_t q = 0; q < rest; ++q) out[out_at + gw + ew + q] = wire[in_at + iw + q];
+        bits += 64 + 6 + (n ? bi + (n - 1) * w + x * bi : 0) + n * (entry_bits(bi, bl, P.quantizer) - bi);
         in_at += iw + rest;
-        out_at += gw + rest;
+        out_at += gw + ew + rest;
     }
     return bits;
 }
@@ -554,23 +593,30 @@ int64_t recode_gaps_row(const Plan& P, const uint32_t* wire, uint32_t* out) {
 void decode_gaps_row(const Plan& P, const uint32_t* packed, uint32_t* wire) {
     const int bl = bits_lvl(P.s);
     const int minmax = P.quantizer == QZ_MINMAX;
-    int64_t in_at = 4 * (int64_t)P.nseg, out_at = 2 * (int64_t)P.nseg;
+    int64_t in_at = 5 * (int64_t)P.nseg, out_at = 2 * (int64_t)P.nseg;
     for (int g = 0; g < P.nseg; ++g) {
         const int64_t n_el = P.off[g + 1] - P.off[g];
-        const int64_t n = minmax ? P.kseg[g] : (int64_t)packed[4 * g];
+        const int64_t n = minmax ? P.kseg[g] : (int64_t)packed[5 * g];
         const int bi = bits_idx(n_el);
-        const int w = (int)packed[4 * g + 2];
-        wire[2 * g] = packed[4 * g];
-        wire[2 * g + 1] = packed[4 * g + 1];
-        uint32_t at = packed[4 * g + 3];
+        const int w = (int)packed[5 * g + 2];
+        const int64_t x = (int64_t)packed[5 * g + 4];
+        const uint32_t escape = w ? (uint32_t)((1ull << w) - 1ull) : 0u;
+        wire[2 * g] = packed[5 * g];
+        wire[2 * g + 1] = packed[5 * g + 1];
+        const int64_t gw = n ? words_for(n - 1, w) : 0, ew = words_for(x, bi), iw = words_for(n, bi);
+        uint32_t at = packed[5 * g + 3];
+        int64_t e = 0;
         for (int64_t j = 0; j < n; ++j) {
-            if (j) at = at + get_bits(packed + in_at, (j - 1) * w, w) + 1u;
+            if (j) {
+                uint32_t gap = get_bits(packed + in_at, (j - 1) * w, w);
+                if (w && gap == escape) gap = get_bits(packed + in_at + gw, (e++) * bi, bi);
+                at = at + gap + 1u;
+            }
             put_bits(wire + out_at, j * bi, bi, at);
         }
-        const int64_t gw = n ? words_for(n - 1, w) : 0, iw = words_for(n, bi);
         const int64_t rest = payload_words(n, bi, bl, P.quantizer) - iw;
-        for (int64_t q = 0; q < rest; ++q) wire[out_at + iw + q] = packed[in_at + gw + q];
-        in_at += gw + rest;
+        for (int64_t q = 0; q < rest; ++q) wire[out_at + iw + q] = packed[in_at + gw + ew + q];
+        in_at += gw + ew + rest;
         out_at += iw + rest;
     }
 }
