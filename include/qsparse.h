@@ -270,13 +270,18 @@ int64_t qs_total_k(const qs_ctx* ctx);
  * Gap-coded records.  The paper measures what the workers send in bits (Section 5, the x-axes
  * of its figures) and leaves the coding of the k indices open.  qs_recode_gaps turns the
  * records of qs_pack / qs_sync_round into a second form in which a segment's ascending indices
- * travel as the first index and the gaps i_j - i_(j-1) - 1, in fields of w bits, w the bit
- * length of the segment's largest gap (0 when n <= 1 or all indices are consecutive);
- * qs_decode_gaps turns them back, word for word, for qs_unpack_accumulate.  Row of a worker:
- *   directory: nseg entries of four words (n, norm bits, w, first index) (the min/max
- *              quantizer keeps (min, max) in the first two, n = k);
- *   per segment: n - 1 gap fields of w bits, LSB first, padded to a word; then the streams
- *              that follow the indices in the plain record (signs, levels or values), unchanged.
+ * travel as the first index and the gaps i_j - i_(j-1) - 1 in fields of w bits.  For w >= 1 the
+ * field value E = 2^w - 1 is an escape: a gap >= E is sent as E and the gap itself follows, in
+ * order, among x exceptions of b_idx bits.  w = 0 (no fields) needs every gap to be 0.  The
+ * width is the one in 0 .. b_idx that makes (n - 1) w + x(w) b_idx smallest (the smallest such
+ * on a tie), so the form is never longer than the plain one by more than its 6 bits of width.
+ * qs_decode_gaps turns the rows back, word for word, for qs_unpack_accumulate.  Row of a worker:
+ *   directory: nseg entries of five words (n, norm bits, w, first index, x) (the min/max
+ *              quantizer keeps (min, max) in the first two, n = k; x is not counted as sent:
+ *              it could be recounted from the fields);
+ *   per segment: n - 1 gap fields of w bits, LSB first, padded to a word; x exception fields
+ *              of b_idx bits, padded to a word; then the streams that follow the indices in
+ *              the plain record (signs, levels or values), unchanged.
  * Words after a record, up to qs_gap_words, are zero.
  *   wire / stride_words     device, rows in the format of qs_pack (stride >= qs_wire_words)
  *   packed / packed_stride  device, rows of packed_stride >= qs_gap_words(ctx) words
@@ -285,10 +290,10 @@ int64_t qs_total_k(const qs_ctx* ctx);
  *                           worker of the job for qs_decode_gaps (the master's side, see
  *                           qs_set_sharding); rows of workers outside it are neither read nor written
  *   bits_out                device, one int64 per worker, or NULL: exact size in bits,
- *                           sum over segments of 64 + 6 + [n >= 1] (b_idx + (n - 1) w) + n (entry bits - b_idx)
+ *                           sum over segments of 64 + 6 + [n >= 1] (b_idx + (n - 1) w + x b_idx) + n (entry bits - b_idx)
  * Both calls are asynchronous on the context's stream, allocate nothing and keep no state; a
- * count above k_seg, a width above b_idx or a first index outside the segment in the input is
- * clipped (the words read and written stay inside the rows).  QS_CAPACITY (nothing written) when
+ * count above k_seg, a width above b_idx, more exceptions than fields or a first index outside
+ * the segment in the input is clipped (the words read and written stay inside the rows).  QS_CAPACITY (nothing written) when
  * a stride is too small.
  */
 int64_t qs_gap_words(const qs_ctx* ctx);

@@ -210,12 +210,13 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.nfb = (uint32_t)h_fb.size();
     c->wire_words = words;
     {
-        int64_t gw = 4 * (int64_t)nseg;
+        int64_t gw = 5 * (int64_t)nseg;
         uint64_t longest = 0, most = 0;
         for (int g = 0; g < nseg; ++g) {
             const uint32_t k = (uint32_t)kseg[g];
             const uint64_t all = streams_words(k, h_bi[g], (uint32_t)P.bl, P.qz);
-            gw += (int64_t)words_for(k - 1, h_bi[g]) + (int64_t)all - (int64_t)words_for(k, h_bi[g]);
+            // fields and exceptions together never exceed (k - 1) b_idx bits; two streams, each padded to a word
+            gw += (int64_t)words_for(k - 1, h_bi[g]) + 1 + (int64_t)all - (int64_t)words_for(k, h_bi[g]);
             longest = std::max<uint64_t>(longest, k);
             most = std::max<uint64_t>(most, all);
         }
@@ -287,8 +288,8 @@ int install_segments(qs_ctx* c, int nseg, const int64_t* offsets, const int64_t*
     P.guess = const_cast<uint32_t*>(g_up);
 #define AL(field, count, zero) if ((rc = dev_alloc(c, &P.field, (size_t)(count), zero)) != QS_OK) return rc
     AL(wary, P.U, true);
-    AL(gap_unit, (size_t)6 * MAX_R * nseg, true);
-    AL(gap_csum, (size_t)MAX_R * c->row_chunks, true);
+    AL(gap_unit, (size_t)gap_unit_words() * MAX_R * nseg, true);
+    AL(gap_csum, (size_t)2 * MAX_R * c->row_chunks, true);
     AL(stage, (size_t)R * P.cap, false);
     AL(tile_cnt, (size_t)R * P.nblk * BLK_TILES, true);
     AL(blk_count, (size_t)R * P.nblk, true);
@@ -612,9 +613,9 @@ int qs_recode_gaps(qs_ctx* c, const uint32_t* wire, int64_t stride_words, const 
     for (int i = 0; i < act.n; ++i)       // words after a record are zero
         QS_CUDA_TRY(c, cudaMemsetAsync(packed + (size_t)act.r[i] * packed_stride, 0, (size_t)c->gap_words * 4, c->st));
     const cudaError_t e = launch_recode_gaps(c->P, act, wire, stride_words, packed, packed_stride,
-                                             reinterpret_cast<long long*>(bits_out), c->longest_k, c->most_words, c->st);
+                                             reinterpret_cast<long long*>(bits_out), c->longest_k, c->most_words, c->row_chunks, c->st);
     if (e != cudaSuccess) return cuda_fail(c, e, "gap-coded records");
-    return after_launch(c, 4, "gap-coded records");
+    return after_launch(c, 6, "gap-coded records");
 }
 
 int qs_decode_gaps(qs_ctx* c, const uint32_t* packed, int64_t packed_stride, const uint8_t* worker_mask, uint32_t* wire,
@@ -629,7 +630,7 @@ int qs_decode_gaps(qs_ctx* c, const uint32_t* packed, int64_t packed_stride, con
     const cudaError_t e = launch_decode_gaps(c->P, act, packed, packed_stride, wire, stride_words, c->longest_k,
                                              c->most_words, c->row_chunks, c->st);
     if (e != cudaSuccess) return cuda_fail(c, e, "plain records from gap-coded ones");
-    return after_launch(c, 4, "plain records from gap-coded ones");
+    return after_launch(c, 6, "plain records from gap-coded ones");
 }
 
 int64_t qs_total_k(const qs_ctx* c) { return c ? (int64_t)c->P.K : (int64_t)QS_INVALID_ARG; }

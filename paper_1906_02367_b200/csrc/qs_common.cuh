@@ -87,8 +87,8 @@ struct Plan {
     // scratch
     uint32_t* guess;           // R x nseg, sort-key space
     uint32_t* wary;            // R x nseg: rounds for which the unit's prediction still aims wide after a miss
-    uint32_t* gap_unit;        // 6 x MAX_R x nseg: per-unit table of the gap-coded record's two directions
-    uint32_t* gap_csum;        // MAX_R x (K / 1024 + nseg + 1): chunk sums of the gap decoder
+    uint32_t* gap_unit;        // 40 x MAX_R x nseg: per-unit table and gap-length counts of the gap-coded record's two directions
+    uint32_t* gap_csum;        // 2 x MAX_R x (K / 1024 + nseg + 1): chunk sums (escapes, index distance) of the gap coder
     uint2* stage;              // R x cap (index, value bits): candidates as the dense pass left them, tile t at t * STILE
     uint32_t* tile_cnt;        // R x (nblk x BLK_TILES): rows padded to whole blocks, the padding stays zero
     uint32_t* blk_count;       // R x nblk, zero between rounds

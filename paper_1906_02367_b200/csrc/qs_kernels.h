@@ -23,9 +23,10 @@ void launch_export(const Plan& P, long long* sel_idx, int* level, uint8_t* sign,
 
 // qs_gaps.cu: plain records <-> gap-coded records
 uint32_t gap_chunk(void);
+uint32_t gap_unit_words(void);           // words of the per-unit table, per (worker, segment)
 cudaError_t launch_recode_gaps(const Plan& P, const Active& act, const uint32_t* wire, long long stride, uint32_t* out,
                                long long out_stride, long long* bits_out, uint32_t longest_k, uint32_t most_words,
-                               cudaStream_t st);
+                               uint32_t row_chunks, cudaStream_t st);
 cudaError_t launch_decode_gaps(const Plan& P, const Active& act, const uint32_t* packed, long long packed_stride,
                                uint32_t* wire, long long stride, uint32_t longest_k, uint32_t most_words,
                                uint32_t row_chunks, cudaStream_t st);
