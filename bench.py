@@ -755,7 +755,11 @@ def run_sharded(args):
     ctx = B.Context(count, d, int(kseg[0]), 1, B.QS_TOPK, B.QS_SIGN_L1, seed=0)
     ctx.bind(x, xw, mem)
     wire = ctx.new_wire()
-    job = sharded.ShardedRound(R, ctx, wire, rank=rank, world=world)
+    gap = {}
+    if args.gap_coded:                    # the records cross the all-gather in their gap-coded form
+        gap = dict(packed_local=torch.zeros((count, ctx.gap_words()), dtype=torch.int32, device=dev),
+                   records=torch.zeros((R, ctx.wire_words()), dtype=torch.int32, device=dev))
+    job = sharded.ShardedRound(R, ctx, wire, rank=rank, world=world, **gap)
 
     def drift():
         e1.exponential_(generator=gen)
@@ -791,7 +795,9 @@ def run_sharded(args):
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "strong", "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"ResNet-50-shaped round, R=8 workers over {world} GPU(s), d={d}, Top_k 0.1% flat, sign/l1; "
-                                   "separate calls with one all-gather of the records", "workers_per_gpu": count}}))
+                                   "separate calls with one all-gather of the records", "workers_per_gpu": count,
+                       "exchange": "gap-coded records" if args.gap_coded else "plain records",
+                       "words_exchanged_per_record": int(job.exchanged_words)}}))
     ctx.destroy()
     if world > 1:
         dist.destroy_process_group()
@@ -806,6 +812,7 @@ def main():
     ap.add_argument("--variant", default="flat", choices=["flat", "per_tensor", "paper_table", "async", "step", "sharded", "config3"])
     ap.add_argument("--shrink", type=int, default=1, help="divide every tensor size (profiling on a small case)")
     ap.add_argument("--sweep5", action="store_true", help="run the d = 2^28 ratio x s sweep instead of the headline workload")
+    ap.add_argument("--gap-coded", action="store_true", help="--variant sharded: exchange the records in their gap-coded form")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--headline-only", action="store_true", help="skip the other workloads (per tensor, config 3, config 5 sweep)")

@@ -47,13 +47,22 @@ class ShardedRound:
     """One rank's share of a job of R workers.  x is this rank's replica of the global model; xw, mem
     (and anchors) hold this rank's workers only."""
 
-    def __init__(self, R, engine, wire_local, rank=None, world=None, group=None, packed_local=None, records=None):
+    def __init__(self, R, engine, wire_local, rank=None, world=None, group=None, packed_local=None, records=None, nseg=1):
         """packed_local (R / G rows of qs_gap_words) and records (R rows of qs_wire_words) given: the
         records travel in their gap-coded form (qs_recode_gaps before the all-gather, qs_decode_gaps
-        after it), which is what shrinks the one collective of the round."""
+        after it).  Rows are sized for the longest record there can be; what crosses the collective
+        is cut to the longest record of the round (its bit count read back, the maximum agreed by a
+        one-word all-reduce), so the exchange shrinks with the records.  nseg: segments per record."""
         self.packed_local, self.records = packed_local, records
         if (packed_local is None) != (records is None):
             raise ValueError("gap-coded exchange needs both packed_local and records")
+        if packed_local is not None:
+            self.gap_bits = torch.zeros(packed_local.shape[0], dtype=torch.int64, device=packed_local.device)
+            self.packed_all = torch.zeros((int(R), packed_local.shape[1]), dtype=packed_local.dtype, device=packed_local.device)
+            # words of a record of b bits: each directory entry holds 5 words against the 70 bits counted
+            # for it, and each of a segment's streams (at most four) is padded to a word
+            self.slack_words = 7 * int(nseg)
+        self.exchanged_words = 0                  # per row, in the last round
         self.group = group
         self.world = world if world is not None else (dist.get_world_size(group) if dist.is_initialized() else 1)
         self.rank = rank if rank is not None else (dist.get_rank(group) if dist.is_initialized() else 0)
@@ -70,13 +79,23 @@ class ShardedRound:
             self.engine.compress_feedback(rnd, mine)
             self.engine.pack(self.wire_local, bits_out)
             if self.packed_local is not None:
-                self.engine.recode_gaps(self.wire_local, self.packed_local, mine)
+                self.gap_bits.zero_()
+                self.engine.recode_gaps(self.wire_local, self.packed_local, mine, self.gap_bits)
         if self.packed_local is not None:
-            packed = gather_records(self.packed_local, self.R, self.group)
-            self.engine.decode_gaps(packed, self.records, mask)
+            busy = mine is None or mine.any()
+            longest = (int(self.gap_bits.max().item()) + 31) // 32 + self.slack_words if busy else 0
+            width = torch.tensor([min(longest, self.packed_local.shape[1])], dtype=torch.int64, device=self.packed_local.device)
+            if self.world > 1:
+                dist.all_reduce(width, op=dist.ReduceOp.MAX, group=self.group)
+            w = int(width.item())
+            self.exchanged_words = w
+            if w:
+                self.packed_all[:, :w] = gather_records(self.packed_local[:, :w].contiguous(), self.R, self.group)
+            self.engine.decode_gaps(self.packed_all, self.records, mask)
             records = self.records
         else:
             records = gather_records(self.wire_local, self.R, self.group)
+            self.exchanged_words = int(self.wire_local.shape[1])
         self.engine.unpack_accumulate(records, mask)
         if mine is None or mine.any():
             self.engine.broadcast(mine)

@@ -93,7 +93,7 @@ class _OracleEngine:
         for r, w in self.records.items():
             wire_local[r] = torch.from_numpy(w.view("int32"))
 
-    def recode_gaps(self, wire_local, packed_local, mask):
+    def recode_gaps(self, wire_local, packed_local, mask, bits_out=None):
         local = self.O.Plan(self.xw.shape[0], self.plan.d, s=self.plan.s, sparsifier=self.plan.sparsifier,
                             quantizer=self.plan.quantizer, seed=self.plan.seed, offsets=self.plan.offsets, kseg=self.plan.kseg)
         out = self.O.recode_gaps(local, wire_local.numpy().view("uint32"), mask)
@@ -101,6 +101,8 @@ class _OracleEngine:
         for r in range(self.xw.shape[0]):
             if mask is None or mask[r]:
                 packed_local[r] = torch.from_numpy(out["packed"][r].view("int32"))
+                if bits_out is not None:
+                    bits_out[r] = int(out["bits"][r])
 
     def decode_gaps(self, packed, records, mask):
         out = self.O.decode_gaps(self.plan, packed.numpy().view("uint32"), mask)
@@ -141,6 +143,8 @@ def _sharded_main(rank, world, port, out, gap_coded):
     for rnd, mask in enumerate(masks):
         eng.xw += I.gaussian_drift(R, d, 8, rnd, std=1e-2)[base:base + count]
         job.round(rnd, mask)
+        if gap_coded:                     # what crossed the collective: the round's longest record, not the rows' capacity
+            assert 0 < job.exchanged_words <= O.gap_words(plan)
     out[rank] = (eng.x.tobytes(), eng.xw.tobytes(), eng.mem.tobytes(), eng.anchors.tobytes())
     dist.destroy_process_group()
 
